@@ -1,0 +1,223 @@
+/*
+ * akvs -- selective-recompute prefill with probe-guided per-unit KV offset correction,
+ * for one NVIDIA B200 (sm_100a).  Plain C ABI: POD structs, raw pointers, sizes.
+ *
+ * The method (paper Section 3, Algorithm 1): every memory unit is encoded once, alone, and
+ * its per-layer K/V cached.  For a request the retrieved units are concatenated in
+ * retrieval order and followed by the query.  At a check layer, per-token divergence
+ * scores between fresh and reused K/V pick, per unit, the top-b tokens by K score and the
+ * top-b by V score (b = ceil(r n)) and fix per-token weights w = min(score, 1).  From the
+ * check layer on only those probe tokens (and the query) are recomputed; per layer and
+ * unit the mean residual (fresh - reused) over the probes is the unit's offset, and every
+ * non-probe token of the unit gets reused + w * offset while probes keep their fresh state.
+ *
+ * Conventions
+ *  - every function returns AKVS_OK or a negative AKVS_ERR_*; nothing is launched when
+ *    validation fails; no exception or abort crosses this boundary;
+ *  - "device" pointers are CUDA global memory owned by the caller, "host" pointers are
+ *    ordinary host memory owned by the caller; the library allocates no device memory
+ *    (scratch comes from the caller's workspace);
+ *  - all work is enqueued on the caller's stream (a cudaStream_t passed as void*; NULL is
+ *    the default stream); only akvs_select_probes and akvs_check synchronise it;
+ *  - linear weights are row-major [out_features][in_features] (y = x W^T), no biases;
+ *  - model dtype AKVS_F32: weights, cache and outputs are float; AKVS_BF16: weights,
+ *    cache and K/V outputs are bfloat16 with float accumulation.  The residual stream
+ *    and `out_hidden` are float in both modes;
+ *  - K is cached AFTER RoPE at unit-local positions 0..n-1 (rotate-half pairing
+ *    (i, i + head_dim/2), angle p * rope_base^(-2i/head_dim)); reuse turns it through the
+ *    unit's global offset.  Residuals, offsets and corrected K live at global positions.
+ */
+#ifndef AKVS_H
+#define AKVS_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define AKVS_OK               0
+#define AKVS_ERR_INVALID_ARG (-1)  /* null pointer, negative size, value out of range      */
+#define AKVS_ERR_SHAPE       (-2)  /* model/cache/request shapes inconsistent or unsupported */
+#define AKVS_ERR_WORKSPACE   (-3)  /* workspace missing, misaligned (256 B) or too small     */
+#define AKVS_ERR_UNSUPPORTED (-4)  /* dtype / kv format / head_dim not handled               */
+#define AKVS_ERR_CUDA        (-5)  /* a CUDA runtime or driver call failed                    */
+#define AKVS_ERR_TIMEOUT     (-6)  /* a bounded device-side wait ran out (no hang, no trap)  */
+#define AKVS_ERR_NAN_SCORE   (-7)  /* a divergence score was NaN                             */
+
+#define AKVS_F32   0
+#define AKVS_BF16  1
+
+#define AKVS_KV_NATIVE 0           /* cache holds the model dtype                            */
+#define AKVS_KV_Q2     2           /* 2-bit codes, asymmetric min-max, groups of 64 along head_dim */
+#define AKVS_KV_Q4     4           /* 4-bit codes, same scheme                               */
+
+#define AKVS_MODE_CORRECTED 0      /* Algorithm 1                                            */
+#define AKVS_MODE_NAIVE     1      /* direct reuse (Section 3.1): only the query is computed */
+#define AKVS_MODE_FULL      2      /* full recompute of context + query (what is approximated) */
+
+/* Decoder description.  All pointers borrowed.  The nine per-layer arrays are HOST arrays
+ * of n_layers DEVICE pointers.  Pre-norm RMSNorm (gain vectors are float), GQA with
+ * q head i reading kv head i / (n_q_heads / n_kv_heads), SwiGLU MLP. */
+typedef struct akvs_model_desc {
+  int32_t n_layers, d_model, n_q_heads, n_kv_heads, head_dim, d_ff, vocab;
+  int32_t dtype;                      /* AKVS_F32 | AKVS_BF16                               */
+  float   rope_base, rms_eps;
+  const void*  tok_emb;               /* device [vocab][d_model], model dtype                */
+  const float* final_norm;            /* device [d_model]                                    */
+  const float* const* attn_norm;      /* [L] -> device [d_model]                             */
+  const void* const* wq;              /* [L] -> device [n_q_heads*head_dim][d_model]         */
+  const void* const* wk;              /* [L] -> device [n_kv_heads*head_dim][d_model]        */
+  const void* const* wv;              /* [L] -> device [n_kv_heads*head_dim][d_model]        */
+  const void* const* wo;              /* [L] -> device [d_model][n_q_heads*head_dim]         */
+  const float* const* mlp_norm;       /* [L] -> device [d_model]                             */
+  const void* const* w_gate;          /* [L] -> device [d_ff][d_model]                       */
+  const void* const* w_up;            /* [L] -> device [d_ff][d_model]                       */
+  const void* const* w_down;          /* [L] -> device [d_model][d_ff]                       */
+} akvs_model_desc;
+
+/* Unit store (Section 3.1: "encoded once").  Filled by akvs_encode_units, read-only to
+ * every other call (the same unit is reused under other contexts). */
+typedef struct akvs_cache {
+  int32_t n_units, n_tokens, kv_format;
+  const int32_t* unit_off;   /* host   [n_units+1], prefix sums of unit lengths, unit_off[0]=0 */
+  const int32_t* token_ids;  /* device [n_tokens], units back to back in store order          */
+  void* k;                   /* device [L][n_tokens][n_kv][head_dim] model dtype, or packed codes
+                                [L][n_tokens][n_kv][head_dim*bits/8] bytes (little-endian in a byte) */
+  void* v;                   /* same layout                                                    */
+  void* k_meta;              /* device half2 (scale, min) [L][n_tokens][n_kv][head_dim/64]; NULL if native */
+  void* v_meta;
+} akvs_cache;
+
+/* One request: which units, in which order (retrieval order differs per query), and the query. */
+typedef struct akvs_request {
+  int32_t n_units;
+  const int32_t* unit_ids;   /* host   [n_units], indices into the unit store                 */
+  int32_t n_query;
+  const int32_t* query_ids;  /* device [n_query]                                              */
+} akvs_request;
+
+/* Probe sets and weights (Section 3.3).  Every array is device memory allocated by the
+ * caller for n_ctx = total context tokens of the request; akvs_select_probes fills them and
+ * the three host counters.  A caller may overwrite the contents (for instance with sets
+ * chosen elsewhere) before akvs_prefill_corrected as long as the counters stay consistent. */
+typedef struct akvs_probes {
+  int32_t  n_ctx;            /* out: N                                                        */
+  int32_t  n_probe_rows;     /* out: P = | union of all S^K and S^V |                         */
+  int32_t  n_rows;           /* out: P + n_query                                              */
+  int32_t* ctx_off;          /* [n_units+1] global offset of each unit in this request        */
+  int32_t* probe_off;        /* [n_units+1] prefix sums of b_u (same for K and V sets)        */
+  int32_t* sk_idx;           /* [n_ctx] first probe_off[n_units] valid: S^K, global positions, ascending per unit */
+  int32_t* sv_idx;           /* [n_ctx] S^V likewise                                          */
+  float*   w_k;              /* [n_ctx] min(d_K, 1)                                           */
+  float*   w_v;              /* [n_ctx] min(d_V, 1)                                           */
+  float*   d_k;              /* [n_ctx] divergence scores at the check layer                  */
+  float*   d_v;              /* [n_ctx]                                                       */
+  int32_t* rows;             /* [n_ctx + n_query] recomputed rows: sorted probe positions, then the query positions */
+} akvs_probes;
+
+/* Bytes of workspace a request of this size needs (monotone in every argument).
+ * Workspace must be 256-byte aligned device memory; its contents carry state from
+ * akvs_select_probes to akvs_prefill_corrected of the same request. */
+int32_t akvs_workspace_bytes(const akvs_model_desc* model, int32_t n_ctx, int32_t n_query,
+                             int32_t n_units, int32_t check_layer, int64_t* out_bytes);
+
+/* Section 3.1 -- isolated encoding.  Runs every unit of cache->token_ids alone (positions
+ * 0..n_u-1, causal within the unit) through all layers and stores, per layer, K after RoPE
+ * at local positions and V, in cache->kv_format.  cache->unit_off/token_ids are inputs;
+ * cache->k/v (and *_meta when quantised) are outputs.  Asynchronous. */
+int32_t akvs_encode_units(const akvs_model_desc* model, akvs_cache* cache,
+                          void* workspace, int64_t ws_bytes, void* stream);
+
+/* Section 3.3, Algorithm 1 line 2 -- probe selection.  Computes layers 1..check_layer-1
+ * densely for all rows (context + query), then at the check layer the fresh K/V of every
+ * context token, the scores d_K, d_V against the re-aligned cache, per unit the top-b sets
+ * (b = ceil(n_u * refresh_bp / 10000), ties to the smaller index, indices ascending), the
+ * weights and the sorted row list.  check_layer is 1-based, 1 <= check_layer <= n_layers.
+ * Synchronises the stream once to return the row counts.  *ctx_inout: pass NULL-initialised
+ * storage the first time; the library creates (or reuses) a small host object that carries
+ * the request's state to akvs_prefill_corrected; release it with akvs_free. */
+int32_t akvs_select_probes(const akvs_model_desc* model, const akvs_cache* cache,
+                           const akvs_request* req, int32_t refresh_bp, int32_t check_layer,
+                           akvs_probes* out, void** ctx_inout,
+                           void* workspace, int64_t ws_bytes, void* stream);
+
+/* Algorithm 1 lines 3-9 around the decoder -- the prefill.
+ *  AKVS_MODE_CORRECTED: needs `probes` and the `ctx` of a preceding akvs_select_probes on
+ *    the same workspace.  From the check layer on, recomputes the rows in probes->rows,
+ *    estimates per-unit offsets from the probes, writes corrected K/V for the whole context.
+ *  AKVS_MODE_NAIVE: probes/ctx may be NULL; context K/V are the re-aligned cache.
+ *  AKVS_MODE_FULL:  probes/ctx may be NULL; everything recomputed (cache K/V unused).
+ * Outputs: out_hidden float [n_query][d_model] (after the final RMSNorm);
+ *          out_k, out_v [L][n_ctx+n_query][n_kv][head_dim] in the model dtype, K after
+ *          RoPE at global positions.  Asynchronous. */
+int32_t akvs_prefill_corrected(const akvs_model_desc* model, const akvs_cache* cache,
+                               const akvs_request* req, const akvs_probes* probes, int32_t mode,
+                               float* out_hidden, void* out_k, void* out_v,
+                               void* ctx, void* workspace, int64_t ws_bytes, void* stream);
+
+/* Releases the host object created by akvs_select_probes.  NULL is allowed. */
+void akvs_free(void* ctx);
+
+/* Synchronises `stream` and returns the device status word kept in `workspace`
+ * (AKVS_OK, AKVS_ERR_TIMEOUT, AKVS_ERR_NAN_SCORE), then clears it. */
+int32_t akvs_check(void* workspace, void* stream);
+
+/* Cross-check switch for the tests: 0 (default) routes bf16 linear layers to the tcgen05
+ * kernels, 1 to the CUDA-core kernels.  Process-wide; not part of the serving surface. */
+int32_t akvs_debug_set_linear_algo(int32_t algo);
+
+/* ------------------------------------------------------------------------------------
+ * Single steps of the path, exported so that each kernel can be checked on its own.
+ * dtype is AKVS_F32 or AKVS_BF16 and names the type of every `void*` tensor.
+ * All asynchronous on `stream`.
+ * ------------------------------------------------------------------------------------ */
+
+/* y[M][N] = x[M][K] * w[N][K]^T, float accumulation.  algo 0: the path's default for the
+ * dtype (tcgen05 tensor cores for bf16, CUDA cores for float); algo 1: CUDA cores. */
+int32_t akvs_op_linear(int32_t dtype, const void* x, const void* w, void* y,
+                       int32_t M, int32_t N, int32_t K, int32_t algo, void* stream);
+
+/* Rotate-half RoPE in place on x[n][n_heads][head_dim] at positions pos[n] (device). */
+int32_t akvs_op_rope(int32_t dtype, void* x, const int32_t* pos, int32_t n, int32_t n_heads,
+                     int32_t head_dim, float rope_base, void* stream);
+
+/* GQA attention: query row r sees key j iff k_lo[r] <= j <= k_hi[r] (device arrays, both
+ * non-decreasing in r).  q [R][n_q][hd], k/v [T][n_kv][hd], out [R][n_q][hd]. */
+int32_t akvs_op_attention(int32_t dtype, const void* q, const void* k, const void* v, void* out,
+                          const int32_t* k_lo, const int32_t* k_hi, int32_t R, int32_t T,
+                          int32_t n_q_heads, int32_t n_kv_heads, int32_t head_dim, int32_t algo, void* stream);
+
+/* Bytes of scratch that akvs_op_select and akvs_op_correct_layer need for these sizes. */
+int64_t akvs_op_scratch_bytes(int32_t n_ctx, int32_t n_query, int32_t n_units, int32_t head_dim);
+
+/* Section 3.3 selection from given scores: fills probe_off, sk_idx, sv_idx, w_k, w_v, rows
+ * (device) exactly as akvs_select_probes does; ctx_off is a HOST array [n_units+1].
+ * scratch: device, 256-byte aligned, akvs_op_scratch_bytes(...) bytes.  Synchronises the stream. */
+int32_t akvs_op_select(const float* d_k, const float* d_v, const int32_t* ctx_off_host, int32_t n_units,
+                       int32_t n_query, int32_t refresh_bp, akvs_probes* out, void* scratch, void* stream);
+
+/* One layer of Algorithm 1 lines 5-8 (mean estimation + correction) over a whole context.
+ * fresh_k/fresh_v [n_rows][n_kv][hd] hold the recomputed rows listed in probes->rows (K
+ * already rotated at global positions).  cache_k/cache_v (+meta) are ONE layer of a unit
+ * store; the request's token j reads store row src_tok[j] (device [n_ctx]).  Writes
+ * out_k/out_v [n_ctx+n_query][n_kv][hd] and the offsets mu_k, mu_v float [n_units][n_kv*hd].
+ * scratch: device, 256-byte aligned, akvs_op_scratch_bytes(...) bytes.  Synchronises the stream
+ * once (it reads the probe count back) before the kernels are enqueued. */
+int32_t akvs_op_correct_layer(int32_t dtype, int32_t kv_format,
+                              const void* cache_k, const void* cache_v, const void* k_meta, const void* v_meta,
+                              const int32_t* src_tok, const void* fresh_k, const void* fresh_v,
+                              const akvs_probes* probes, int32_t n_units, int32_t n_query,
+                              int32_t n_kv_heads, int32_t head_dim, float rope_base,
+                              void* out_k, void* out_v, float* mu_k, float* mu_v,
+                              void* scratch, void* stream);
+
+/* Group quantiser of the cache (asymmetric min-max, groups of 64 along head_dim, float16
+ * scale and minimum): x [n][n_kv][hd] -> codes [n][n_kv][hd*bits/8], meta half2 [n][n_kv][hd/64]. */
+int32_t akvs_op_quantize(int32_t dtype, const void* x, int32_t n, int32_t n_kv_heads, int32_t head_dim,
+                         int32_t bits, void* codes, void* meta, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* AKVS_H */

@@ -1,0 +1,155 @@
+// Shared device/host helpers for the akvs kernels (sm_100a only).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <stdint.h>
+
+#include "akvs.h"
+
+typedef __nv_bfloat16 bf16;
+
+#define AKVS_TRY(expr)                              \
+  do {                                              \
+    int32_t rc_ = (expr);                           \
+    if (rc_ != AKVS_OK) return rc_;                 \
+  } while (0)
+
+#define AKVS_CUDA(expr)                             \
+  do {                                              \
+    if ((expr) != cudaSuccess) return AKVS_ERR_CUDA; \
+  } while (0)
+
+#define AKVS_LAUNCHED()                             \
+  do {                                              \
+    if (cudaPeekAtLastError() != cudaSuccess) return AKVS_ERR_CUDA; \
+  } while (0)
+
+static inline int64_t akvs_align_up(int64_t x, int64_t a) { return (x + a - 1) / a * a; }
+static inline int akvs_cdiv(int64_t a, int64_t b) { return (int)((a + b - 1) / b); }
+
+// ---------------------------------------------------------------------------------------
+// 16-byte vector access: VEC elements of T <-> float registers.
+// ---------------------------------------------------------------------------------------
+template <typename T> struct VecOf;
+template <> struct VecOf<float> { static constexpr int N = 4; };
+template <> struct VecOf<bf16> { static constexpr int N = 8; };
+
+__device__ __forceinline__ void ld16(const float* p, float (&o)[4]) {
+  float4 v = *reinterpret_cast<const float4*>(p);
+  o[0] = v.x; o[1] = v.y; o[2] = v.z; o[3] = v.w;
+}
+__device__ __forceinline__ void st16(float* p, const float (&o)[4]) {
+  *reinterpret_cast<float4*>(p) = make_float4(o[0], o[1], o[2], o[3]);
+}
+__device__ __forceinline__ void ld16(const bf16* p, float (&o)[8]) {
+  uint4 v = *reinterpret_cast<const uint4*>(p);
+  const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    o[2 * i] = __uint_as_float(w[i] << 16);
+    o[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
+  }
+}
+__device__ __forceinline__ uint32_t pack_bf16x2(float a, float b) {
+  __nv_bfloat162 h = __floats2bfloat162_rn(a, b);   // .x = a (low half), .y = b
+  return *reinterpret_cast<uint32_t*>(&h);
+}
+__device__ __forceinline__ void st16(bf16* p, const float (&o)[8]) {
+  uint4 v;
+  v.x = pack_bf16x2(o[0], o[1]);
+  v.y = pack_bf16x2(o[2], o[3]);
+  v.z = pack_bf16x2(o[4], o[5]);
+  v.w = pack_bf16x2(o[6], o[7]);
+  *reinterpret_cast<uint4*>(p) = v;
+}
+
+__device__ __forceinline__ float to_f(float x) { return x; }
+__device__ __forceinline__ float to_f(bf16 x) { return __bfloat162float(x); }
+template <typename T> __device__ __forceinline__ T from_f(float x);
+template <> __device__ __forceinline__ float from_f<float>(float x) { return x; }
+template <> __device__ __forceinline__ bf16 from_f<bf16>(float x) { return __float2bfloat16_rn(x); }
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+  return v;
+}
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xFFFFFFFFu, v, o));
+  return v;
+}
+__device__ __forceinline__ float warp_min(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fminf(v, __shfl_xor_sync(0xFFFFFFFFu, v, o));
+  return v;
+}
+
+// Device status word: first error wins.
+__device__ __forceinline__ void set_status(int32_t* status, int32_t code) {
+  if (status) atomicCAS(status, 0, code);
+}
+
+// ---------------------------------------------------------------------------------------
+// Internal launchers (host).  All take the model dtype as a runtime value.
+// ---------------------------------------------------------------------------------------
+struct KvLayer {            // one layer of a unit store, as the correction kernels read it
+  const void* k;
+  const void* v;
+  const void* k_meta;       // half2 (scale, min) per 64-group, or null
+  const void* v_meta;
+  int fmt;                  // AKVS_KV_NATIVE | AKVS_KV_Q2 | AKVS_KV_Q4
+};
+
+struct ReqMaps {            // per-request index maps (device)
+  const int32_t* ctx_off;   // [M+1]
+  const int32_t* tok_unit;  // [N] unit slot of context token j
+  const int32_t* tok_src;   // [N] row of token j in the unit store
+  const int32_t* row_of_pos;// [T] index into the recomputed rows, or -1
+  const uint8_t* kflag;     // [N] 1 if j in S^K
+  const uint8_t* vflag;     // [N]
+};
+
+int32_t launch_embed(int dtype, const void* tok_emb, const int32_t* ids, const int32_t* gather, int n, int d,
+                     float* h, cudaStream_t st);
+int32_t launch_gather_rows(const float* src, const int32_t* rows, int n, int d, float* dst, cudaStream_t st);
+int32_t launch_rmsnorm(int out_dtype, const float* h, const float* gain, float eps, int n, int d, void* x,
+                       cudaStream_t st);
+int32_t launch_rope_table(float base, int hd, int n_pos, float2* table, cudaStream_t st);
+int32_t launch_rope(int dtype, void* x, const int32_t* pos, int n, int n_heads, int hd, int ld,
+                    const float2* table, float base, cudaStream_t st);
+int32_t launch_iota(int32_t* p, int n, int start, cudaStream_t st);
+int32_t launch_quantize(int dtype, const void* x, int n, int n_kv, int hd, int bits, void* codes, void* meta,
+                        cudaStream_t st);
+
+int32_t launch_linear_simt(int dtype, const void* x, const void* w, const void* w2, void* y, float* resid,
+                           int M, int N, int K, int ldy, cudaStream_t st);
+
+// bf16 tensor-core linear layers (gemm_tc.cu).  epi 0: out[i] = x w[i]^T; 1: out[0] (float) += x w[0]^T;
+// 2: out[0] = silu(x w[0]^T) * (x w[1]^T).
+int32_t launch_linear_tc(int epi, const void* x, int M, int K, int n_seg, const void* const* w, const int* n,
+                         void* const* out, const int* ldc, int32_t* status, cudaStream_t st);
+
+int32_t launch_attention_simt(int dtype, const void* q, const void* k, const void* v, void* out,
+                              const int32_t* k_lo, const int32_t* k_hi, int R, int n_q, int n_kv, int hd,
+                              cudaStream_t st);
+
+int32_t launch_tok_maps(const int32_t* ctx_off, const int32_t* slot_src_off, int M, int N, int32_t* tok_unit,
+                        int32_t* tok_src, cudaStream_t st);
+int32_t launch_row_maps(const int32_t* rows, int n_rows, const int32_t* sk_idx, const int32_t* sv_idx, int n_probe,
+                        int N, int T, int32_t* row_of_pos, uint8_t* kflag, uint8_t* vflag, cudaStream_t st);
+int32_t launch_scores(int dtype, const KvLayer& kv, const ReqMaps& maps, const void* k_fresh, const void* v_fresh,
+                      int N, int n_kv, int hd, const float2* table, float* d_k, float* d_v, cudaStream_t st);
+int32_t launch_select(const float* d_k, const float* d_v, const int32_t* ctx_off, const int32_t* probe_off, int M,
+                      int N, int n_query, int32_t* sk_idx, int32_t* sv_idx, float* w_k, float* w_v, int32_t* rows,
+                      uint64_t* keys /*[2N]*/, uint8_t* flags /*[2N]*/, int32_t* counts /*[2]*/, int32_t* status,
+                      cudaStream_t st);
+int32_t launch_offsets(int dtype, const KvLayer& kv, const ReqMaps& maps, const int32_t* probe_off,
+                       const int32_t* sk_idx, const int32_t* sv_idx, const void* k_fresh, const void* v_fresh, int M,
+                       int n_kv, int hd, const float2* table, float* mu_k, float* mu_v, cudaStream_t st);
+int32_t launch_correct(int dtype, const KvLayer& kv, const ReqMaps& maps, const void* k_fresh, const void* v_fresh,
+                       const float* w_k, const float* w_v, const float* mu_k, const float* mu_v, int N, int n_query,
+                       int n_probe_rows, int n_kv, int hd, const float2* table, void* out_k, void* out_v,
+                       cudaStream_t st);

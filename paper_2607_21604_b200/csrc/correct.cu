@@ -1,0 +1,512 @@
+// Probe selection, per-unit offset estimation and the correction pass
+// (paper Section 3.3 and Algorithm 1 lines 2, 5-8).
+//
+// Layouts: fresh rows [n_rows][n_kv][hd]; one layer of the unit store [store_tok][n_kv][hd]
+// (model dtype) or packed 2/4-bit codes with half2 (scale, min) per 64-dim group;
+// outputs [T][n_kv][hd].  A "pair chunk" is a 16-byte vector of the lower half of a head
+// together with its RoPE partner 16 bytes in the upper half; one thread owns one pair chunk
+// so that the re-alignment rotation needs no exchange between threads and every global
+// access is a full 16-byte vector.
+#include "common.cuh"
+
+// ---------------------------------------------------------------------------------------
+// Reading one pair chunk of the reused K or V of store row `src`, head `h`, chunk `c`.
+// ---------------------------------------------------------------------------------------
+template <int BYTES>
+__device__ __forceinline__ uint32_t ld_codes(const uint8_t* p) {
+  if constexpr (BYTES == 4) return *reinterpret_cast<const uint32_t*>(p);
+  else if constexpr (BYTES == 2) return *reinterpret_cast<const uint16_t*>(p);
+  else return *p;
+}
+
+template <typename T, int FMT>
+__device__ __forceinline__ void load_cached_chunk(const void* base, const void* meta, int64_t src, int n_kv, int hd,
+                                                  int h, int dim0, float (&out)[VecOf<T>::N]) {
+  constexpr int V = VecOf<T>::N;
+  if constexpr (FMT == AKVS_KV_NATIVE) {
+    ld16(reinterpret_cast<const T*>(base) + ((size_t)src * n_kv + h) * hd + dim0, out);
+  } else {
+    constexpr int BITS = FMT;
+    constexpr int BYTES = V * BITS / 8;
+    const uint8_t* cp = reinterpret_cast<const uint8_t*>(base) + (((size_t)src * n_kv + h) * hd + dim0) * BITS / 8;
+    const uint32_t packed = ld_codes<BYTES>(cp);
+    const __half2 sm = reinterpret_cast<const __half2*>(meta)[((size_t)src * n_kv + h) * (hd / 64) + dim0 / 64];
+    const float s = __low2float(sm), m = __high2float(sm);
+#pragma unroll
+    for (int i = 0; i < V; ++i)
+      out[i] = __fmaf_rn((float)((packed >> (BITS * i)) & ((1u << BITS) - 1u)), s, m);
+  }
+}
+
+// ---------------------------------------------------------------------------------------
+// Index maps of a request.
+// ---------------------------------------------------------------------------------------
+__global__ void tok_maps_kernel(const int32_t* __restrict__ ctx_off, const int32_t* __restrict__ slot_src_off, int M,
+                                int N, int32_t* __restrict__ tok_unit, int32_t* __restrict__ tok_src) {
+  const int j = blockIdx.x * blockDim.x + threadIdx.x;
+  if (j >= N) return;
+  int lo = 0, hi = M;                 // largest u with ctx_off[u] <= j (empty units skipped)
+  while (hi - lo > 1) {
+    const int mid = (lo + hi) >> 1;
+    if (ctx_off[mid] <= j) lo = mid; else hi = mid;
+  }
+  tok_unit[j] = lo;
+  tok_src[j] = slot_src_off[lo] + (j - ctx_off[lo]);
+}
+
+int32_t launch_tok_maps(const int32_t* ctx_off, const int32_t* slot_src_off, int M, int N, int32_t* tok_unit,
+                        int32_t* tok_src, cudaStream_t st) {
+  if (N == 0) return AKVS_OK;
+  tok_maps_kernel<<<akvs_cdiv(N, 256), 256, 0, st>>>(ctx_off, slot_src_off, M, N, tok_unit, tok_src);
+  AKVS_LAUNCHED();
+  return AKVS_OK;
+}
+
+__global__ void row_maps_clear_kernel(int N, int T, int32_t* __restrict__ row_of_pos, uint8_t* __restrict__ kflag,
+                                      uint8_t* __restrict__ vflag) {
+  const int j = blockIdx.x * blockDim.x + threadIdx.x;
+  if (j < T) row_of_pos[j] = -1;
+  if (j < N) { kflag[j] = 0; vflag[j] = 0; }
+}
+__global__ void row_maps_fill_kernel(const int32_t* __restrict__ rows, int n_rows, const int32_t* __restrict__ sk_idx,
+                                     const int32_t* __restrict__ sv_idx, int n_probe, int N, int T,
+                                     int32_t* __restrict__ row_of_pos, uint8_t* __restrict__ kflag,
+                                     uint8_t* __restrict__ vflag) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n_rows) { const int p = rows[i]; if (p >= 0 && p < T) row_of_pos[p] = i; }
+  if (i < n_probe) {
+    const int a = sk_idx[i], b = sv_idx[i];
+    if (a >= 0 && a < N) kflag[a] = 1;
+    if (b >= 0 && b < N) vflag[b] = 1;
+  }
+}
+
+int32_t launch_row_maps(const int32_t* rows, int n_rows, const int32_t* sk_idx, const int32_t* sv_idx, int n_probe,
+                        int N, int T, int32_t* row_of_pos, uint8_t* kflag, uint8_t* vflag, cudaStream_t st) {
+  if (T == 0) return AKVS_OK;
+  row_maps_clear_kernel<<<akvs_cdiv(T, 256), 256, 0, st>>>(N, T, row_of_pos, kflag, vflag);
+  AKVS_LAUNCHED();
+  const int m = n_rows > n_probe ? n_rows : n_probe;
+  if (m > 0) {
+    row_maps_fill_kernel<<<akvs_cdiv(m, 256), 256, 0, st>>>(rows, n_rows, sk_idx, sv_idx, n_probe, N, T, row_of_pos,
+                                                            kflag, vflag);
+    AKVS_LAUNCHED();
+  }
+  return AKVS_OK;
+}
+
+// ---------------------------------------------------------------------------------------
+// Divergence scores at the check layer (Section 3.3): one warp per context token,
+// d_K = || k_fresh - Rot(off_u) k_cached ||_2 over all kv heads, d_V likewise.
+// ---------------------------------------------------------------------------------------
+template <typename T, int FMT>
+__global__ void scores_kernel(KvLayer kv, ReqMaps maps, const T* __restrict__ k_fresh, const T* __restrict__ v_fresh,
+                              int N, int n_kv, int hd, const float2* __restrict__ table, float* __restrict__ d_k,
+                              float* __restrict__ d_v) {
+  constexpr int V = VecOf<T>::N;
+  const int j = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (j >= N) return;
+  const int lane = threadIdx.x & 31;
+  const int half = hd / 2, ch = half / V;
+  const int u = maps.tok_unit[j];
+  const int64_t src = maps.tok_src[j];
+  const float2* rot = table + (size_t)maps.ctx_off[u] * half;
+  float sk = 0.f, sv = 0.f;
+  for (int pc = lane; pc < n_kv * ch; pc += 32) {
+    const int h = pc / ch, c = pc % ch;
+    float lo[V], hi[V], flo[V], fhi[V];
+    load_cached_chunk<T, FMT>(kv.k, kv.k_meta, src, n_kv, hd, h, c * V, lo);
+    load_cached_chunk<T, FMT>(kv.k, kv.k_meta, src, n_kv, hd, h, half + c * V, hi);
+    const T* fp = k_fresh + ((size_t)j * n_kv + h) * hd + c * V;
+    ld16(fp, flo);
+    ld16(fp + half, fhi);
+#pragma unroll
+    for (int i = 0; i < V; ++i) {
+      const float2 t = rot[c * V + i];
+      const float a = flo[i] - (lo[i] * t.x - hi[i] * t.y);
+      const float b = fhi[i] - (hi[i] * t.x + lo[i] * t.y);
+      sk += a * a + b * b;
+    }
+    load_cached_chunk<T, FMT>(kv.v, kv.v_meta, src, n_kv, hd, h, c * V, lo);
+    load_cached_chunk<T, FMT>(kv.v, kv.v_meta, src, n_kv, hd, h, half + c * V, hi);
+    const T* vp = v_fresh + ((size_t)j * n_kv + h) * hd + c * V;
+    ld16(vp, flo);
+    ld16(vp + half, fhi);
+#pragma unroll
+    for (int i = 0; i < V; ++i) {
+      const float a = flo[i] - lo[i], b = fhi[i] - hi[i];
+      sv += a * a + b * b;
+    }
+  }
+  sk = warp_sum(sk);
+  sv = warp_sum(sv);
+  if (lane == 0) { d_k[j] = sqrtf(sk); d_v[j] = sqrtf(sv); }
+}
+
+#define DISPATCH_T_FMT(KERNEL, GRID, BLOCK, SMEM, ST, ...)                                          \
+  do {                                                                                              \
+    if (dtype == AKVS_F32) {                                                                        \
+      if (kv.fmt == AKVS_KV_NATIVE) KERNEL<float, AKVS_KV_NATIVE><<<GRID, BLOCK, SMEM, ST>>>(__VA_ARGS__); \
+      else if (kv.fmt == AKVS_KV_Q4) KERNEL<float, AKVS_KV_Q4><<<GRID, BLOCK, SMEM, ST>>>(__VA_ARGS__);     \
+      else KERNEL<float, AKVS_KV_Q2><<<GRID, BLOCK, SMEM, ST>>>(__VA_ARGS__);                       \
+    } else {                                                                                        \
+      if (kv.fmt == AKVS_KV_NATIVE) KERNEL<bf16, AKVS_KV_NATIVE><<<GRID, BLOCK, SMEM, ST>>>(__VA_ARGS__);  \
+      else if (kv.fmt == AKVS_KV_Q4) KERNEL<bf16, AKVS_KV_Q4><<<GRID, BLOCK, SMEM, ST>>>(__VA_ARGS__);      \
+      else KERNEL<bf16, AKVS_KV_Q2><<<GRID, BLOCK, SMEM, ST>>>(__VA_ARGS__);                        \
+    }                                                                                               \
+  } while (0)
+
+static int32_t check_kv_shape(int dtype, const KvLayer& kv, int hd) {
+  const int V = dtype == AKVS_F32 ? 4 : 8;
+  if (hd % (2 * V) != 0) return AKVS_ERR_UNSUPPORTED;
+  if (kv.fmt != AKVS_KV_NATIVE && kv.fmt != AKVS_KV_Q4 && kv.fmt != AKVS_KV_Q2) return AKVS_ERR_UNSUPPORTED;
+  if (kv.fmt != AKVS_KV_NATIVE && (hd % 64 != 0 || !kv.k_meta || !kv.v_meta)) return AKVS_ERR_UNSUPPORTED;
+  return AKVS_OK;
+}
+
+int32_t launch_scores(int dtype, const KvLayer& kv, const ReqMaps& maps, const void* k_fresh, const void* v_fresh,
+                      int N, int n_kv, int hd, const float2* table, float* d_k, float* d_v, cudaStream_t st) {
+  if (N == 0) return AKVS_OK;
+  AKVS_TRY(check_kv_shape(dtype, kv, hd));
+  const int grid = akvs_cdiv(N, 8);
+  if (dtype == AKVS_F32) {
+    const float *kf = (const float*)k_fresh, *vf = (const float*)v_fresh;
+    if (kv.fmt == AKVS_KV_NATIVE) scores_kernel<float, AKVS_KV_NATIVE><<<grid, 256, 0, st>>>(kv, maps, kf, vf, N, n_kv, hd, table, d_k, d_v);
+    else if (kv.fmt == AKVS_KV_Q4) scores_kernel<float, AKVS_KV_Q4><<<grid, 256, 0, st>>>(kv, maps, kf, vf, N, n_kv, hd, table, d_k, d_v);
+    else scores_kernel<float, AKVS_KV_Q2><<<grid, 256, 0, st>>>(kv, maps, kf, vf, N, n_kv, hd, table, d_k, d_v);
+  } else {
+    const bf16 *kf = (const bf16*)k_fresh, *vf = (const bf16*)v_fresh;
+    if (kv.fmt == AKVS_KV_NATIVE) scores_kernel<bf16, AKVS_KV_NATIVE><<<grid, 256, 0, st>>>(kv, maps, kf, vf, N, n_kv, hd, table, d_k, d_v);
+    else if (kv.fmt == AKVS_KV_Q4) scores_kernel<bf16, AKVS_KV_Q4><<<grid, 256, 0, st>>>(kv, maps, kf, vf, N, n_kv, hd, table, d_k, d_v);
+    else scores_kernel<bf16, AKVS_KV_Q2><<<grid, 256, 0, st>>>(kv, maps, kf, vf, N, n_kv, hd, table, d_k, d_v);
+  }
+  AKVS_LAUNCHED();
+  return AKVS_OK;
+}
+
+// ---------------------------------------------------------------------------------------
+// Top-b selection (Section 3.3).  Order: larger score first, equal scores by smaller token
+// index; -0.0 counts as +0.0; NaN raises the status word.  Scores are non-negative, so the
+// float bit pattern orders them; key = (~bits << 32) | local index sorts ascending into the
+// wanted order and is unique, hence rank = #{keys smaller} and "rank < b" is the set.
+// ---------------------------------------------------------------------------------------
+__global__ void select_keys_kernel(const float* __restrict__ d_k, const float* __restrict__ d_v,
+                                   const int32_t* __restrict__ ctx_off, int M, int N, uint64_t* __restrict__ keys,
+                                   float* __restrict__ w_k, float* __restrict__ w_v, int32_t* status) {
+  const int j = blockIdx.x * blockDim.x + threadIdx.x;
+  if (j >= N) return;
+  int lo = 0, hi = M;
+  while (hi - lo > 1) {
+    const int mid = (lo + hi) >> 1;
+    if (ctx_off[mid] <= j) lo = mid; else hi = mid;
+  }
+  const uint32_t local = (uint32_t)(j - ctx_off[lo]);
+  const float a = d_k[j] + 0.0f, b = d_v[j] + 0.0f;
+  if (a != a || b != b) set_status(status, AKVS_ERR_NAN_SCORE);
+  keys[j] = ((uint64_t)(~__float_as_uint(a)) << 32) | local;
+  keys[N + j] = ((uint64_t)(~__float_as_uint(b)) << 32) | local;
+  w_k[j] = fminf(a, 1.0f);
+  w_v[j] = fminf(b, 1.0f);
+}
+
+constexpr int SEL_THREADS = 256;
+constexpr int SEL_TILE = 1024;
+
+// grid (M, 2): unit u, set s (0 = K, 1 = V).
+__global__ void __launch_bounds__(SEL_THREADS)
+select_rank_kernel(const uint64_t* __restrict__ keys, const int32_t* __restrict__ ctx_off,
+                   const int32_t* __restrict__ probe_off, int N, uint8_t* __restrict__ flags,
+                   int32_t* __restrict__ sk_idx, int32_t* __restrict__ sv_idx) {
+  __shared__ uint64_t tile[SEL_TILE];
+  __shared__ int warp_tot[SEL_THREADS / 32];
+  __shared__ int carry;
+  const int u = blockIdx.x, s = blockIdx.y;
+  const int a = ctx_off[u], n = ctx_off[u + 1] - a;
+  const int b = probe_off[u + 1] - probe_off[u];
+  const uint64_t* key = keys + (size_t)s * N + a;
+  uint8_t* flag = flags + (size_t)s * N + a;
+  int32_t* out = (s == 0 ? sk_idx : sv_idx) + probe_off[u];
+
+  // ranks, SEL_THREADS tokens at a time against key tiles staged in shared memory
+  for (int j0 = 0; j0 < n; j0 += SEL_THREADS) {
+    const int j = j0 + threadIdx.x;
+    const uint64_t mine = j < n ? key[j] : 0;
+    int rank = 0;
+    for (int t0 = 0; t0 < n; t0 += SEL_TILE) {
+      const int tn = min(SEL_TILE, n - t0);
+      __syncthreads();
+      for (int i = threadIdx.x; i < tn; i += SEL_THREADS) tile[i] = key[t0 + i];
+      __syncthreads();
+      if (j < n)
+        for (int i = 0; i < tn; ++i) rank += tile[i] < mine;
+    }
+    if (j < n) flag[j] = rank < b;
+  }
+  __syncthreads();
+  // compaction in ascending token order: block scan over the flags
+  if (threadIdx.x == 0) carry = 0;
+  __syncthreads();
+  const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+  for (int j0 = 0; j0 < n; j0 += SEL_THREADS) {
+    const int j = j0 + threadIdx.x;
+    const int f = j < n ? flag[j] : 0;
+    int incl = f;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int t = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+      if (lane >= o) incl += t;
+    }
+    if (lane == 31) warp_tot[wid] = incl;
+    __syncthreads();
+    int before = carry;
+    for (int w = 0; w < wid; ++w) before += warp_tot[w];
+    if (f) out[before + incl - 1] = a + j;
+    __syncthreads();
+    if (threadIdx.x == SEL_THREADS - 1) carry = before + incl;
+    __syncthreads();
+  }
+}
+
+// One CTA: rows = sorted union of both flag sets, then the query positions.
+__global__ void __launch_bounds__(1024)
+select_rows_kernel(const uint8_t* __restrict__ flags, int N, int n_query, int32_t* __restrict__ rows,
+                   int32_t* __restrict__ counts) {
+  __shared__ int warp_tot[32];
+  __shared__ int carry;
+  if (threadIdx.x == 0) carry = 0;
+  __syncthreads();
+  const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+  for (int j0 = 0; j0 < N; j0 += 1024) {
+    const int j = j0 + threadIdx.x;
+    const int f = j < N ? (flags[j] | flags[N + j]) : 0;
+    int incl = f;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int t = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+      if (lane >= o) incl += t;
+    }
+    if (lane == 31) warp_tot[wid] = incl;
+    __syncthreads();
+    int before = carry;
+    for (int w = 0; w < wid; ++w) before += warp_tot[w];
+    if (f) rows[before + incl - 1] = j;
+    __syncthreads();
+    if (threadIdx.x == 1023) carry = before + incl;
+    __syncthreads();
+  }
+  const int P = carry;
+  for (int i = threadIdx.x; i < n_query; i += 1024) rows[P + i] = N + i;
+  if (threadIdx.x == 0) { counts[0] = P; counts[1] = P + n_query; }
+}
+
+int32_t launch_select(const float* d_k, const float* d_v, const int32_t* ctx_off, const int32_t* probe_off, int M,
+                      int N, int n_query, int32_t* sk_idx, int32_t* sv_idx, float* w_k, float* w_v, int32_t* rows,
+                      uint64_t* keys, uint8_t* flags, int32_t* counts, int32_t* status, cudaStream_t st) {
+  if (N > 0) {
+    select_keys_kernel<<<akvs_cdiv(N, 256), 256, 0, st>>>(d_k, d_v, ctx_off, M, N, keys, w_k, w_v, status);
+    AKVS_LAUNCHED();
+    select_rank_kernel<<<dim3(M, 2), SEL_THREADS, 0, st>>>(keys, ctx_off, probe_off, N, flags, sk_idx, sv_idx);
+    AKVS_LAUNCHED();
+  }
+  select_rows_kernel<<<1, 1024, 0, st>>>(flags, N, n_query, rows, counts);
+  AKVS_LAUNCHED();
+  return AKVS_OK;
+}
+
+// ---------------------------------------------------------------------------------------
+// Mean estimation (Section 3.3; Algorithm 1 line 5): mu_u = (1/b_u) sum_{j in S_u} (fresh_j -
+// reuse_j).  One CTA per (unit, kv head, K|V); each warp takes every 8th probe, lanes own
+// rotation pairs; warps are combined through shared memory in a fixed order.
+// ---------------------------------------------------------------------------------------
+constexpr int OFF_WARPS = 8;
+
+template <typename T, int FMT>
+__global__ void __launch_bounds__(OFF_WARPS * 32)
+offsets_kernel(KvLayer kv, ReqMaps maps, const int32_t* __restrict__ probe_off, const int32_t* __restrict__ sk_idx,
+               const int32_t* __restrict__ sv_idx, const T* __restrict__ k_fresh, const T* __restrict__ v_fresh,
+               int n_kv, int hd, const float2* __restrict__ table, float* __restrict__ mu_k, float* __restrict__ mu_v) {
+  extern __shared__ float part[];                 // [OFF_WARPS][hd]
+  const int u = blockIdx.x, h = blockIdx.y, is_v = blockIdx.z;
+  const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+  const int half = hd / 2;
+  const int p0 = probe_off[u], b = probe_off[u + 1] - p0;
+  const int32_t* S = (is_v ? sv_idx : sk_idx) + p0;
+  const float2* rot = table + (size_t)maps.ctx_off[u] * half;
+  const T* fresh = is_v ? v_fresh : k_fresh;
+  const void* cbase = is_v ? kv.v : kv.k;
+  const void* cmeta = is_v ? kv.v_meta : kv.k_meta;
+
+  for (int e = lane; e < half; e += 32) { part[wid * hd + e] = 0.f; part[wid * hd + half + e] = 0.f; }
+  for (int i = wid; i < b; i += OFF_WARPS) {
+    const int j = S[i];
+    const int row = maps.row_of_pos[j];
+    const int64_t src = maps.tok_src[j];
+    if (row < 0) continue;                         // inconsistent caller-supplied sets: skip
+    const T* fp = fresh + ((size_t)row * n_kv + h) * hd;
+    for (int e = lane; e < half; e += 32) {
+      float lo, hi;
+      if constexpr (FMT == AKVS_KV_NATIVE) {
+        const T* cp = reinterpret_cast<const T*>(cbase) + ((size_t)src * n_kv + h) * hd;
+        lo = to_f(cp[e]);
+        hi = to_f(cp[half + e]);
+      } else {
+        const uint8_t* cp = reinterpret_cast<const uint8_t*>(cbase) + ((size_t)src * n_kv + h) * hd * FMT / 8;
+        const __half2* mp = reinterpret_cast<const __half2*>(cmeta) + ((size_t)src * n_kv + h) * (hd / 64);
+        const int e2 = half + e;
+        const uint32_t qa = (cp[e * FMT / 8] >> ((e * FMT) & 7)) & ((1u << FMT) - 1u);
+        const uint32_t qb = (cp[e2 * FMT / 8] >> ((e2 * FMT) & 7)) & ((1u << FMT) - 1u);
+        const __half2 ma = mp[e / 64], mb = mp[e2 / 64];
+        lo = __fmaf_rn((float)qa, __low2float(ma), __high2float(ma));
+        hi = __fmaf_rn((float)qb, __low2float(mb), __high2float(mb));
+      }
+      if (!is_v) {
+        const float2 t = rot[e];
+        const float rlo = lo * t.x - hi * t.y, rhi = hi * t.x + lo * t.y;
+        lo = rlo;
+        hi = rhi;
+      }
+      part[wid * hd + e] += to_f(fp[e]) - lo;
+      part[wid * hd + half + e] += to_f(fp[half + e]) - hi;
+    }
+  }
+  __syncthreads();
+  float* mu = (is_v ? mu_v : mu_k) + ((size_t)u * n_kv + h) * hd;
+  for (int e = threadIdx.x; e < hd; e += OFF_WARPS * 32) {
+    float s = 0.f;
+#pragma unroll
+    for (int w = 0; w < OFF_WARPS; ++w) s += part[w * hd + e];
+    mu[e] = b > 0 ? s / (float)b : 0.f;
+  }
+}
+
+int32_t launch_offsets(int dtype, const KvLayer& kv, const ReqMaps& maps, const int32_t* probe_off,
+                       const int32_t* sk_idx, const int32_t* sv_idx, const void* k_fresh, const void* v_fresh, int M,
+                       int n_kv, int hd, const float2* table, float* mu_k, float* mu_v, cudaStream_t st) {
+  if (M == 0) return AKVS_OK;
+  AKVS_TRY(check_kv_shape(dtype, kv, hd));
+  const dim3 grid(M, n_kv, 2);
+  const size_t smem = (size_t)OFF_WARPS * hd * sizeof(float);
+  if (dtype == AKVS_F32) {
+    const float *kf = (const float*)k_fresh, *vf = (const float*)v_fresh;
+    if (kv.fmt == AKVS_KV_NATIVE) offsets_kernel<float, AKVS_KV_NATIVE><<<grid, OFF_WARPS * 32, smem, st>>>(kv, maps, probe_off, sk_idx, sv_idx, kf, vf, n_kv, hd, table, mu_k, mu_v);
+    else if (kv.fmt == AKVS_KV_Q4) offsets_kernel<float, AKVS_KV_Q4><<<grid, OFF_WARPS * 32, smem, st>>>(kv, maps, probe_off, sk_idx, sv_idx, kf, vf, n_kv, hd, table, mu_k, mu_v);
+    else offsets_kernel<float, AKVS_KV_Q2><<<grid, OFF_WARPS * 32, smem, st>>>(kv, maps, probe_off, sk_idx, sv_idx, kf, vf, n_kv, hd, table, mu_k, mu_v);
+  } else {
+    const bf16 *kf = (const bf16*)k_fresh, *vf = (const bf16*)v_fresh;
+    if (kv.fmt == AKVS_KV_NATIVE) offsets_kernel<bf16, AKVS_KV_NATIVE><<<grid, OFF_WARPS * 32, smem, st>>>(kv, maps, probe_off, sk_idx, sv_idx, kf, vf, n_kv, hd, table, mu_k, mu_v);
+    else if (kv.fmt == AKVS_KV_Q4) offsets_kernel<bf16, AKVS_KV_Q4><<<grid, OFF_WARPS * 32, smem, st>>>(kv, maps, probe_off, sk_idx, sv_idx, kf, vf, n_kv, hd, table, mu_k, mu_v);
+    else offsets_kernel<bf16, AKVS_KV_Q2><<<grid, OFF_WARPS * 32, smem, st>>>(kv, maps, probe_off, sk_idx, sv_idx, kf, vf, n_kv, hd, table, mu_k, mu_v);
+  }
+  AKVS_LAUNCHED();
+  return AKVS_OK;
+}
+
+// ---------------------------------------------------------------------------------------
+// Correction pass (Algorithm 1 lines 6-8) fused with dequantisation and re-alignment:
+//   context token j of unit u, not in S^K:  K_out = Rot(off_u) deq(K_cached) + w_K[j] mu_K[u]
+//                              in S^K:      K_out = fresh K of its recomputed row
+//   V likewise with S^V (no rotation);  query token i: fresh K/V of row P + i.
+// One thread per pair chunk; it moves 4 x 16 B in and 4 x 16 B out.
+// ---------------------------------------------------------------------------------------
+template <typename T, int FMT>
+__global__ void __launch_bounds__(256)
+correct_kernel(KvLayer kv, ReqMaps maps, const T* __restrict__ k_fresh, const T* __restrict__ v_fresh,
+               const float* __restrict__ w_k, const float* __restrict__ w_v, const float* __restrict__ mu_k,
+               const float* __restrict__ mu_v, int N, int T_tok, int n_probe_rows, int n_kv, int hd,
+               const float2* __restrict__ table, T* __restrict__ out_k, T* __restrict__ out_v) {
+  constexpr int V = VecOf<T>::N;
+  const int half = hd / 2, ch = half / V;
+  const int64_t total = (int64_t)T_tok * n_kv * ch;
+  for (int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
+       idx += (int64_t)gridDim.x * blockDim.x) {
+    const int c = (int)(idx % ch);
+    const int h = (int)((idx / ch) % n_kv);
+    const int j = (int)(idx / ((int64_t)ch * n_kv));
+    const size_t o = ((size_t)j * n_kv + h) * hd + c * V;
+    float lo[V], hi[V];
+    int row_k = -1, row_v = -1, u = 0;
+    int64_t src = 0;
+    float wk = 0.f, wv = 0.f;
+    if (j >= N) {
+      row_k = row_v = n_probe_rows + (j - N);
+    } else {
+      const int row = maps.row_of_pos[j];
+      if (maps.kflag[j]) row_k = row;
+      if (maps.vflag[j]) row_v = row;
+      u = maps.tok_unit[j];
+      src = maps.tok_src[j];
+      if (w_k) { wk = w_k[j]; wv = w_v[j]; }
+    }
+    // ---- K
+    if (row_k >= 0) {
+      const T* fp = k_fresh + ((size_t)row_k * n_kv + h) * hd + c * V;
+      ld16(fp, lo);
+      ld16(fp + half, hi);
+    } else {
+      float clo[V], chi[V];
+      load_cached_chunk<T, FMT>(kv.k, kv.k_meta, src, n_kv, hd, h, c * V, clo);
+      load_cached_chunk<T, FMT>(kv.k, kv.k_meta, src, n_kv, hd, h, half + c * V, chi);
+      const float2* rot = table + (size_t)maps.ctx_off[u] * half + c * V;
+      const float* mu = mu_k + ((size_t)u * n_kv + h) * hd + c * V;
+#pragma unroll
+      for (int i = 0; i < V; ++i) {
+        const float2 t = rot[i];
+        lo[i] = clo[i] * t.x - chi[i] * t.y;
+        hi[i] = chi[i] * t.x + clo[i] * t.y;
+        if (w_k) {
+          lo[i] = fmaf(wk, mu[i], lo[i]);
+          hi[i] = fmaf(wk, mu[half + i], hi[i]);
+        }
+      }
+    }
+    st16(out_k + o, lo);
+    st16(out_k + o + half, hi);
+    // ---- V
+    if (row_v >= 0) {
+      const T* fp = v_fresh + ((size_t)row_v * n_kv + h) * hd + c * V;
+      ld16(fp, lo);
+      ld16(fp + half, hi);
+    } else {
+      load_cached_chunk<T, FMT>(kv.v, kv.v_meta, src, n_kv, hd, h, c * V, lo);
+      load_cached_chunk<T, FMT>(kv.v, kv.v_meta, src, n_kv, hd, h, half + c * V, hi);
+      if (w_k) {
+        const float* mu = mu_v + ((size_t)u * n_kv + h) * hd + c * V;
+#pragma unroll
+        for (int i = 0; i < V; ++i) {
+          lo[i] = fmaf(wv, mu[i], lo[i]);
+          hi[i] = fmaf(wv, mu[half + i], hi[i]);
+        }
+      }
+    }
+    st16(out_v + o, lo);
+    st16(out_v + o + half, hi);
+  }
+}
+
+int32_t launch_correct(int dtype, const KvLayer& kv, const ReqMaps& maps, const void* k_fresh, const void* v_fresh,
+                       const float* w_k, const float* w_v, const float* mu_k, const float* mu_v, int N, int n_query,
+                       int n_probe_rows, int n_kv, int hd, const float2* table, void* out_k, void* out_v,
+                       cudaStream_t st) {
+  const int T_tok = N + n_query;
+  if (T_tok == 0) return AKVS_OK;
+  AKVS_TRY(check_kv_shape(dtype, kv, hd));
+  const int V = dtype == AKVS_F32 ? 4 : 8;
+  const int64_t total = (int64_t)T_tok * n_kv * (hd / 2 / V);
+  int64_t want = (total + 255) / 256;
+  const int grid = (int)(want < 148 * 8 ? want : 148 * 8);   // grid-stride; 8 CTAs of 256 threads per SM
+  if (dtype == AKVS_F32) {
+    const float *kf = (const float*)k_fresh, *vf = (const float*)v_fresh;
+    float *ok = (float*)out_k, *ov = (float*)out_v;
+    if (kv.fmt == AKVS_KV_NATIVE) correct_kernel<float, AKVS_KV_NATIVE><<<grid, 256, 0, st>>>(kv, maps, kf, vf, w_k, w_v, mu_k, mu_v, N, T_tok, n_probe_rows, n_kv, hd, table, ok, ov);
+    else if (kv.fmt == AKVS_KV_Q4) correct_kernel<float, AKVS_KV_Q4><<<grid, 256, 0, st>>>(kv, maps, kf, vf, w_k, w_v, mu_k, mu_v, N, T_tok, n_probe_rows, n_kv, hd, table, ok, ov);
+    else correct_kernel<float, AKVS_KV_Q2><<<grid, 256, 0, st>>>(kv, maps, kf, vf, w_k, w_v, mu_k, mu_v, N, T_tok, n_probe_rows, n_kv, hd, table, ok, ov);
+  } else {
+    const bf16 *kf = (const bf16*)k_fresh, *vf = (const bf16*)v_fresh;
+    bf16 *ok = (bf16*)out_k, *ov = (bf16*)out_v;
+    if (kv.fmt == AKVS_KV_NATIVE) correct_kernel<bf16, AKVS_KV_NATIVE><<<grid, 256, 0, st>>>(kv, maps, kf, vf, w_k, w_v, mu_k, mu_v, N, T_tok, n_probe_rows, n_kv, hd, table, ok, ov);
+    else if (kv.fmt == AKVS_KV_Q4) correct_kernel<bf16, AKVS_KV_Q4><<<grid, 256, 0, st>>>(kv, maps, kf, vf, w_k, w_v, mu_k, mu_v, N, T_tok, n_probe_rows, n_kv, hd, table, ok, ov);
+    else correct_kernel<bf16, AKVS_KV_Q2><<<grid, 256, 0, st>>>(kv, maps, kf, vf, w_k, w_v, mu_k, mu_v, N, T_tok, n_probe_rows, n_kv, hd, table, ok, ov);
+  }
+  AKVS_LAUNCHED();
+  return AKVS_OK;
+}

@@ -1,0 +1,254 @@
+// Elementwise and row-wise steps of the decoder: embedding lookup, row gather, RMSNorm,
+// RoPE table + rotation, and the cache group quantiser.  All are HBM-bound; every global
+// access is a 16-byte vector where the layout allows it.
+#include "common.cuh"
+
+// ---------------------------------------------------------------------------------------
+// h[r][:] = float(tok_emb[ids[gather ? gather[r] : r]][:])
+// ---------------------------------------------------------------------------------------
+template <typename T>
+__global__ void embed_kernel(const T* __restrict__ emb, const int32_t* __restrict__ ids,
+                             const int32_t* __restrict__ gather, int n, int d, float* __restrict__ h) {
+  constexpr int V = VecOf<T>::N;
+  const int r = blockIdx.x;
+  const int id = ids[gather ? gather[r] : r];
+  const T* src = emb + (size_t)id * d;
+  float* dst = h + (size_t)r * d;
+  for (int c = threadIdx.x * V; c < d; c += blockDim.x * V) {
+    float v[V];
+    ld16(src + c, v);
+#pragma unroll
+    for (int i = 0; i < V; i += 4) {
+      float t[4] = {v[i], v[i + 1], v[i + 2], v[i + 3]};
+      st16(dst + c + i, t);
+    }
+  }
+}
+
+int32_t launch_embed(int dtype, const void* tok_emb, const int32_t* ids, const int32_t* gather, int n, int d,
+                     float* h, cudaStream_t st) {
+  if (n == 0) return AKVS_OK;
+  if (dtype == AKVS_F32)
+    embed_kernel<float><<<n, 128, 0, st>>>((const float*)tok_emb, ids, gather, n, d, h);
+  else
+    embed_kernel<bf16><<<n, 128, 0, st>>>((const bf16*)tok_emb, ids, gather, n, d, h);
+  AKVS_LAUNCHED();
+  return AKVS_OK;
+}
+
+__global__ void gather_rows_kernel(const float* __restrict__ src, const int32_t* __restrict__ rows, int d,
+                                   float* __restrict__ dst) {
+  const int r = blockIdx.x;
+  const float4* s = reinterpret_cast<const float4*>(src + (size_t)rows[r] * d);
+  float4* t = reinterpret_cast<float4*>(dst + (size_t)r * d);
+  for (int c = threadIdx.x; c < d / 4; c += blockDim.x) t[c] = s[c];
+}
+
+int32_t launch_gather_rows(const float* src, const int32_t* rows, int n, int d, float* dst, cudaStream_t st) {
+  if (n == 0) return AKVS_OK;
+  gather_rows_kernel<<<n, 256, 0, st>>>(src, rows, d, dst);
+  AKVS_LAUNCHED();
+  return AKVS_OK;
+}
+
+__global__ void iota_kernel(int32_t* p, int n, int start) {
+  int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) p[i] = start + i;
+}
+int32_t launch_iota(int32_t* p, int n, int start, cudaStream_t st) {
+  if (n == 0) return AKVS_OK;
+  iota_kernel<<<akvs_cdiv(n, 256), 256, 0, st>>>(p, n, start);
+  AKVS_LAUNCHED();
+  return AKVS_OK;
+}
+
+// ---------------------------------------------------------------------------------------
+// RMSNorm: x = h * rsqrt(mean(h^2) + eps) * gain.  One CTA per row; the row (float) is read
+// once into registers (d <= 256 threads * 4 * RMS_MAX_V elements).
+// ---------------------------------------------------------------------------------------
+constexpr int RMS_THREADS = 256;
+constexpr int RMS_MAX_V = 8;           // float4 per thread: d <= 8192
+
+template <typename TO>
+__global__ void __launch_bounds__(RMS_THREADS)
+rmsnorm_kernel(const float* __restrict__ h, const float* __restrict__ gain, float eps, int d, TO* __restrict__ x) {
+  const int r = blockIdx.x;
+  const float4* hp = reinterpret_cast<const float4*>(h + (size_t)r * d);
+  const float4* gp = reinterpret_cast<const float4*>(gain);
+  const int nv = d / 4;
+  float4 v[RMS_MAX_V];
+  float ss = 0.f;
+#pragma unroll
+  for (int i = 0; i < RMS_MAX_V; ++i) {
+    const int c = threadIdx.x + i * RMS_THREADS;
+    if (c < nv) {
+      v[i] = hp[c];
+      ss += v[i].x * v[i].x + v[i].y * v[i].y + v[i].z * v[i].z + v[i].w * v[i].w;
+    }
+  }
+  __shared__ float part[RMS_THREADS / 32];
+  ss = warp_sum(ss);
+  if ((threadIdx.x & 31) == 0) part[threadIdx.x >> 5] = ss;
+  __syncthreads();
+  float tot = 0.f;
+#pragma unroll
+  for (int i = 0; i < RMS_THREADS / 32; ++i) tot += part[i];
+  const float scale = rsqrtf(tot / (float)d + eps);
+  TO* xp = x + (size_t)r * d;
+#pragma unroll
+  for (int i = 0; i < RMS_MAX_V; ++i) {
+    const int c = threadIdx.x + i * RMS_THREADS;
+    if (c < nv) {
+      const float4 g = gp[c];
+      const float o0 = v[i].x * scale * g.x, o1 = v[i].y * scale * g.y;
+      const float o2 = v[i].z * scale * g.z, o3 = v[i].w * scale * g.w;
+      if constexpr (sizeof(TO) == 4) {
+        reinterpret_cast<float4*>(xp)[c] = make_float4(o0, o1, o2, o3);
+      } else {
+        uint2 pk;
+        pk.x = pack_bf16x2(o0, o1);
+        pk.y = pack_bf16x2(o2, o3);
+        reinterpret_cast<uint2*>(xp)[c] = pk;
+      }
+    }
+  }
+}
+
+int32_t launch_rmsnorm(int out_dtype, const float* h, const float* gain, float eps, int n, int d, void* x,
+                       cudaStream_t st) {
+  if (n == 0) return AKVS_OK;
+  if (d % 4 != 0 || d > RMS_THREADS * 4 * RMS_MAX_V) return AKVS_ERR_UNSUPPORTED;
+  if (out_dtype == AKVS_F32)
+    rmsnorm_kernel<float><<<n, RMS_THREADS, 0, st>>>(h, gain, eps, d, (float*)x);
+  else
+    rmsnorm_kernel<bf16><<<n, RMS_THREADS, 0, st>>>(h, gain, eps, d, (bf16*)x);
+  AKVS_LAUNCHED();
+  return AKVS_OK;
+}
+
+// ---------------------------------------------------------------------------------------
+// RoPE.  table[p][i] = (cos, sin)(p * base^(-2i/hd)), angle formed in double so that the
+// float table is the correctly rounded value for every position the request can reach.
+// ---------------------------------------------------------------------------------------
+__global__ void rope_table_kernel(double base, int hd, int n_pos, float2* __restrict__ table) {
+  const int half = hd / 2;
+  const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= n_pos * half) return;
+  const int p = idx / half, i = idx % half;
+  const double inv_freq = pow(base, -2.0 * (double)i / (double)hd);
+  double s, c;
+  sincos((double)p * inv_freq, &s, &c);
+  table[idx] = make_float2((float)c, (float)s);
+}
+
+int32_t launch_rope_table(float base, int hd, int n_pos, float2* table, cudaStream_t st) {
+  if (n_pos == 0) return AKVS_OK;
+  rope_table_kernel<<<akvs_cdiv((int64_t)n_pos * (hd / 2), 256), 256, 0, st>>>((double)base, hd, n_pos, table);
+  AKVS_LAUNCHED();
+  return AKVS_OK;
+}
+
+// In place on x[n][n_heads][hd] (row stride ld elements).  One thread per 16-byte chunk of
+// the lower half; it also owns the partner chunk in the upper half.
+template <typename T>
+__global__ void rope_kernel(T* __restrict__ x, const int32_t* __restrict__ pos, int n, int n_heads, int hd, int ld,
+                            const float2* __restrict__ table, double base) {
+  constexpr int V = VecOf<T>::N;
+  const int half = hd / 2, ch = half / V;
+  const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= (int64_t)n * n_heads * ch) return;
+  const int c = (int)(idx % ch);
+  const int hh = (int)((idx / ch) % n_heads);
+  const int r = (int)(idx / ((int64_t)ch * n_heads));
+  const int p = pos[r];
+  T* lo_p = x + (size_t)r * ld + (size_t)hh * hd + c * V;
+  T* hi_p = lo_p + half;
+  float lo[V], hi[V], olo[V], ohi[V];
+  ld16(lo_p, lo);
+  ld16(hi_p, hi);
+#pragma unroll
+  for (int i = 0; i < V; ++i) {
+    float cs, sn;
+    if (table) {
+      const float2 t = table[(size_t)p * half + c * V + i];
+      cs = t.x;
+      sn = t.y;
+    } else {
+      const double inv_freq = pow(base, -2.0 * (double)(c * V + i) / (double)hd);
+      double s_, c_;
+      sincos((double)p * inv_freq, &s_, &c_);
+      cs = (float)c_;
+      sn = (float)s_;
+    }
+    olo[i] = lo[i] * cs - hi[i] * sn;
+    ohi[i] = hi[i] * cs + lo[i] * sn;
+  }
+  st16(lo_p, olo);
+  st16(hi_p, ohi);
+}
+
+int32_t launch_rope(int dtype, void* x, const int32_t* pos, int n, int n_heads, int hd, int ld,
+                    const float2* table, float base, cudaStream_t st) {
+  if (n == 0) return AKVS_OK;
+  const int V = dtype == AKVS_F32 ? 4 : 8;
+  if (hd % (2 * V) != 0) return AKVS_ERR_UNSUPPORTED;
+  const int64_t total = (int64_t)n * n_heads * (hd / 2 / V);
+  const int blocks = akvs_cdiv(total, 256);
+  if (dtype == AKVS_F32)
+    rope_kernel<float><<<blocks, 256, 0, st>>>((float*)x, pos, n, n_heads, hd, ld, table, (double)base);
+  else
+    rope_kernel<bf16><<<blocks, 256, 0, st>>>((bf16*)x, pos, n, n_heads, hd, ld, table, (double)base);
+  AKVS_LAUNCHED();
+  return AKVS_OK;
+}
+
+// ---------------------------------------------------------------------------------------
+// Group quantiser of the cache (asymmetric min-max, 64 consecutive dims, float16 scale and
+// minimum).  One warp per group: lane l owns elements 2l and 2l+1.  All decisions are
+// float32 round-to-nearest operations with no contraction, so codes are reproducible:
+//   scale = half((max - min) / levels); min16 = half(min);
+//   code  = clamp(rint((x - min16) / scale), 0, levels), 0 when scale == 0.
+// Packing: little-endian within a byte, dimension ascending.
+// ---------------------------------------------------------------------------------------
+template <typename T>
+__global__ void quantize_kernel(const T* __restrict__ x, int64_t n_groups, int bits, uint8_t* __restrict__ codes,
+                                __half2* __restrict__ meta) {
+  const int64_t g = (int64_t)blockIdx.x * (blockDim.x / 32) + (threadIdx.x >> 5);
+  if (g >= n_groups) return;
+  const int lane = threadIdx.x & 31;
+  const T* xp = x + g * 64 + 2 * lane;
+  const float a = to_f(xp[0]), b = to_f(xp[1]);
+  const float mn = warp_min(fminf(a, b));
+  const float mx = warp_max(fmaxf(a, b));
+  const float levels = (float)((1 << bits) - 1);
+  const __half s16 = __float2half_rn(__fdiv_rn(__fsub_rn(mx, mn), levels));
+  const __half m16 = __float2half_rn(mn);
+  const float s = __half2float(s16), m = __half2float(m16);
+  uint32_t c0 = 0, c1 = 0;
+  if (s != 0.f) {
+    c0 = (uint32_t)fminf(fmaxf(rintf(__fdiv_rn(__fsub_rn(a, m), s)), 0.f), levels);
+    c1 = (uint32_t)fminf(fmaxf(rintf(__fdiv_rn(__fsub_rn(b, m), s)), 0.f), levels);
+  }
+  if (bits == 4) {
+    codes[g * 32 + lane] = (uint8_t)(c0 | (c1 << 4));
+  } else {
+    const uint32_t nib = c0 | (c1 << 2);
+    const uint32_t other = __shfl_down_sync(0xFFFFFFFFu, nib, 1);
+    if ((lane & 1) == 0) codes[g * 16 + (lane >> 1)] = (uint8_t)(nib | (other << 4));
+  }
+  if (lane == 0) meta[g] = __halves2half2(s16, m16);
+}
+
+int32_t launch_quantize(int dtype, const void* x, int n, int n_kv, int hd, int bits, void* codes, void* meta,
+                        cudaStream_t st) {
+  if (n == 0) return AKVS_OK;
+  if (hd % 64 != 0 || (bits != 2 && bits != 4)) return AKVS_ERR_UNSUPPORTED;
+  const int64_t n_groups = (int64_t)n * n_kv * (hd / 64);
+  const int blocks = akvs_cdiv(n_groups, 8);
+  if (dtype == AKVS_F32)
+    quantize_kernel<float><<<blocks, 256, 0, st>>>((const float*)x, n_groups, bits, (uint8_t*)codes, (__half2*)meta);
+  else
+    quantize_kernel<bf16><<<blocks, 256, 0, st>>>((const bf16*)x, n_groups, bits, (uint8_t*)codes, (__half2*)meta);
+  AKVS_LAUNCHED();
+  return AKVS_OK;
+}

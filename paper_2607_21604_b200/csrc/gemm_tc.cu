@@ -1,0 +1,344 @@
+// bf16 linear layers on the 5th-generation tensor cores (tcgen05), float accumulation in
+// tensor memory.  y = x W^T with x [M][K] and W [N][K], both K-major, staged by TMA in
+// 128-byte-swizzled 64-wide k slabs.
+//
+// Persistent kernel, one CTA per SM, 6 warps:
+//   warp 0      TMA producer (one elected lane), 4-stage ring of (A 128x64, B 256x64) slabs
+//   warp 1      tensor-memory allocation + MMA issue (one lane): 128x256x16 tcgen05.mma
+//   warps 2-5   epilogue: tcgen05.ld the 128x256 float accumulator (row per thread), fuse
+//               the layer's elementwise tail, store.  Two accumulators (2 x 256 columns)
+//               let the epilogue of tile i overlap the main loop of tile i+1.
+// The 256 accumulator columns are two 128-row blocks of B that may come from different
+// weight matrices: (Wq | Wk | Wv) share one launch, and (W_gate, W_up) land side by side
+// so that silu(gate) * up is formed in registers and only the activation is written.
+#include "tc_common.cuh"
+
+namespace {
+
+constexpr int BM = 128, BNH = 128, BK = 64, STAGES = 4;
+constexpr int A_BYTES = BM * BK * 2, BH_BYTES = BNH * BK * 2;
+constexpr int STAGE_BYTES = A_BYTES + 2 * BH_BYTES;        // 49152
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr int THREADS = 192;
+
+enum { EPI_STORE = 0, EPI_RESID = 1, EPI_SWIGLU = 2 };
+
+struct GemmParams {
+  int M, K, tiles_m, tiles_n;
+  int n_seg;
+  int seg_blocks[3];      // 128-row blocks of each B matrix
+  void* seg_out[3];       // output of each segment (bf16 [M][ldc], or float for EPI_RESID)
+  int seg_ldc[3];
+  int32_t* status;
+};
+
+// Which weight matrix and which of its rows the 128-row block `block` of the concatenated
+// output columns comes from.  Past the last matrix the row lies beyond its extent and the
+// TMA load fills zeros.
+__device__ __forceinline__ void locate(const GemmParams& p, int block, int& seg, int& row) {
+  seg = 0;
+  while (seg < p.n_seg - 1 && block >= p.seg_blocks[seg]) {
+    block -= p.seg_blocks[seg];
+    ++seg;
+  }
+  row = block * BNH;
+}
+
+template <int EPI>
+__global__ void __launch_bounds__(THREADS, 1)
+gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB0,
+               const __grid_constant__ CUtensorMap tmB1, const __grid_constant__ CUtensorMap tmB2,
+               const GemmParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + STAGES * STAGE_BYTES);
+  uint64_t* full = bars;                    // [STAGES]
+  uint64_t* empty = bars + STAGES;          // [STAGES]
+  uint64_t* acc_full = bars + 2 * STAGES;   // [2]
+  uint64_t* acc_empty = acc_full + 2;       // [2]
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int KB = (p.K + BK - 1) / BK;
+  const int n_tiles = p.tiles_m * p.tiles_n;
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < STAGES; ++i) { tc::mbar_init(&full[i], 1); tc::mbar_init(&empty[i], 1); }
+    for (int i = 0; i < 2; ++i) { tc::mbar_init(&acc_full[i], 1); tc::mbar_init(&acc_empty[i], 4); }
+    *abort_flag = 0;
+    tc::fence_barrier_init();
+    tc::fence_proxy_async();
+  }
+  if (warp == 1) {
+    tc::tmem_alloc(tmem_slot, 512);
+    tc::tmem_relinquish();
+  }
+  tc::fence_before_sync();
+  __syncthreads();
+  tc::fence_after_sync();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      tc::prefetch_tmap(&tmA);
+      tc::prefetch_tmap(&tmB0);
+      int s = 0;
+      uint32_t ph = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+        const int tn = tile / p.tiles_m, tm = tile % p.tiles_m;
+        int seg0, row0, seg1, row1;
+        if (EPI == EPI_SWIGLU) {
+          seg0 = 0; seg1 = 1; row0 = row1 = tn * BNH;
+        } else {
+          locate(p, 2 * tn, seg0, row0);
+          locate(p, 2 * tn + 1, seg1, row1);
+        }
+        const CUtensorMap* m0 = seg0 == 0 ? &tmB0 : (seg0 == 1 ? &tmB1 : &tmB2);
+        const CUtensorMap* m1 = seg1 == 0 ? &tmB0 : (seg1 == 1 ? &tmB1 : &tmB2);
+        for (int kb = 0; kb < KB; ++kb) {
+          if (!tc::mbar_wait(&empty[s], ph ^ 1, abort_flag)) { ok = false; break; }
+          uint8_t* st = smem + s * STAGE_BYTES;
+          tc::mbar_expect_tx(&full[s], STAGE_BYTES);
+          tc::tma_load_2d(st, &tmA, kb * BK, tm * BM, &full[s]);
+          tc::tma_load_2d(st + A_BYTES, m0, kb * BK, row0, &full[s]);
+          tc::tma_load_2d(st + A_BYTES + BH_BYTES, m1, kb * BK, row1, &full[s]);
+          if (++s == STAGES) { s = 0; ph ^= 1; }
+        }
+      }
+      if (!ok) { *abort_flag = 1; set_status(p.status, AKVS_ERR_TIMEOUT); }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc = tc::idesc_bf16(BM, 2 * BNH, 0);
+      int s = 0;
+      uint32_t ph = 0;
+      bool ok = true;
+      int it = 0;
+      for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++it) {
+        const int acc = it & 1;
+        if (!tc::mbar_wait(&acc_empty[acc], ((it >> 1) & 1) ^ 1, abort_flag)) { ok = false; break; }
+        tc::fence_after_sync();
+        const uint32_t d_tmem = tmem_base + acc * (2 * BNH);
+        for (int kb = 0; kb < KB; ++kb) {
+          if (!tc::mbar_wait(&full[s], ph, abort_flag)) { ok = false; break; }
+          tc::fence_after_sync();
+          const uint32_t a_addr = tc::smem_u32(smem + s * STAGE_BYTES);
+          const uint32_t b_addr = a_addr + A_BYTES;
+#pragma unroll
+          for (int k = 0; k < BK / 16; ++k) {
+            const uint64_t da = tc::smem_desc_k_sw128(a_addr + k * 32);
+            const uint64_t db = tc::smem_desc_k_sw128(b_addr + k * 32);
+            tc::mma_bf16(d_tmem, da, db, idesc, (kb | k) != 0);
+          }
+          tc::mma_commit(&empty[s]);            // frees the stage once these MMAs retire
+          if (++s == STAGES) { s = 0; ph ^= 1; }
+        }
+        if (ok) tc::mma_commit(&acc_full[acc]);
+      }
+      if (!ok) { *abort_flag = 1; set_status(p.status, AKVS_ERR_TIMEOUT); }
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue
+    const int quad = warp & 3;                 // tensor-memory lane quadrant of this warp
+    bool ok = true;
+    int it = 0;
+    for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++it) {
+      const int acc = it & 1;
+      const int tn = tile / p.tiles_m, tm = tile % p.tiles_m;
+      if (!tc::mbar_wait(&acc_full[acc], (it >> 1) & 1, abort_flag)) { ok = false; break; }
+      tc::fence_after_sync();
+      const int row = tm * BM + quad * 32 + lane;
+      const uint32_t t_addr = tmem_base + acc * (2 * BNH) + ((uint32_t)(quad * 32) << 16);
+      if (EPI == EPI_SWIGLU) {
+        bf16* out = reinterpret_cast<bf16*>(p.seg_out[0]);
+        const int ldc = p.seg_ldc[0];
+        const int n_valid = p.seg_blocks[0] * BNH;
+#pragma unroll 1
+        for (int c = 0; c < BNH / 32; ++c) {
+          float g[32], u[32];
+          tc::tmem_ld32(t_addr + c * 32, g);
+          tc::tmem_ld32(t_addr + BNH + c * 32, u);
+          tc::tmem_ld_wait();
+          const int col = tn * BNH + c * 32;
+          if (row < p.M && col < n_valid) {
+            bf16* o = out + (size_t)row * ldc + col;
+#pragma unroll
+            for (int v = 0; v < 4; ++v) {
+              float r[8];
+#pragma unroll
+              for (int i = 0; i < 8; ++i) {
+                const float x = g[v * 8 + i];
+                r[i] = x / (1.f + __expf(-x)) * u[v * 8 + i];
+              }
+              st16(o + v * 8, r);
+            }
+          }
+        }
+      } else {
+#pragma unroll 1
+        for (int hf = 0; hf < 2; ++hf) {
+          int seg, brow;
+          locate(p, 2 * tn + hf, seg, brow);
+          const bool valid = brow < p.seg_blocks[seg] * BNH;
+          const int ldc = p.seg_ldc[seg];
+#pragma unroll 1
+          for (int c = 0; c < BNH / 32; ++c) {
+            float a[32];
+            tc::tmem_ld32(t_addr + hf * BNH + c * 32, a);
+            tc::tmem_ld_wait();
+            if (row < p.M && valid) {
+              const int col = brow + c * 32;
+              if (EPI == EPI_RESID) {
+                float* o = reinterpret_cast<float*>(p.seg_out[seg]) + (size_t)row * ldc + col;
+#pragma unroll
+                for (int v = 0; v < 8; ++v) {
+                  float4 t = *reinterpret_cast<float4*>(o + v * 4);
+                  t.x += a[v * 4]; t.y += a[v * 4 + 1]; t.z += a[v * 4 + 2]; t.w += a[v * 4 + 3];
+                  *reinterpret_cast<float4*>(o + v * 4) = t;
+                }
+              } else {
+                bf16* o = reinterpret_cast<bf16*>(p.seg_out[seg]) + (size_t)row * ldc + col;
+#pragma unroll
+                for (int v = 0; v < 4; ++v) {
+                  float r[8];
+#pragma unroll
+                  for (int i = 0; i < 8; ++i) r[i] = a[v * 8 + i];
+                  st16(o + v * 8, r);
+                }
+              }
+            }
+          }
+        }
+      }
+      tc::fence_before_sync();
+      __syncwarp();
+      if (lane == 0) tc::mbar_arrive(&acc_empty[acc]);
+    }
+    if (!ok && lane == 0) { *abort_flag = 1; set_status(p.status, AKVS_ERR_TIMEOUT); }
+  }
+
+  // ---------------------------------------------------------------------- teardown
+  if (*abort_flag) __nanosleep(200000);       // let loads already in flight land before the CTA exits
+  tc::fence_before_sync();
+  __syncthreads();
+  if (warp == 1) {
+    __syncwarp();
+    tc::fence_after_sync();
+    tc::tmem_dealloc(tmem_base, 512);
+  }
+}
+
+typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                             const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                             CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeFn get_encoder() {
+  static EncodeFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess)
+      return nullptr;
+    fn = reinterpret_cast<EncodeFn>(p);
+  }
+  return fn;
+}
+
+int g_sm_count = 0;
+int sm_count() {
+  if (!g_sm_count) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&g_sm_count, cudaDevAttrMultiProcessorCount, dev);
+    if (g_sm_count <= 0) g_sm_count = 148;
+  }
+  return g_sm_count;
+}
+
+}  // namespace
+
+int32_t encode_tmap_2d_bf16(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, uint64_t ld,
+                            uint32_t box_rows) {
+  EncodeFn enc = get_encoder();
+  if (!enc) return AKVS_ERR_CUDA;
+  if ((reinterpret_cast<uintptr_t>(base) & 15) || (ld * 2) % 16 != 0) return AKVS_ERR_SHAPE;
+  const cuuint64_t dims[2] = {cols, rows};
+  const cuuint64_t strides[1] = {ld * 2};
+  const cuuint32_t box[2] = {64, box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  const CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? AKVS_OK : AKVS_ERR_CUDA;
+}
+
+int32_t encode_tmap_3d_bf16(CUtensorMap* map, const void* base, uint64_t d0, uint64_t d1, uint64_t d2, uint64_t ld1,
+                            uint64_t ld2, uint32_t b1, uint32_t b2) {
+  EncodeFn enc = get_encoder();
+  if (!enc) return AKVS_ERR_CUDA;
+  if ((reinterpret_cast<uintptr_t>(base) & 15) || (ld1 * 2) % 16 != 0 || (ld2 * 2) % 16 != 0) return AKVS_ERR_SHAPE;
+  const cuuint64_t dims[3] = {d0, d1, d2};
+  const cuuint64_t strides[2] = {ld1 * 2, ld2 * 2};
+  const cuuint32_t box[3] = {64, b1, b2};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  const CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? AKVS_OK : AKVS_ERR_CUDA;
+}
+
+// x [M][K] bf16; up to three weight matrices w[i] [n[i]][K] (n[i] a multiple of 128) whose
+// outputs go to out[i] with row stride ldc[i].
+//   epi 0: out[i] = x w[i]^T (bf16);   epi 1: out[0] (float) += x w[0]^T;
+//   epi 2: out[0] = silu(x w[0]^T) * (x w[1]^T) (bf16), n[0] == n[1].
+int32_t launch_linear_tc(int epi, const void* x, int M, int K, int n_seg, const void* const* w, const int* n,
+                         void* const* out, const int* ldc, int32_t* status, cudaStream_t st) {
+  if (M == 0) return AKVS_OK;
+  if (K % 8 != 0 || n_seg < 1 || n_seg > 3) return AKVS_ERR_SHAPE;
+  static bool attr_set = false;
+  if (!attr_set) {
+    AKVS_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI_STORE>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES));
+    AKVS_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI_RESID>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES));
+    AKVS_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI_SWIGLU>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES));
+    attr_set = true;
+  }
+  GemmParams p;
+  p.M = M;
+  p.K = K;
+  p.n_seg = n_seg;
+  p.status = status;
+  CUtensorMap tmA, tmB[3];
+  AKVS_TRY(encode_tmap_2d_bf16(&tmA, x, M, K, K, BM));
+  int blocks = 0;
+  for (int i = 0; i < 3; ++i) {
+    const int s = i < n_seg ? i : 0;
+    if (n[s] % BNH != 0) return AKVS_ERR_SHAPE;
+    AKVS_TRY(encode_tmap_2d_bf16(&tmB[i], w[s], n[s], K, K, BNH));
+    p.seg_blocks[i] = n[s] / BNH;
+    p.seg_out[i] = out[i < n_seg && (epi != EPI_SWIGLU || i == 0) ? i : 0];
+    p.seg_ldc[i] = ldc[i < n_seg && (epi != EPI_SWIGLU || i == 0) ? i : 0];
+    if (i < n_seg) blocks += n[s] / BNH;
+  }
+  if (epi == EPI_SWIGLU) {
+    if (n_seg != 2 || n[0] != n[1]) return AKVS_ERR_SHAPE;
+    p.tiles_n = n[0] / BNH;
+  } else {
+    p.tiles_n = (blocks + 1) / 2;
+  }
+  p.tiles_m = (M + BM - 1) / BM;
+  const int n_tiles = p.tiles_m * p.tiles_n;
+  const int grid = n_tiles < sm_count() ? n_tiles : sm_count();
+  switch (epi) {
+    case EPI_STORE: gemm_tc_kernel<EPI_STORE><<<grid, THREADS, SMEM_BYTES, st>>>(tmA, tmB[0], tmB[1], tmB[2], p); break;
+    case EPI_RESID: gemm_tc_kernel<EPI_RESID><<<grid, THREADS, SMEM_BYTES, st>>>(tmA, tmB[0], tmB[1], tmB[2], p); break;
+    case EPI_SWIGLU: gemm_tc_kernel<EPI_SWIGLU><<<grid, THREADS, SMEM_BYTES, st>>>(tmA, tmB[0], tmB[1], tmB[2], p); break;
+    default: return AKVS_ERR_INVALID_ARG;
+  }
+  AKVS_LAUNCHED();
+  return AKVS_OK;
+}

@@ -24,3 +24,14 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+@pytest.fixture(scope="session", autouse=True)
+def _linear_algo_override():
+    """AKVS_TEST_LINEAR_ALGO=1 runs the bf16 pipeline tests on the CUDA-core linear kernels
+    (a cross-check of the tensor-core ones); the default is the product configuration."""
+    algo = os.environ.get("AKVS_TEST_LINEAR_ALGO")
+    if algo is not None:
+        import paper_2607_21604_b200 as a
+        a.lib.akvs_debug_set_linear_algo(int(algo))
+    yield
