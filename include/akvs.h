@@ -20,9 +20,11 @@
  *  - all work is enqueued on the caller's stream (a cudaStream_t passed as void*; NULL is
  *    the default stream); only akvs_select_probes and akvs_check synchronise it;
  *  - linear weights are row-major [out_features][in_features] (y = x W^T), no biases;
- *  - model dtype AKVS_F32: weights, cache and outputs are float; AKVS_BF16: weights,
- *    cache and K/V outputs are bfloat16 with float accumulation.  The residual stream
- *    and `out_hidden` are float in both modes;
+ *  - model dtype AKVS_F32 / AKVS_BF16 / AKVS_F16: weights, the native unit cache, every
+ *    activation tensor and the K/V outputs have that type; accumulation, the residual
+ *    stream and `out_hidden` are float in every mode.  The 16-bit modes run the linear
+ *    layers on the tensor cores at the same rate; float16 keeps three more mantissa bits
+ *    (conversions saturate instead of producing infinities);
  *  - K is cached AFTER RoPE at unit-local positions 0..n-1 (rotate-half pairing
  *    (i, i + head_dim/2), angle p * rope_base^(-2i/head_dim)); reuse turns it through the
  *    unit's global offset.  Residuals, offsets and corrected K live at global positions.
@@ -47,6 +49,7 @@ extern "C" {
 
 #define AKVS_F32   0
 #define AKVS_BF16  1
+#define AKVS_F16   2
 
 #define AKVS_KV_NATIVE 0           /* cache holds the model dtype                            */
 #define AKVS_KV_Q2     2           /* 2-bit codes, asymmetric min-max, groups of 64 along head_dim */
@@ -61,7 +64,7 @@ extern "C" {
  * q head i reading kv head i / (n_q_heads / n_kv_heads), SwiGLU MLP. */
 typedef struct akvs_model_desc {
   int32_t n_layers, d_model, n_q_heads, n_kv_heads, head_dim, d_ff, vocab;
-  int32_t dtype;                      /* AKVS_F32 | AKVS_BF16                               */
+  int32_t dtype;                      /* AKVS_F32 | AKVS_BF16 | AKVS_F16                    */
   float   rope_base, rms_eps;
   const void*  tok_emb;               /* device [vocab][d_model], model dtype                */
   const float* final_norm;            /* device [d_model]                                    */
@@ -163,18 +166,30 @@ void akvs_free(void* ctx);
  * (AKVS_OK, AKVS_ERR_TIMEOUT, AKVS_ERR_NAN_SCORE), then clears it. */
 int32_t akvs_check(void* workspace, void* stream);
 
-/* Cross-check switch for the tests: 0 (default) routes bf16 linear layers to the tcgen05
+/* Cross-check switch for the tests: 0 (default) routes 16-bit linear layers to the tcgen05
  * kernels, 1 to the CUDA-core kernels.  Process-wide; not part of the serving surface. */
 int32_t akvs_debug_set_linear_algo(int32_t algo);
 
+/* Number of kernels this library has launched in this process so far. */
+int64_t akvs_launch_count(void);
+
+/* Per-launch device timing of one kernel class with CUDA events recorded on the launching
+ * stream: kind 1 = tensor-core linear layers (sub = epilogue: 0 store, 1 residual, 2 SwiGLU;
+ * work = flops), kind 2 = correction pass (sub = kv format; work = algorithmic bytes),
+ * kind 0 = off.  akvs_prof_enable allocates max_records event pairs (host objects only);
+ * akvs_prof_read waits for the recorded events and returns elapsed ms, work and sub per
+ * launch; akvs_prof_reset forgets the records but keeps the events.  Not thread-safe. */
+int32_t akvs_prof_enable(int32_t kind, int32_t max_records);
+int32_t akvs_prof_reset(void);
+int32_t akvs_prof_read(int32_t capacity, float* ms, double* work, int32_t* sub, int32_t* n_out);
+
 /* ------------------------------------------------------------------------------------
  * Single steps of the path, exported so that each kernel can be checked on its own.
- * dtype is AKVS_F32 or AKVS_BF16 and names the type of every `void*` tensor.
- * All asynchronous on `stream`.
+ * dtype names the element type of every `void*` tensor.  Asynchronous on `stream` unless stated.
  * ------------------------------------------------------------------------------------ */
 
 /* y[M][N] = x[M][K] * w[N][K]^T, float accumulation.  algo 0: the path's default for the
- * dtype (tcgen05 tensor cores for bf16, CUDA cores for float); algo 1: CUDA cores. */
+ * dtype (tcgen05 tensor cores for the 16-bit types, CUDA cores for float); algo 1: CUDA cores. */
 int32_t akvs_op_linear(int32_t dtype, const void* x, const void* w, void* y,
                        int32_t M, int32_t N, int32_t K, int32_t algo, void* stream);
 

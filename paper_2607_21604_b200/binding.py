@@ -17,11 +17,12 @@ LIB_PATH = os.path.join(_HERE, "libakvs.so")
 OK = 0
 ERR = {0: "AKVS_OK", -1: "AKVS_ERR_INVALID_ARG", -2: "AKVS_ERR_SHAPE", -3: "AKVS_ERR_WORKSPACE",
        -4: "AKVS_ERR_UNSUPPORTED", -5: "AKVS_ERR_CUDA", -6: "AKVS_ERR_TIMEOUT", -7: "AKVS_ERR_NAN_SCORE"}
-F32, BF16 = 0, 1
+F32, BF16, F16 = 0, 1, 2
 KV_NATIVE, KV_Q2, KV_Q4 = 0, 2, 4
 MODE_CORRECTED, MODE_NAIVE, MODE_FULL = 0, 1, 2
 
-EXPORTS = ["akvs_workspace_bytes", "akvs_debug_set_linear_algo", "akvs_encode_units", "akvs_select_probes", "akvs_prefill_corrected",
+EXPORTS = ["akvs_workspace_bytes", "akvs_debug_set_linear_algo", "akvs_launch_count", "akvs_prof_enable",
+           "akvs_prof_reset", "akvs_prof_read", "akvs_encode_units", "akvs_select_probes", "akvs_prefill_corrected",
            "akvs_free", "akvs_check", "akvs_op_linear", "akvs_op_rope", "akvs_op_attention",
            "akvs_op_scratch_bytes", "akvs_op_select", "akvs_op_correct_layer", "akvs_op_quantize"]
 
@@ -66,6 +67,7 @@ def _load():
     for name in EXPORTS:
         getattr(lib, name)                       # raises AttributeError if a symbol is absent
     lib.akvs_op_scratch_bytes.restype = C.c_int64
+    lib.akvs_launch_count.restype = C.c_int64
     lib.akvs_free.restype = None
     return lib
 
@@ -86,8 +88,14 @@ def _chk(code, where):
         raise AkvsError(code, where)
 
 
-def _tdtype(dtype):
-    return torch.float32 if dtype == F32 else torch.bfloat16
+_TORCH = {F32: torch.float32, BF16: torch.bfloat16, F16: torch.float16}
+
+
+def torch_dtype(dtype):
+    return _TORCH[dtype]
+
+
+_tdtype = torch_dtype
 
 
 class Model:
@@ -115,7 +123,7 @@ class Model:
     @classmethod
     def from_numpy(cls, cfg, tok_emb, layers, final_norm=None, device="cuda"):
         """Uploads host arrays (float32 values, bf16-representable for bf16 models)."""
-        dtype = F32 if cfg.dtype == "f32" else BF16
+        dtype = {"f32": F32, "bf16": BF16, "f16": F16}[cfg.dtype]
         td = _tdtype(dtype)
         up = lambda a, t: torch.from_numpy(a).to(device=device, dtype=t).contiguous()
         dl = [{n: up(lw[n], torch.float32 if "norm" in n else td) for n in cls.NAMES} for lw in layers]
@@ -229,6 +237,27 @@ def check(workspace):
     return lib.akvs_check(_ptr(workspace), _stream())
 
 
+def launch_count():
+    return int(lib.akvs_launch_count())
+
+
+def prof_enable(kind, max_records=0):
+    _chk(lib.akvs_prof_enable(kind, max_records), "akvs_prof_enable")
+
+
+def prof_reset():
+    lib.akvs_prof_reset()
+
+
+def prof_read(capacity=1 << 16):
+    ms = (C.c_float * capacity)()
+    work = (C.c_double * capacity)()
+    sub = (C.c_int32 * capacity)()
+    n = C.c_int32(0)
+    _chk(lib.akvs_prof_read(capacity, ms, work, sub, C.byref(n)), "akvs_prof_read")
+    return [(ms[i], work[i], sub[i]) for i in range(n.value)]
+
+
 def alloc_outputs(model, n_ctx, n_query, device="cuda"):
     cfg = model.cfg
     td = _tdtype(model.dtype)
@@ -240,8 +269,12 @@ def alloc_outputs(model, n_ctx, n_query, device="cuda"):
 
 # ------------------------------------------------------------------------------- single steps
 
+def _dt(t):
+    return {torch.float32: F32, torch.bfloat16: BF16, torch.float16: F16}[t.dtype]
+
+
 def op_linear(x, w, algo=0):
-    dtype = F32 if x.dtype == torch.float32 else BF16
+    dtype = _dt(x)
     M, K = x.shape
     N = w.shape[0]
     y = torch.empty((M, N), dtype=x.dtype, device=x.device)
@@ -250,14 +283,14 @@ def op_linear(x, w, algo=0):
 
 
 def op_rope(x, pos, base):
-    dtype = F32 if x.dtype == torch.float32 else BF16
+    dtype = _dt(x)
     n, H, hd = x.shape
     _chk(lib.akvs_op_rope(dtype, _ptr(x), _ptr(pos), n, H, hd, C.c_float(base), _stream()), "akvs_op_rope")
     return x
 
 
 def op_attention(q, k, v, k_lo, k_hi, algo=0):
-    dtype = F32 if q.dtype == torch.float32 else BF16
+    dtype = _dt(q)
     R, nq, hd = q.shape
     T, nkv, _ = k.shape
     out = torch.empty_like(q)
@@ -300,7 +333,7 @@ def op_correct_layer(dtype, kv_format, cache_k, cache_v, k_meta, v_meta, src_tok
 
 
 def op_quantize(x, bits):
-    dtype = F32 if x.dtype == torch.float32 else BF16
+    dtype = _dt(x)
     n, nkv, hd = x.shape
     codes = torch.empty((n, nkv, hd * bits // 8), dtype=torch.uint8, device=x.device)
     meta = torch.empty((n, nkv, hd // 64, 2), dtype=torch.float16, device=x.device)

@@ -7,6 +7,29 @@
 
 #include "common.cuh"
 
+unsigned long long g_akvs_launches = 0;
+
+// ----------------------------------------------------------------------------- profiling hooks
+namespace {
+struct ProfRec { cudaEvent_t a, b; int sub; double work; };
+int g_prof_kind = 0;
+std::vector<ProfRec> g_prof;
+size_t g_prof_used = 0;
+}  // namespace
+
+void akvs_prof_mark(int kind, int sub, double work, bool begin, cudaStream_t st) {
+  if (kind != g_prof_kind || g_prof_used >= g_prof.size()) return;
+  ProfRec& r = g_prof[g_prof_used];
+  if (begin) {
+    r.sub = sub;
+    r.work = work;
+    cudaEventRecord(r.a, st);
+  } else {
+    cudaEventRecord(r.b, st);
+    ++g_prof_used;
+  }
+}
+
 namespace {
 
 constexpr uint32_t kCtxMagic = 0x616B7673u;   // "akvs"
@@ -18,7 +41,7 @@ struct Dims {
 
 int32_t check_model(const akvs_model_desc* m, Dims& D) {
   if (!m) return AKVS_ERR_INVALID_ARG;
-  if (m->dtype != AKVS_F32 && m->dtype != AKVS_BF16) return AKVS_ERR_UNSUPPORTED;
+  if (m->dtype != AKVS_F32 && m->dtype != AKVS_BF16 && m->dtype != AKVS_F16) return AKVS_ERR_UNSUPPORTED;
   if (m->n_layers <= 0 || m->d_model <= 0 || m->n_q_heads <= 0 || m->n_kv_heads <= 0 || m->head_dim <= 0 ||
       m->d_ff <= 0 || m->vocab <= 0)
     return AKVS_ERR_INVALID_ARG;
@@ -34,7 +57,7 @@ int32_t check_model(const akvs_model_desc* m, Dims& D) {
       return AKVS_ERR_INVALID_ARG;
   D.L = m->n_layers; D.d = m->d_model; D.nq = m->n_q_heads; D.nkv = m->n_kv_heads; D.hd = m->head_dim;
   D.f = m->d_ff; D.vocab = m->vocab; D.dq = D.nq * D.hd; D.dkv = D.nkv * D.hd; D.dtype = m->dtype;
-  D.es = m->dtype == AKVS_F32 ? 4 : 2;
+  D.es = dtype_size(m->dtype);
   return AKVS_OK;
 }
 
@@ -128,33 +151,33 @@ struct Ctx {                   // host object that carries a request from select
 };
 
 // ----------------------------------------------------------------------------- linear layers
-int g_bf16_linear_algo = 0;    // 0: tcgen05; 1: CUDA cores (kept for cross-checking)
+int g_bf16_linear_algo = 0;    // 16-bit models: 0 = tcgen05; 1 = CUDA cores (kept for cross-checking)
 
 int32_t linear_multi(const Dims& D, const void* x, int M, int K, int n_seg, const void* const* w, const int* n,
                      void* const* out, const int* ldc, int32_t* status, cudaStream_t st) {
-  bool tc_ok = D.dtype == AKVS_BF16 && g_bf16_linear_algo == 0 && K % 8 == 0;
+  bool tc_ok = D.dtype != AKVS_F32 && g_bf16_linear_algo == 0 && K % 8 == 0;
   for (int i = 0; i < n_seg; ++i) tc_ok = tc_ok && n[i] % 128 == 0;
-  if (tc_ok) return launch_linear_tc(0, x, M, K, n_seg, w, n, out, ldc, status, st);
+  if (tc_ok) return launch_linear_tc(D.dtype, 0, x, M, K, n_seg, w, n, out, ldc, status, st);
   for (int i = 0; i < n_seg; ++i)
     AKVS_TRY(launch_linear_simt(D.dtype, x, w[i], nullptr, out[i], nullptr, M, n[i], K, ldc[i], st));
   return AKVS_OK;
 }
 int32_t linear_resid(const Dims& D, const void* x, int M, int K, const void* w, int n, float* h, int32_t* status,
                      cudaStream_t st) {
-  if (D.dtype == AKVS_BF16 && g_bf16_linear_algo == 0 && K % 8 == 0 && n % 128 == 0) {
+  if (D.dtype != AKVS_F32 && g_bf16_linear_algo == 0 && K % 8 == 0 && n % 128 == 0) {
     void* out = h;
-    return launch_linear_tc(1, x, M, K, 1, &w, &n, &out, &n, status, st);
+    return launch_linear_tc(D.dtype, 1, x, M, K, 1, &w, &n, &out, &n, status, st);
   }
   return launch_linear_simt(D.dtype, x, w, nullptr, nullptr, h, M, n, K, n, st);
 }
 int32_t linear_swiglu(const Dims& D, const void* x, int M, int K, const void* wg, const void* wu, int n, void* act,
                       int32_t* status, cudaStream_t st) {
-  if (D.dtype == AKVS_BF16 && g_bf16_linear_algo == 0 && K % 8 == 0 && n % 128 == 0) {
+  if (D.dtype != AKVS_F32 && g_bf16_linear_algo == 0 && K % 8 == 0 && n % 128 == 0) {
     const void* w[2] = {wg, wu};
     const int ns[2] = {n, n};
     void* out[2] = {act, act};
     const int ld[2] = {n, n};
-    return launch_linear_tc(2, x, M, K, 2, w, ns, out, ld, status, st);
+    return launch_linear_tc(D.dtype, 2, x, M, K, 2, w, ns, out, ld, status, st);
   }
   return launch_linear_simt(D.dtype, x, wg, wu, act, nullptr, M, n, K, n, st);
 }
@@ -288,6 +311,39 @@ int32_t akvs_debug_set_linear_algo(int32_t algo) {
   return AKVS_OK;
 }
 
+int64_t akvs_launch_count(void) { return (int64_t)g_akvs_launches; }
+
+int32_t akvs_prof_enable(int32_t kind, int32_t max_records) {
+  for (ProfRec& r : g_prof) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
+  g_prof.clear();
+  g_prof_used = 0;
+  g_prof_kind = kind;
+  if (kind == 0) return AKVS_OK;
+  if (max_records < 0) return AKVS_ERR_INVALID_ARG;
+  g_prof.resize(max_records);
+  for (ProfRec& r : g_prof)
+    if (cudaEventCreate(&r.a) != cudaSuccess || cudaEventCreate(&r.b) != cudaSuccess) return AKVS_ERR_CUDA;
+  return AKVS_OK;
+}
+
+int32_t akvs_prof_reset(void) {
+  g_prof_used = 0;
+  return AKVS_OK;
+}
+
+int32_t akvs_prof_read(int32_t capacity, float* ms, double* work, int32_t* sub, int32_t* n_out) {
+  if (!ms || !work || !sub || !n_out || capacity < 0) return AKVS_ERR_INVALID_ARG;
+  const size_t n = g_prof_used < (size_t)capacity ? g_prof_used : (size_t)capacity;
+  for (size_t i = 0; i < n; ++i) {
+    if (cudaEventSynchronize(g_prof[i].b) != cudaSuccess) return AKVS_ERR_CUDA;
+    if (cudaEventElapsedTime(&ms[i], g_prof[i].a, g_prof[i].b) != cudaSuccess) return AKVS_ERR_CUDA;
+    work[i] = g_prof[i].work;
+    sub[i] = g_prof[i].sub;
+  }
+  *n_out = (int32_t)n;
+  return AKVS_OK;
+}
+
 int32_t akvs_workspace_bytes(const akvs_model_desc* model, int32_t n_ctx, int32_t n_query, int32_t n_units,
                              int32_t check_layer, int64_t* out_bytes) {
   Dims D;
@@ -322,6 +378,8 @@ int32_t akvs_encode_units(const akvs_model_desc* model, akvs_cache* cache, void*
   const size_t lstride = (size_t)N * kv_row_bytes(D, cache->kv_format);
   const size_t mstride = (size_t)N * D.nkv * (D.hd / 64) * 4;
   for (int l = 0; l < D.L; ++l) {
+    // native cache: the layer's K/V go straight into the store; quantised cache: attention
+    // inside the unit reads the unquantised K/V and the codes are written beside
     void* k_dst = native ? reinterpret_cast<char*>(cache->k) + l * lstride : ws.k;
     void* v_dst = native ? reinterpret_cast<char*>(cache->v) + l * lstride : ws.v;
     std::function<int32_t()> store;
@@ -330,10 +388,9 @@ int32_t akvs_encode_units(const akvs_model_desc* model, akvs_cache* cache, void*
         AKVS_TRY(launch_quantize(D.dtype, ws.k, N, D.nkv, D.hd, cache->kv_format,
                                  reinterpret_cast<char*>(cache->k) + l * lstride,
                                  reinterpret_cast<char*>(cache->k_meta) + l * mstride, st));
-        AKVS_TRY(launch_quantize(D.dtype, ws.v, N, D.nkv, D.hd, cache->kv_format,
-                                 reinterpret_cast<char*>(cache->v) + l * lstride,
-                                 reinterpret_cast<char*>(cache->v_meta) + l * mstride, st));
-        return AKVS_OK;
+        return launch_quantize(D.dtype, ws.v, N, D.nkv, D.hd, cache->kv_format,
+                               reinterpret_cast<char*>(cache->v) + l * lstride,
+                               reinterpret_cast<char*>(cache->v_meta) + l * mstride, st);
       };
     AKVS_TRY(run_layer(model, D, l, ws, N, local_pos, ws.lo, ws.pos, k_dst, v_dst, k_dst, v_dst, store, st));
   }
@@ -525,11 +582,11 @@ int32_t akvs_check(void* workspace, void* stream) {
 int32_t akvs_op_linear(int32_t dtype, const void* x, const void* w, void* y, int32_t M, int32_t N, int32_t K,
                        int32_t algo, void* stream) {
   if (!x || !w || !y || M < 0 || N <= 0 || K <= 0) return AKVS_ERR_INVALID_ARG;
-  if (dtype != AKVS_F32 && dtype != AKVS_BF16) return AKVS_ERR_UNSUPPORTED;
+  if (dtype != AKVS_F32 && dtype != AKVS_BF16 && dtype != AKVS_F16) return AKVS_ERR_UNSUPPORTED;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
-  if (dtype == AKVS_BF16 && algo == 0) {
+  if (dtype != AKVS_F32 && algo == 0) {
     if (N % 128 != 0 || K % 8 != 0) return AKVS_ERR_SHAPE;
-    return launch_linear_tc(0, x, M, K, 1, &w, &N, &y, &N, nullptr, st);
+    return launch_linear_tc(dtype, 0, x, M, K, 1, &w, &N, &y, &N, nullptr, st);
   }
   return launch_linear_simt(dtype, x, w, nullptr, y, nullptr, M, N, K, N, st);
 }
@@ -537,7 +594,7 @@ int32_t akvs_op_linear(int32_t dtype, const void* x, const void* w, void* y, int
 int32_t akvs_op_rope(int32_t dtype, void* x, const int32_t* pos, int32_t n, int32_t n_heads, int32_t head_dim,
                      float rope_base, void* stream) {
   if (!x || !pos || n < 0 || n_heads <= 0 || head_dim <= 0) return AKVS_ERR_INVALID_ARG;
-  if (dtype != AKVS_F32 && dtype != AKVS_BF16) return AKVS_ERR_UNSUPPORTED;
+  if (dtype != AKVS_F32 && dtype != AKVS_BF16 && dtype != AKVS_F16) return AKVS_ERR_UNSUPPORTED;
   return launch_rope(dtype, x, pos, n, n_heads, head_dim, n_heads * head_dim, nullptr, rope_base,
                      reinterpret_cast<cudaStream_t>(stream));
 }
@@ -546,7 +603,7 @@ int32_t akvs_op_attention(int32_t dtype, const void* q, const void* k, const voi
                           const int32_t* k_hi, int32_t R, int32_t T, int32_t n_q_heads, int32_t n_kv_heads,
                           int32_t head_dim, int32_t algo, void* stream) {
   if (!q || !k || !v || !out || !k_lo || !k_hi || R < 0 || T < 0) return AKVS_ERR_INVALID_ARG;
-  if (dtype != AKVS_F32 && dtype != AKVS_BF16) return AKVS_ERR_UNSUPPORTED;
+  if (dtype != AKVS_F32 && dtype != AKVS_BF16 && dtype != AKVS_F16) return AKVS_ERR_UNSUPPORTED;
   (void)algo;
   return launch_attention_simt(dtype, q, k, v, out, k_lo, k_hi, R, n_q_heads, n_kv_heads, head_dim,
                                reinterpret_cast<cudaStream_t>(stream));
@@ -602,7 +659,7 @@ int32_t akvs_op_correct_layer(int32_t dtype, int32_t kv_format, const void* cach
     return AKVS_ERR_INVALID_ARG;
   if (probes->n_ctx > 0 && (!cache_k || !cache_v || !src_tok)) return AKVS_ERR_INVALID_ARG;
   if (probes->n_rows > 0 && (!fresh_k || !fresh_v)) return AKVS_ERR_INVALID_ARG;
-  if (dtype != AKVS_F32 && dtype != AKVS_BF16) return AKVS_ERR_UNSUPPORTED;
+  if (dtype != AKVS_F32 && dtype != AKVS_BF16 && dtype != AKVS_F16) return AKVS_ERR_UNSUPPORTED;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
   const int N = probes->n_ctx, T = N + n_query, M = n_units;
   if (probes->n_rows != probes->n_probe_rows + n_query) return AKVS_ERR_SHAPE;
@@ -636,7 +693,7 @@ int32_t akvs_op_correct_layer(int32_t dtype, int32_t kv_format, const void* cach
 int32_t akvs_op_quantize(int32_t dtype, const void* x, int32_t n, int32_t n_kv_heads, int32_t head_dim, int32_t bits,
                          void* codes, void* meta, void* stream) {
   if (!x || !codes || !meta || n < 0) return AKVS_ERR_INVALID_ARG;
-  if (dtype != AKVS_F32 && dtype != AKVS_BF16) return AKVS_ERR_UNSUPPORTED;
+  if (dtype != AKVS_F32 && dtype != AKVS_BF16 && dtype != AKVS_F16) return AKVS_ERR_UNSUPPORTED;
   return launch_quantize(dtype, x, n, n_kv_heads, head_dim, bits, codes, meta, reinterpret_cast<cudaStream_t>(stream));
 }
 

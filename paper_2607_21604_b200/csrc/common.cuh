@@ -9,7 +9,12 @@
 #include "akvs.h"
 
 typedef __nv_bfloat16 bf16;
+typedef __half f16;
 
+// Model dtypes: AKVS_F32 (everything float), AKVS_BF16 and AKVS_F16 (weights, unit cache,
+// activations and K/V outputs in that 16-bit type).  Accumulation, the residual stream,
+// softmax, norms, offsets and scores are float in every mode.  The tensor cores take either
+// 16-bit type at the same rate, but both operands of one MMA must have the same type.
 #define AKVS_TRY(expr)                              \
   do {                                              \
     int32_t rc_ = (expr);                           \
@@ -21,10 +26,46 @@ typedef __nv_bfloat16 bf16;
     if ((expr) != cudaSuccess) return AKVS_ERR_CUDA; \
   } while (0)
 
+// Every kernel launch of the library goes through this: it counts the launch (the count is
+// what akvs_launch_count reports) and turns a launch failure into an error code.
+extern unsigned long long g_akvs_launches;
 #define AKVS_LAUNCHED()                             \
   do {                                              \
+    ++g_akvs_launches;                              \
     if (cudaPeekAtLastError() != cudaSuccess) return AKVS_ERR_CUDA; \
   } while (0)
+
+// Optional per-launch timing of one kernel class with CUDA events on the launching stream
+// (akvs_prof_*).  kind: 1 = tensor-core linear layers, 2 = correction pass, 3 = attention.
+void akvs_prof_mark(int kind, int sub, double work, bool begin, cudaStream_t st);
+struct ProfScope {
+  int kind, sub; double work; cudaStream_t st;
+  ProfScope(int k, int s, double w, cudaStream_t t) : kind(k), sub(s), work(w), st(t) { akvs_prof_mark(k, s, w, true, t); }
+  ~ProfScope() { akvs_prof_mark(kind, sub, work, false, st); }
+};
+
+#include <type_traits>
+// Calls f(T{}) with T = float | bf16 | f16 for the model dtype.
+template <typename F>
+static inline int32_t dispatch_dtype(int dtype, F&& f) {
+  switch (dtype) {
+    case AKVS_F32: return f(float{});
+    case AKVS_BF16: return f(bf16{});
+    case AKVS_F16: return f(f16{});
+    default: return AKVS_ERR_UNSUPPORTED;
+  }
+}
+// Calls f(std::integral_constant<int, FMT>{}) for the cache format.
+template <typename F>
+static inline int32_t dispatch_fmt(int fmt, F&& f) {
+  switch (fmt) {
+    case AKVS_KV_NATIVE: return f(std::integral_constant<int, AKVS_KV_NATIVE>{});
+    case AKVS_KV_Q4: return f(std::integral_constant<int, AKVS_KV_Q4>{});
+    case AKVS_KV_Q2: return f(std::integral_constant<int, AKVS_KV_Q2>{});
+    default: return AKVS_ERR_UNSUPPORTED;
+  }
+}
+static inline size_t dtype_size(int dtype) { return dtype == AKVS_F32 ? 4 : 2; }
 
 static inline int64_t akvs_align_up(int64_t x, int64_t a) { return (x + a - 1) / a * a; }
 static inline int akvs_cdiv(int64_t a, int64_t b) { return (int)((a + b - 1) / b); }
@@ -35,6 +76,7 @@ static inline int akvs_cdiv(int64_t a, int64_t b) { return (int)((a + b - 1) / b
 template <typename T> struct VecOf;
 template <> struct VecOf<float> { static constexpr int N = 4; };
 template <> struct VecOf<bf16> { static constexpr int N = 8; };
+template <> struct VecOf<f16> { static constexpr int N = 8; };
 
 __device__ __forceinline__ void ld16(const float* p, float (&o)[4]) {
   float4 v = *reinterpret_cast<const float4*>(p);
@@ -65,11 +107,45 @@ __device__ __forceinline__ void st16(bf16* p, const float (&o)[8]) {
   *reinterpret_cast<uint4*>(p) = v;
 }
 
+__device__ __forceinline__ void ld16(const f16* p, float (&o)[8]) {
+  uint4 v = *reinterpret_cast<const uint4*>(p);
+  const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&w[i]));
+    o[2 * i] = f.x;
+    o[2 * i + 1] = f.y;
+  }
+}
+// float -> half with saturation to the largest finite value (no infinities are produced)
+__device__ __forceinline__ uint32_t pack_f16x2(float a, float b) {
+  a = fminf(fmaxf(a, -65504.f), 65504.f);
+  b = fminf(fmaxf(b, -65504.f), 65504.f);
+  __half2 h = __floats2half2_rn(a, b);
+  return *reinterpret_cast<uint32_t*>(&h);
+}
+__device__ __forceinline__ void st16(f16* p, const float (&o)[8]) {
+  uint4 v;
+  v.x = pack_f16x2(o[0], o[1]);
+  v.y = pack_f16x2(o[2], o[3]);
+  v.z = pack_f16x2(o[4], o[5]);
+  v.w = pack_f16x2(o[6], o[7]);
+  *reinterpret_cast<uint4*>(p) = v;
+}
+
+template <typename T> __device__ __forceinline__ uint32_t pack2(float a, float b);
+template <> __device__ __forceinline__ uint32_t pack2<bf16>(float a, float b) { return pack_bf16x2(a, b); }
+template <> __device__ __forceinline__ uint32_t pack2<f16>(float a, float b) { return pack_f16x2(a, b); }
+
 __device__ __forceinline__ float to_f(float x) { return x; }
+__device__ __forceinline__ float to_f(f16 x) { return __half2float(x); }
 __device__ __forceinline__ float to_f(bf16 x) { return __bfloat162float(x); }
 template <typename T> __device__ __forceinline__ T from_f(float x);
 template <> __device__ __forceinline__ float from_f<float>(float x) { return x; }
 template <> __device__ __forceinline__ bf16 from_f<bf16>(float x) { return __float2bfloat16_rn(x); }
+template <> __device__ __forceinline__ f16 from_f<f16>(float x) {
+  return __float2half_rn(fminf(fmaxf(x, -65504.f), 65504.f));
+}
 
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
@@ -127,9 +203,9 @@ int32_t launch_quantize(int dtype, const void* x, int n, int n_kv, int hd, int b
 int32_t launch_linear_simt(int dtype, const void* x, const void* w, const void* w2, void* y, float* resid,
                            int M, int N, int K, int ldy, cudaStream_t st);
 
-// bf16 tensor-core linear layers (gemm_tc.cu).  epi 0: out[i] = x w[i]^T; 1: out[0] (float) += x w[0]^T;
+// 16-bit tensor-core linear layers (gemm_tc.cu), dtype AKVS_BF16 or AKVS_F16.  epi 0: out[i] = x w[i]^T; 1: out[0] (float) += x w[0]^T;
 // 2: out[0] = silu(x w[0]^T) * (x w[1]^T).
-int32_t launch_linear_tc(int epi, const void* x, int M, int K, int n_seg, const void* const* w, const int* n,
+int32_t launch_linear_tc(int dtype, int epi, const void* x, int M, int K, int n_seg, const void* const* w, const int* n,
                          void* const* out, const int* ldc, int32_t* status, cudaStream_t st);
 
 int32_t launch_attention_simt(int dtype, const void* q, const void* k, const void* v, void* out,

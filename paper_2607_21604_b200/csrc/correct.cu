@@ -1,8 +1,8 @@
 // Probe selection, per-unit offset estimation and the correction pass
 // (paper Section 3.3 and Algorithm 1 lines 2, 5-8).
 //
-// Layouts: fresh rows [n_rows][n_kv][hd]; one layer of the unit store [store_tok][n_kv][hd]
-// (model dtype) or packed 2/4-bit codes with half2 (scale, min) per 64-dim group;
+// Layouts: fresh rows [n_rows][n_kv][hd] (type T); one layer of the unit store
+// [store_tok][n_kv][hd] (type TW, equal to T in every shipped configuration) or packed 2/4-bit codes with half2 (scale, min) per 64-dim group;
 // outputs [T][n_kv][hd].  A "pair chunk" is a 16-byte vector of the lower half of a head
 // together with its RoPE partner 16 bytes in the upper half; one thread owns one pair chunk
 // so that the re-alignment rotation needs no exchange between threads and every global
@@ -99,7 +99,7 @@ int32_t launch_row_maps(const int32_t* rows, int n_rows, const int32_t* sk_idx, 
 // Divergence scores at the check layer (Section 3.3): one warp per context token,
 // d_K = || k_fresh - Rot(off_u) k_cached ||_2 over all kv heads, d_V likewise.
 // ---------------------------------------------------------------------------------------
-template <typename T, int FMT>
+template <typename T, typename TW, int FMT>
 __global__ void scores_kernel(KvLayer kv, ReqMaps maps, const T* __restrict__ k_fresh, const T* __restrict__ v_fresh,
                               int N, int n_kv, int hd, const float2* __restrict__ table, float* __restrict__ d_k,
                               float* __restrict__ d_v) {
@@ -115,8 +115,8 @@ __global__ void scores_kernel(KvLayer kv, ReqMaps maps, const T* __restrict__ k_
   for (int pc = lane; pc < n_kv * ch; pc += 32) {
     const int h = pc / ch, c = pc % ch;
     float lo[V], hi[V], flo[V], fhi[V];
-    load_cached_chunk<T, FMT>(kv.k, kv.k_meta, src, n_kv, hd, h, c * V, lo);
-    load_cached_chunk<T, FMT>(kv.k, kv.k_meta, src, n_kv, hd, h, half + c * V, hi);
+    load_cached_chunk<TW, FMT>(kv.k, kv.k_meta, src, n_kv, hd, h, c * V, lo);
+    load_cached_chunk<TW, FMT>(kv.k, kv.k_meta, src, n_kv, hd, h, half + c * V, hi);
     const T* fp = k_fresh + ((size_t)j * n_kv + h) * hd + c * V;
     ld16(fp, flo);
     ld16(fp + half, fhi);
@@ -127,8 +127,8 @@ __global__ void scores_kernel(KvLayer kv, ReqMaps maps, const T* __restrict__ k_
       const float b = fhi[i] - (hi[i] * t.x + lo[i] * t.y);
       sk += a * a + b * b;
     }
-    load_cached_chunk<T, FMT>(kv.v, kv.v_meta, src, n_kv, hd, h, c * V, lo);
-    load_cached_chunk<T, FMT>(kv.v, kv.v_meta, src, n_kv, hd, h, half + c * V, hi);
+    load_cached_chunk<TW, FMT>(kv.v, kv.v_meta, src, n_kv, hd, h, c * V, lo);
+    load_cached_chunk<TW, FMT>(kv.v, kv.v_meta, src, n_kv, hd, h, half + c * V, hi);
     const T* vp = v_fresh + ((size_t)j * n_kv + h) * hd + c * V;
     ld16(vp, flo);
     ld16(vp + half, fhi);
@@ -143,19 +143,6 @@ __global__ void scores_kernel(KvLayer kv, ReqMaps maps, const T* __restrict__ k_
   if (lane == 0) { d_k[j] = sqrtf(sk); d_v[j] = sqrtf(sv); }
 }
 
-#define DISPATCH_T_FMT(KERNEL, GRID, BLOCK, SMEM, ST, ...)                                          \
-  do {                                                                                              \
-    if (dtype == AKVS_F32) {                                                                        \
-      if (kv.fmt == AKVS_KV_NATIVE) KERNEL<float, AKVS_KV_NATIVE><<<GRID, BLOCK, SMEM, ST>>>(__VA_ARGS__); \
-      else if (kv.fmt == AKVS_KV_Q4) KERNEL<float, AKVS_KV_Q4><<<GRID, BLOCK, SMEM, ST>>>(__VA_ARGS__);     \
-      else KERNEL<float, AKVS_KV_Q2><<<GRID, BLOCK, SMEM, ST>>>(__VA_ARGS__);                       \
-    } else {                                                                                        \
-      if (kv.fmt == AKVS_KV_NATIVE) KERNEL<bf16, AKVS_KV_NATIVE><<<GRID, BLOCK, SMEM, ST>>>(__VA_ARGS__);  \
-      else if (kv.fmt == AKVS_KV_Q4) KERNEL<bf16, AKVS_KV_Q4><<<GRID, BLOCK, SMEM, ST>>>(__VA_ARGS__);      \
-      else KERNEL<bf16, AKVS_KV_Q2><<<GRID, BLOCK, SMEM, ST>>>(__VA_ARGS__);                        \
-    }                                                                                               \
-  } while (0)
-
 static int32_t check_kv_shape(int dtype, const KvLayer& kv, int hd) {
   const int V = dtype == AKVS_F32 ? 4 : 8;
   if (hd % (2 * V) != 0) return AKVS_ERR_UNSUPPORTED;
@@ -169,19 +156,15 @@ int32_t launch_scores(int dtype, const KvLayer& kv, const ReqMaps& maps, const v
   if (N == 0) return AKVS_OK;
   AKVS_TRY(check_kv_shape(dtype, kv, hd));
   const int grid = akvs_cdiv(N, 8);
-  if (dtype == AKVS_F32) {
-    const float *kf = (const float*)k_fresh, *vf = (const float*)v_fresh;
-    if (kv.fmt == AKVS_KV_NATIVE) scores_kernel<float, AKVS_KV_NATIVE><<<grid, 256, 0, st>>>(kv, maps, kf, vf, N, n_kv, hd, table, d_k, d_v);
-    else if (kv.fmt == AKVS_KV_Q4) scores_kernel<float, AKVS_KV_Q4><<<grid, 256, 0, st>>>(kv, maps, kf, vf, N, n_kv, hd, table, d_k, d_v);
-    else scores_kernel<float, AKVS_KV_Q2><<<grid, 256, 0, st>>>(kv, maps, kf, vf, N, n_kv, hd, table, d_k, d_v);
-  } else {
-    const bf16 *kf = (const bf16*)k_fresh, *vf = (const bf16*)v_fresh;
-    if (kv.fmt == AKVS_KV_NATIVE) scores_kernel<bf16, AKVS_KV_NATIVE><<<grid, 256, 0, st>>>(kv, maps, kf, vf, N, n_kv, hd, table, d_k, d_v);
-    else if (kv.fmt == AKVS_KV_Q4) scores_kernel<bf16, AKVS_KV_Q4><<<grid, 256, 0, st>>>(kv, maps, kf, vf, N, n_kv, hd, table, d_k, d_v);
-    else scores_kernel<bf16, AKVS_KV_Q2><<<grid, 256, 0, st>>>(kv, maps, kf, vf, N, n_kv, hd, table, d_k, d_v);
-  }
-  AKVS_LAUNCHED();
-  return AKVS_OK;
+  return dispatch_dtype(dtype, [&](auto tag) -> int32_t {
+    using T = decltype(tag);
+    return dispatch_fmt(kv.fmt, [&](auto f) -> int32_t {
+      scores_kernel<T, T, decltype(f)::value><<<grid, 256, 0, st>>>(kv, maps, (const T*)k_fresh, (const T*)v_fresh, N,
+                                                                   n_kv, hd, table, d_k, d_v);
+      AKVS_LAUNCHED();
+      return AKVS_OK;
+    });
+  });
 }
 
 // ---------------------------------------------------------------------------------------
@@ -320,7 +303,7 @@ int32_t launch_select(const float* d_k, const float* d_v, const int32_t* ctx_off
 // ---------------------------------------------------------------------------------------
 constexpr int OFF_WARPS = 8;
 
-template <typename T, int FMT>
+template <typename T, typename TW, int FMT>
 __global__ void __launch_bounds__(OFF_WARPS * 32)
 offsets_kernel(KvLayer kv, ReqMaps maps, const int32_t* __restrict__ probe_off, const int32_t* __restrict__ sk_idx,
                const int32_t* __restrict__ sv_idx, const T* __restrict__ k_fresh, const T* __restrict__ v_fresh,
@@ -346,7 +329,7 @@ offsets_kernel(KvLayer kv, ReqMaps maps, const int32_t* __restrict__ probe_off, 
     for (int e = lane; e < half; e += 32) {
       float lo, hi;
       if constexpr (FMT == AKVS_KV_NATIVE) {
-        const T* cp = reinterpret_cast<const T*>(cbase) + ((size_t)src * n_kv + h) * hd;
+        const TW* cp = reinterpret_cast<const TW*>(cbase) + ((size_t)src * n_kv + h) * hd;
         lo = to_f(cp[e]);
         hi = to_f(cp[half + e]);
       } else {
@@ -386,19 +369,15 @@ int32_t launch_offsets(int dtype, const KvLayer& kv, const ReqMaps& maps, const 
   AKVS_TRY(check_kv_shape(dtype, kv, hd));
   const dim3 grid(M, n_kv, 2);
   const size_t smem = (size_t)OFF_WARPS * hd * sizeof(float);
-  if (dtype == AKVS_F32) {
-    const float *kf = (const float*)k_fresh, *vf = (const float*)v_fresh;
-    if (kv.fmt == AKVS_KV_NATIVE) offsets_kernel<float, AKVS_KV_NATIVE><<<grid, OFF_WARPS * 32, smem, st>>>(kv, maps, probe_off, sk_idx, sv_idx, kf, vf, n_kv, hd, table, mu_k, mu_v);
-    else if (kv.fmt == AKVS_KV_Q4) offsets_kernel<float, AKVS_KV_Q4><<<grid, OFF_WARPS * 32, smem, st>>>(kv, maps, probe_off, sk_idx, sv_idx, kf, vf, n_kv, hd, table, mu_k, mu_v);
-    else offsets_kernel<float, AKVS_KV_Q2><<<grid, OFF_WARPS * 32, smem, st>>>(kv, maps, probe_off, sk_idx, sv_idx, kf, vf, n_kv, hd, table, mu_k, mu_v);
-  } else {
-    const bf16 *kf = (const bf16*)k_fresh, *vf = (const bf16*)v_fresh;
-    if (kv.fmt == AKVS_KV_NATIVE) offsets_kernel<bf16, AKVS_KV_NATIVE><<<grid, OFF_WARPS * 32, smem, st>>>(kv, maps, probe_off, sk_idx, sv_idx, kf, vf, n_kv, hd, table, mu_k, mu_v);
-    else if (kv.fmt == AKVS_KV_Q4) offsets_kernel<bf16, AKVS_KV_Q4><<<grid, OFF_WARPS * 32, smem, st>>>(kv, maps, probe_off, sk_idx, sv_idx, kf, vf, n_kv, hd, table, mu_k, mu_v);
-    else offsets_kernel<bf16, AKVS_KV_Q2><<<grid, OFF_WARPS * 32, smem, st>>>(kv, maps, probe_off, sk_idx, sv_idx, kf, vf, n_kv, hd, table, mu_k, mu_v);
-  }
-  AKVS_LAUNCHED();
-  return AKVS_OK;
+  return dispatch_dtype(dtype, [&](auto tag) -> int32_t {
+    using T = decltype(tag);
+    return dispatch_fmt(kv.fmt, [&](auto f) -> int32_t {
+      offsets_kernel<T, T, decltype(f)::value><<<grid, OFF_WARPS * 32, smem, st>>>(
+          kv, maps, probe_off, sk_idx, sv_idx, (const T*)k_fresh, (const T*)v_fresh, n_kv, hd, table, mu_k, mu_v);
+      AKVS_LAUNCHED();
+      return AKVS_OK;
+    });
+  });
 }
 
 // ---------------------------------------------------------------------------------------
@@ -408,7 +387,7 @@ int32_t launch_offsets(int dtype, const KvLayer& kv, const ReqMaps& maps, const 
 //   V likewise with S^V (no rotation);  query token i: fresh K/V of row P + i.
 // One thread per pair chunk; it moves 4 x 16 B in and 4 x 16 B out.
 // ---------------------------------------------------------------------------------------
-template <typename T, int FMT>
+template <typename T, typename TW, int FMT>
 __global__ void __launch_bounds__(256)
 correct_kernel(KvLayer kv, ReqMaps maps, const T* __restrict__ k_fresh, const T* __restrict__ v_fresh,
                const float* __restrict__ w_k, const float* __restrict__ w_v, const float* __restrict__ mu_k,
@@ -444,8 +423,8 @@ correct_kernel(KvLayer kv, ReqMaps maps, const T* __restrict__ k_fresh, const T*
       ld16(fp + half, hi);
     } else {
       float clo[V], chi[V];
-      load_cached_chunk<T, FMT>(kv.k, kv.k_meta, src, n_kv, hd, h, c * V, clo);
-      load_cached_chunk<T, FMT>(kv.k, kv.k_meta, src, n_kv, hd, h, half + c * V, chi);
+      load_cached_chunk<TW, FMT>(kv.k, kv.k_meta, src, n_kv, hd, h, c * V, clo);
+      load_cached_chunk<TW, FMT>(kv.k, kv.k_meta, src, n_kv, hd, h, half + c * V, chi);
       const float2* rot = table + (size_t)maps.ctx_off[u] * half + c * V;
       const float* mu = mu_k + ((size_t)u * n_kv + h) * hd + c * V;
 #pragma unroll
@@ -467,8 +446,8 @@ correct_kernel(KvLayer kv, ReqMaps maps, const T* __restrict__ k_fresh, const T*
       ld16(fp, lo);
       ld16(fp + half, hi);
     } else {
-      load_cached_chunk<T, FMT>(kv.v, kv.v_meta, src, n_kv, hd, h, c * V, lo);
-      load_cached_chunk<T, FMT>(kv.v, kv.v_meta, src, n_kv, hd, h, half + c * V, hi);
+      load_cached_chunk<TW, FMT>(kv.v, kv.v_meta, src, n_kv, hd, h, c * V, lo);
+      load_cached_chunk<TW, FMT>(kv.v, kv.v_meta, src, n_kv, hd, h, half + c * V, hi);
       if (w_k) {
         const float* mu = mu_v + ((size_t)u * n_kv + h) * hd + c * V;
 #pragma unroll
@@ -494,19 +473,20 @@ int32_t launch_correct(int dtype, const KvLayer& kv, const ReqMaps& maps, const 
   const int64_t total = (int64_t)T_tok * n_kv * (hd / 2 / V);
   int64_t want = (total + 255) / 256;
   const int grid = (int)(want < 148 * 8 ? want : 148 * 8);   // grid-stride; 8 CTAs of 256 threads per SM
-  if (dtype == AKVS_F32) {
-    const float *kf = (const float*)k_fresh, *vf = (const float*)v_fresh;
-    float *ok = (float*)out_k, *ov = (float*)out_v;
-    if (kv.fmt == AKVS_KV_NATIVE) correct_kernel<float, AKVS_KV_NATIVE><<<grid, 256, 0, st>>>(kv, maps, kf, vf, w_k, w_v, mu_k, mu_v, N, T_tok, n_probe_rows, n_kv, hd, table, ok, ov);
-    else if (kv.fmt == AKVS_KV_Q4) correct_kernel<float, AKVS_KV_Q4><<<grid, 256, 0, st>>>(kv, maps, kf, vf, w_k, w_v, mu_k, mu_v, N, T_tok, n_probe_rows, n_kv, hd, table, ok, ov);
-    else correct_kernel<float, AKVS_KV_Q2><<<grid, 256, 0, st>>>(kv, maps, kf, vf, w_k, w_v, mu_k, mu_v, N, T_tok, n_probe_rows, n_kv, hd, table, ok, ov);
-  } else {
-    const bf16 *kf = (const bf16*)k_fresh, *vf = (const bf16*)v_fresh;
-    bf16 *ok = (bf16*)out_k, *ov = (bf16*)out_v;
-    if (kv.fmt == AKVS_KV_NATIVE) correct_kernel<bf16, AKVS_KV_NATIVE><<<grid, 256, 0, st>>>(kv, maps, kf, vf, w_k, w_v, mu_k, mu_v, N, T_tok, n_probe_rows, n_kv, hd, table, ok, ov);
-    else if (kv.fmt == AKVS_KV_Q4) correct_kernel<bf16, AKVS_KV_Q4><<<grid, 256, 0, st>>>(kv, maps, kf, vf, w_k, w_v, mu_k, mu_v, N, T_tok, n_probe_rows, n_kv, hd, table, ok, ov);
-    else correct_kernel<bf16, AKVS_KV_Q2><<<grid, 256, 0, st>>>(kv, maps, kf, vf, w_k, w_v, mu_k, mu_v, N, T_tok, n_probe_rows, n_kv, hd, table, ok, ov);
-  }
-  AKVS_LAUNCHED();
-  return AKVS_OK;
+  // algorithmic bytes: every context K and V element read once in its cache format and
+  // written once; fresh rows and query rows copied; 8 bytes of weights per context token
+  const double in_b = kv.fmt == AKVS_KV_NATIVE ? (double)dtype_size(dtype) : kv.fmt / 8.0 + 4.0 / 64.0;
+  const double out_b = (double)dtype_size(dtype);
+  const double bytes = 2.0 * n_kv * hd * ((double)N * (in_b + out_b) + (double)n_query * 2 * out_b) + 8.0 * N;
+  ProfScope prof(2, kv.fmt, bytes, st);
+  return dispatch_dtype(dtype, [&](auto tag) -> int32_t {
+    using T = decltype(tag);
+    return dispatch_fmt(kv.fmt, [&](auto f) -> int32_t {
+      correct_kernel<T, T, decltype(f)::value><<<grid, 256, 0, st>>>(kv, maps, (const T*)k_fresh, (const T*)v_fresh, w_k,
+                                                                    w_v, mu_k, mu_v, N, T_tok, n_probe_rows, n_kv, hd,
+                                                                    table, (T*)out_k, (T*)out_v);
+      AKVS_LAUNCHED();
+      return AKVS_OK;
+    });
+  });
 }

@@ -28,12 +28,12 @@ __global__ void embed_kernel(const T* __restrict__ emb, const int32_t* __restric
 int32_t launch_embed(int dtype, const void* tok_emb, const int32_t* ids, const int32_t* gather, int n, int d,
                      float* h, cudaStream_t st) {
   if (n == 0) return AKVS_OK;
-  if (dtype == AKVS_F32)
-    embed_kernel<float><<<n, 128, 0, st>>>((const float*)tok_emb, ids, gather, n, d, h);
-  else
-    embed_kernel<bf16><<<n, 128, 0, st>>>((const bf16*)tok_emb, ids, gather, n, d, h);
-  AKVS_LAUNCHED();
-  return AKVS_OK;
+  return dispatch_dtype(dtype, [&](auto tag) -> int32_t {
+    using T = decltype(tag);
+    embed_kernel<T><<<n, 128, 0, st>>>((const T*)tok_emb, ids, gather, n, d, h);
+    AKVS_LAUNCHED();
+    return AKVS_OK;
+  });
 }
 
 __global__ void gather_rows_kernel(const float* __restrict__ src, const int32_t* __restrict__ rows, int d,
@@ -106,8 +106,8 @@ rmsnorm_kernel(const float* __restrict__ h, const float* __restrict__ gain, floa
         reinterpret_cast<float4*>(xp)[c] = make_float4(o0, o1, o2, o3);
       } else {
         uint2 pk;
-        pk.x = pack_bf16x2(o0, o1);
-        pk.y = pack_bf16x2(o2, o3);
+        pk.x = pack2<TO>(o0, o1);
+        pk.y = pack2<TO>(o2, o3);
         reinterpret_cast<uint2*>(xp)[c] = pk;
       }
     }
@@ -118,12 +118,12 @@ int32_t launch_rmsnorm(int out_dtype, const float* h, const float* gain, float e
                        cudaStream_t st) {
   if (n == 0) return AKVS_OK;
   if (d % 4 != 0 || d > RMS_THREADS * 4 * RMS_MAX_V) return AKVS_ERR_UNSUPPORTED;
-  if (out_dtype == AKVS_F32)
-    rmsnorm_kernel<float><<<n, RMS_THREADS, 0, st>>>(h, gain, eps, d, (float*)x);
-  else
-    rmsnorm_kernel<bf16><<<n, RMS_THREADS, 0, st>>>(h, gain, eps, d, (bf16*)x);
-  AKVS_LAUNCHED();
-  return AKVS_OK;
+  return dispatch_dtype(out_dtype, [&](auto tag) -> int32_t {
+    using T = decltype(tag);
+    rmsnorm_kernel<T><<<n, RMS_THREADS, 0, st>>>(h, gain, eps, d, (T*)x);
+    AKVS_LAUNCHED();
+    return AKVS_OK;
+  });
 }
 
 // ---------------------------------------------------------------------------------------
@@ -194,12 +194,12 @@ int32_t launch_rope(int dtype, void* x, const int32_t* pos, int n, int n_heads, 
   if (hd % (2 * V) != 0) return AKVS_ERR_UNSUPPORTED;
   const int64_t total = (int64_t)n * n_heads * (hd / 2 / V);
   const int blocks = akvs_cdiv(total, 256);
-  if (dtype == AKVS_F32)
-    rope_kernel<float><<<blocks, 256, 0, st>>>((float*)x, pos, n, n_heads, hd, ld, table, (double)base);
-  else
-    rope_kernel<bf16><<<blocks, 256, 0, st>>>((bf16*)x, pos, n, n_heads, hd, ld, table, (double)base);
-  AKVS_LAUNCHED();
-  return AKVS_OK;
+  return dispatch_dtype(dtype, [&](auto tag) -> int32_t {
+    using T = decltype(tag);
+    rope_kernel<T><<<blocks, 256, 0, st>>>((T*)x, pos, n, n_heads, hd, ld, table, (double)base);
+    AKVS_LAUNCHED();
+    return AKVS_OK;
+  });
 }
 
 // ---------------------------------------------------------------------------------------
@@ -245,10 +245,10 @@ int32_t launch_quantize(int dtype, const void* x, int n, int n_kv, int hd, int b
   if (hd % 64 != 0 || (bits != 2 && bits != 4)) return AKVS_ERR_UNSUPPORTED;
   const int64_t n_groups = (int64_t)n * n_kv * (hd / 64);
   const int blocks = akvs_cdiv(n_groups, 8);
-  if (dtype == AKVS_F32)
-    quantize_kernel<float><<<blocks, 256, 0, st>>>((const float*)x, n_groups, bits, (uint8_t*)codes, (__half2*)meta);
-  else
-    quantize_kernel<bf16><<<blocks, 256, 0, st>>>((const bf16*)x, n_groups, bits, (uint8_t*)codes, (__half2*)meta);
-  AKVS_LAUNCHED();
-  return AKVS_OK;
+  return dispatch_dtype(dtype, [&](auto tag) -> int32_t {
+    using T = decltype(tag);
+    quantize_kernel<T><<<blocks, 256, 0, st>>>((const T*)x, n_groups, bits, (uint8_t*)codes, (__half2*)meta);
+    AKVS_LAUNCHED();
+    return AKVS_OK;
+  });
 }

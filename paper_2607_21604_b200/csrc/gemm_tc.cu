@@ -1,5 +1,6 @@
-// bf16 linear layers on the 5th-generation tensor cores (tcgen05), float accumulation in
-// tensor memory.  y = x W^T with x [M][K] and W [N][K], both K-major, staged by TMA in
+// Linear layers of the 16-bit models (bfloat16 or float16, both operands the same type) on
+// the 5th-generation tensor cores (tcgen05), float accumulation in tensor memory.  y = x W^T with
+// x [M][K] and W [N][K], both K-major, staged by TMA in
 // 128-byte-swizzled 64-wide k slabs.
 //
 // Persistent kernel, one CTA per SM, 6 warps:
@@ -27,9 +28,10 @@ struct GemmParams {
   int M, K, tiles_m, tiles_n;
   int n_seg;
   int seg_blocks[3];      // 128-row blocks of each B matrix
-  void* seg_out[3];       // output of each segment (bf16 [M][ldc], or float for EPI_RESID)
+  void* seg_out[3];       // output of each segment (16-bit [M][ldc], or float for EPI_RESID)
   int seg_ldc[3];
   int32_t* status;
+  uint32_t idesc;         // tcgen05 instruction descriptor (operand formats, M, N)
 };
 
 // Which weight matrix and which of its rows the 128-row block `block` of the concatenated
@@ -44,7 +46,7 @@ __device__ __forceinline__ void locate(const GemmParams& p, int block, int& seg,
   row = block * BNH;
 }
 
-template <int EPI>
+template <int EPI, typename T>
 __global__ void __launch_bounds__(THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB0,
                const __grid_constant__ CUtensorMap tmB1, const __grid_constant__ CUtensorMap tmB2,
@@ -113,7 +115,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
-      constexpr uint32_t idesc = tc::idesc_bf16(BM, 2 * BNH, 0);
+      const uint32_t idesc = p.idesc;
       int s = 0;
       uint32_t ph = 0;
       bool ok = true;
@@ -132,7 +134,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           for (int k = 0; k < BK / 16; ++k) {
             const uint64_t da = tc::smem_desc_k_sw128(a_addr + k * 32);
             const uint64_t db = tc::smem_desc_k_sw128(b_addr + k * 32);
-            tc::mma_bf16(d_tmem, da, db, idesc, (kb | k) != 0);
+            tc::mma_f16(d_tmem, da, db, idesc, (kb | k) != 0);
           }
           tc::mma_commit(&empty[s]);            // frees the stage once these MMAs retire
           if (++s == STAGES) { s = 0; ph ^= 1; }
@@ -154,7 +156,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       const int row = tm * BM + quad * 32 + lane;
       const uint32_t t_addr = tmem_base + acc * (2 * BNH) + ((uint32_t)(quad * 32) << 16);
       if (EPI == EPI_SWIGLU) {
-        bf16* out = reinterpret_cast<bf16*>(p.seg_out[0]);
+        T* out = reinterpret_cast<T*>(p.seg_out[0]);
         const int ldc = p.seg_ldc[0];
         const int n_valid = p.seg_blocks[0] * BNH;
 #pragma unroll 1
@@ -165,7 +167,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           tc::tmem_ld_wait();
           const int col = tn * BNH + c * 32;
           if (row < p.M && col < n_valid) {
-            bf16* o = out + (size_t)row * ldc + col;
+            T* o = out + (size_t)row * ldc + col;
 #pragma unroll
             for (int v = 0; v < 4; ++v) {
               float r[8];
@@ -201,7 +203,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                   *reinterpret_cast<float4*>(o + v * 4) = t;
                 }
               } else {
-                bf16* o = reinterpret_cast<bf16*>(p.seg_out[seg]) + (size_t)row * ldc + col;
+                T* o = reinterpret_cast<T*>(p.seg_out[seg]) + (size_t)row * ldc + col;
 #pragma unroll
                 for (int v = 0; v < 4; ++v) {
                   float r[8];
@@ -262,7 +264,7 @@ int sm_count() {
 
 }  // namespace
 
-int32_t encode_tmap_2d_bf16(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, uint64_t ld,
+int32_t encode_tmap_2d_16bit(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, uint64_t ld,
                             uint32_t box_rows) {
   EncodeFn enc = get_encoder();
   if (!enc) return AKVS_ERR_CUDA;
@@ -271,13 +273,13 @@ int32_t encode_tmap_2d_bf16(CUtensorMap* map, const void* base, uint64_t rows, u
   const cuuint64_t strides[1] = {ld * 2};
   const cuuint32_t box[2] = {64, box_rows};
   const cuuint32_t estr[2] = {1, 1};
-  const CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+  const CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_UINT16, 2, const_cast<void*>(base), dims, strides, box, estr,
                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS ? AKVS_OK : AKVS_ERR_CUDA;
 }
 
-int32_t encode_tmap_3d_bf16(CUtensorMap* map, const void* base, uint64_t d0, uint64_t d1, uint64_t d2, uint64_t ld1,
+int32_t encode_tmap_3d_16bit(CUtensorMap* map, const void* base, uint64_t d0, uint64_t d1, uint64_t d2, uint64_t ld1,
                             uint64_t ld2, uint32_t b1, uint32_t b2) {
   EncodeFn enc = get_encoder();
   if (!enc) return AKVS_ERR_CUDA;
@@ -286,25 +288,29 @@ int32_t encode_tmap_3d_bf16(CUtensorMap* map, const void* base, uint64_t d0, uin
   const cuuint64_t strides[2] = {ld1 * 2, ld2 * 2};
   const cuuint32_t box[3] = {64, b1, b2};
   const cuuint32_t estr[3] = {1, 1, 1};
-  const CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+  const CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_UINT16, 3, const_cast<void*>(base), dims, strides, box, estr,
                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS ? AKVS_OK : AKVS_ERR_CUDA;
 }
 
-// x [M][K] bf16; up to three weight matrices w[i] [n[i]][K] (n[i] a multiple of 128) whose
+// x [M][K]; up to three weight matrices w[i] [n[i]][K] of the same 16-bit type (n[i] a multiple of 128) whose
 // outputs go to out[i] with row stride ldc[i].
-//   epi 0: out[i] = x w[i]^T (bf16);   epi 1: out[0] (float) += x w[0]^T;
-//   epi 2: out[0] = silu(x w[0]^T) * (x w[1]^T) (bf16), n[0] == n[1].
-int32_t launch_linear_tc(int epi, const void* x, int M, int K, int n_seg, const void* const* w, const int* n,
+//   epi 0: out[i] = x w[i]^T (16-bit);   epi 1: out[0] (float) += x w[0]^T;
+//   epi 2: out[0] = silu(x w[0]^T) * (x w[1]^T) (16-bit), n[0] == n[1].
+int32_t launch_linear_tc(int dtype, int epi, const void* x, int M, int K, int n_seg, const void* const* w, const int* n,
                          void* const* out, const int* ldc, int32_t* status, cudaStream_t st) {
   if (M == 0) return AKVS_OK;
   if (K % 8 != 0 || n_seg < 1 || n_seg > 3) return AKVS_ERR_SHAPE;
+  if (dtype != AKVS_BF16 && dtype != AKVS_F16) return AKVS_ERR_UNSUPPORTED;
   static bool attr_set = false;
   if (!attr_set) {
-    AKVS_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI_STORE>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES));
-    AKVS_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI_RESID>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES));
-    AKVS_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI_SWIGLU>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES));
+    AKVS_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI_STORE, bf16>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES));
+    AKVS_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI_RESID, bf16>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES));
+    AKVS_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI_SWIGLU, bf16>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES));
+    AKVS_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI_STORE, f16>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES));
+    AKVS_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI_RESID, f16>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES));
+    AKVS_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI_SWIGLU, f16>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES));
     attr_set = true;
   }
   GemmParams p;
@@ -312,13 +318,15 @@ int32_t launch_linear_tc(int epi, const void* x, int M, int K, int n_seg, const 
   p.K = K;
   p.n_seg = n_seg;
   p.status = status;
+  const uint32_t fmt = dtype == AKVS_F16 ? tc::kF16 : tc::kBF16;
+  p.idesc = tc::idesc_f16(fmt, fmt, BM, 2 * BNH, 0);
   CUtensorMap tmA, tmB[3];
-  AKVS_TRY(encode_tmap_2d_bf16(&tmA, x, M, K, K, BM));
+  AKVS_TRY(encode_tmap_2d_16bit(&tmA, x, M, K, K, BM));
   int blocks = 0;
   for (int i = 0; i < 3; ++i) {
     const int s = i < n_seg ? i : 0;
     if (n[s] % BNH != 0) return AKVS_ERR_SHAPE;
-    AKVS_TRY(encode_tmap_2d_bf16(&tmB[i], w[s], n[s], K, K, BNH));
+    AKVS_TRY(encode_tmap_2d_16bit(&tmB[i], w[s], n[s], K, K, BNH));
     p.seg_blocks[i] = n[s] / BNH;
     p.seg_out[i] = out[i < n_seg && (epi != EPI_SWIGLU || i == 0) ? i : 0];
     p.seg_ldc[i] = ldc[i < n_seg && (epi != EPI_SWIGLU || i == 0) ? i : 0];
@@ -333,12 +341,21 @@ int32_t launch_linear_tc(int epi, const void* x, int M, int K, int n_seg, const 
   p.tiles_m = (M + BM - 1) / BM;
   const int n_tiles = p.tiles_m * p.tiles_n;
   const int grid = n_tiles < sm_count() ? n_tiles : sm_count();
-  switch (epi) {
-    case EPI_STORE: gemm_tc_kernel<EPI_STORE><<<grid, THREADS, SMEM_BYTES, st>>>(tmA, tmB[0], tmB[1], tmB[2], p); break;
-    case EPI_RESID: gemm_tc_kernel<EPI_RESID><<<grid, THREADS, SMEM_BYTES, st>>>(tmA, tmB[0], tmB[1], tmB[2], p); break;
-    case EPI_SWIGLU: gemm_tc_kernel<EPI_SWIGLU><<<grid, THREADS, SMEM_BYTES, st>>>(tmA, tmB[0], tmB[1], tmB[2], p); break;
-    default: return AKVS_ERR_INVALID_ARG;
+  double flops = 0;
+  for (int i = 0; i < n_seg; ++i) flops += 2.0 * M * (double)n[i] * K;
+  ProfScope prof(1, epi, flops, st);
+  if (epi < 0 || epi > 2) return AKVS_ERR_INVALID_ARG;
+#define AKVS_GEMM_LAUNCH(E, T) gemm_tc_kernel<E, T><<<grid, THREADS, SMEM_BYTES, st>>>(tmA, tmB[0], tmB[1], tmB[2], p)
+  if (dtype == AKVS_BF16) {
+    if (epi == EPI_STORE) AKVS_GEMM_LAUNCH(EPI_STORE, bf16);
+    else if (epi == EPI_RESID) AKVS_GEMM_LAUNCH(EPI_RESID, bf16);
+    else AKVS_GEMM_LAUNCH(EPI_SWIGLU, bf16);
+  } else {
+    if (epi == EPI_STORE) AKVS_GEMM_LAUNCH(EPI_STORE, f16);
+    else if (epi == EPI_RESID) AKVS_GEMM_LAUNCH(EPI_RESID, f16);
+    else AKVS_GEMM_LAUNCH(EPI_SWIGLU, f16);
   }
+#undef AKVS_GEMM_LAUNCH
   AKVS_LAUNCHED();
   return AKVS_OK;
 }

@@ -9,9 +9,9 @@
 // ---------------------------------------------------------------------------------------
 constexpr int SG_BM = 64, SG_BN = 64, SG_BK = 16;
 
-template <typename T, bool DUAL>
+template <typename T, typename TW, bool DUAL>
 __global__ void __launch_bounds__(256)
-linear_simt_kernel(const T* __restrict__ x, const T* __restrict__ w, const T* __restrict__ w2, T* __restrict__ y,
+linear_simt_kernel(const T* __restrict__ x, const TW* __restrict__ w, const TW* __restrict__ w2, T* __restrict__ y,
                    float* __restrict__ resid, int M, int N, int K, int ldy) {
   __shared__ float xs[SG_BK][SG_BM + 4];
   __shared__ float ws[SG_BK][SG_BN + 4];
@@ -68,15 +68,13 @@ int32_t launch_linear_simt(int dtype, const void* x, const void* w, const void* 
                            int M, int N, int K, int ldy, cudaStream_t st) {
   if (M == 0 || N == 0) return AKVS_OK;
   const dim3 grid(akvs_cdiv(N, SG_BN), akvs_cdiv(M, SG_BM));
-  if (dtype == AKVS_F32) {
-    if (w2) linear_simt_kernel<float, true><<<grid, 256, 0, st>>>((const float*)x, (const float*)w, (const float*)w2, (float*)y, resid, M, N, K, ldy);
-    else linear_simt_kernel<float, false><<<grid, 256, 0, st>>>((const float*)x, (const float*)w, nullptr, (float*)y, resid, M, N, K, ldy);
-  } else {
-    if (w2) linear_simt_kernel<bf16, true><<<grid, 256, 0, st>>>((const bf16*)x, (const bf16*)w, (const bf16*)w2, (bf16*)y, resid, M, N, K, ldy);
-    else linear_simt_kernel<bf16, false><<<grid, 256, 0, st>>>((const bf16*)x, (const bf16*)w, nullptr, (bf16*)y, resid, M, N, K, ldy);
-  }
-  AKVS_LAUNCHED();
-  return AKVS_OK;
+  return dispatch_dtype(dtype, [&](auto tag) -> int32_t {
+    using T = decltype(tag);
+    if (w2) linear_simt_kernel<T, T, true><<<grid, 256, 0, st>>>((const T*)x, (const T*)w, (const T*)w2, (T*)y, resid, M, N, K, ldy);
+    else linear_simt_kernel<T, T, false><<<grid, 256, 0, st>>>((const T*)x, (const T*)w, nullptr, (T*)y, resid, M, N, K, ldy);
+    AKVS_LAUNCHED();
+    return AKVS_OK;
+  });
 }
 
 // ---------------------------------------------------------------------------------------
@@ -189,12 +187,10 @@ int32_t launch_attention_simt(int dtype, const void* q, const void* k, const voi
                               cudaStream_t st) {
   if (R == 0) return AKVS_OK;
   if (n_kv <= 0 || n_q % n_kv != 0) return AKVS_ERR_SHAPE;
-  if (dtype == AKVS_F32) {
-    if (hd == 64) return launch_attention_simt_t<float, 64>(q, k, v, out, k_lo, k_hi, R, n_q, n_kv, st);
-    if (hd == 128) return launch_attention_simt_t<float, 128>(q, k, v, out, k_lo, k_hi, R, n_q, n_kv, st);
-  } else {
-    if (hd == 64) return launch_attention_simt_t<bf16, 64>(q, k, v, out, k_lo, k_hi, R, n_q, n_kv, st);
-    if (hd == 128) return launch_attention_simt_t<bf16, 128>(q, k, v, out, k_lo, k_hi, R, n_q, n_kv, st);
-  }
-  return AKVS_ERR_UNSUPPORTED;
+  return dispatch_dtype(dtype, [&](auto tag) -> int32_t {
+    using T = decltype(tag);
+    if (hd == 64) return launch_attention_simt_t<T, 64>(q, k, v, out, k_lo, k_hi, R, n_q, n_kv, st);
+    if (hd == 128) return launch_attention_simt_t<T, 128>(q, k, v, out, k_lo, k_hi, R, n_q, n_kv, st);
+    return AKVS_ERR_UNSUPPORTED;
+  });
 }

@@ -5,8 +5,9 @@ layer's weights can be produced without producing any other layer's: the 32B-cla
 configuration never has to be resident on the host in full.
 
 Weights: i.i.d. N(0, 0.02^2); stored [out_features][in_features]; rounded to bf16
-(round-to-nearest-even) for the bf16 configurations so that both consumers see the
-same representable values.  RMSNorm gains are 1.  Token ids are uniform on [0, vocab).
+(round-to-nearest-even) for the 16-bit configurations so that both consumers see the
+same representable values ("f16" additionally rounds the bf16 values to float16, which
+changes only magnitudes below 2^-17).  RMSNorm gains are 1.  Token ids are uniform on [0, vocab).
 Unit lengths are uniform on the closed interval the configuration names.
 """
 from __future__ import annotations
@@ -27,7 +28,7 @@ class ModelCfg:
     head_dim: int
     d_ff: int
     vocab: int
-    dtype: str            # "f32" | "bf16"
+    dtype: str            # "f32" | "bf16" | "f16" (bf16-valued weights in float16 containers)
     rope_base: float = 1.0e4
     rms_eps: float = 1.0e-6
 
@@ -123,7 +124,12 @@ def _rng(seed: int, what: str, index: int = 0) -> np.random.Generator:
 def _normal(seed, what, index, shape, dtype):
     w = _rng(seed, what, index).standard_normal(size=shape, dtype=np.float32)
     w *= np.float32(WEIGHT_STD)
-    return bf16_round(w) if dtype == "bf16" else w
+    if dtype == "f32":
+        return w
+    w = bf16_round(w)                       # the configurations' weights are bf16 values
+    if dtype == "f16":                      # held in float16 containers: exact for |w| >= 2^-17
+        w = w.astype(np.float16).astype(np.float32)
+    return w
 
 
 def embedding(m: ModelCfg, seed: int) -> np.ndarray:

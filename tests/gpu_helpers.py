@@ -9,7 +9,7 @@ import testgen
 from oracle import akvs_oracle as orc
 from helpers import oracle_model, make_inputs
 
-TOL = {"f32": 2e-3, "bf16": 1e-2}          # max relative L2 error per tensor (the benchmark spec)
+TOL = {"f32": 2e-3, "bf16": 1e-2, "f16": 1e-2}          # max relative L2 error per tensor (the benchmark spec)
 
 
 def t2n(t):
@@ -50,12 +50,20 @@ class Case:
         return orc.encode_units(self.omodel, self.units_ids, kv_bits=bits)
 
     def load_oracle_cache(self, units):
-        """Overwrites the GPU store with the oracle's cache (values, or codes + meta)."""
+        """Gives both sides the same cache: the oracle's values in the store's format.  A
+        16-bit store rounds them; the rounded values are written back into `units` so that
+        the oracle reads exactly what the library reads (the cache is an input of the prefill)."""
         k = np.concatenate([u["K"] for u in units], axis=1)
         v = np.concatenate([u["V"] for u in units], axis=1)
         if self.kv_format == 0:
             self.store.k.copy_(torch.from_numpy(k).to(self.store.k.dtype))
             self.store.v.copy_(torch.from_numpy(v).to(self.store.v.dtype))
+            ks, vs = t2n(self.store.k), t2n(self.store.v)
+            o = 0
+            for u in units:
+                n = u["K"].shape[1]
+                u["K"], u["V"] = ks[:, o:o + n], vs[:, o:o + n]
+                o += n
         else:
             for name, dst, dmeta in (("K", self.store.k, self.store.k_meta), ("V", self.store.v, self.store.v_meta)):
                 codes = np.concatenate([u[name + "_codes"] for u in units], axis=1)

@@ -23,20 +23,26 @@ def n64(t):
     return t.detach().float().cpu().numpy().astype(np.float64)
 
 
+EPS = {torch.float32: 2.0 ** -23, torch.bfloat16: 2.0 ** -8, torch.float16: 2.0 ** -11}   # one rounding
+H16 = [torch.bfloat16, torch.float16]
+
+
 # ----------------------------------------------------------------------------- linear layers
 
 @pytest.mark.parametrize("M,N,K", [(1, 128, 64), (77, 256, 200), (128, 128, 64), (130, 384, 1024), (1357, 1024, 4096),
                                    (300, 11008, 2048)])
 @pytest.mark.parametrize("algo", [0, 1])
-def test_linear_bf16(akvs, M, N, K, algo):
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float16])
+def test_linear_16bit(akvs, M, N, K, algo, dtype):
     g = np.random.default_rng(M * 7 + N)
-    x = dev(g.standard_normal((M, K)).astype(np.float32), torch.bfloat16)
-    w = dev((g.standard_normal((N, K)) * 0.05).astype(np.float32), torch.bfloat16)
+    x = dev(g.standard_normal((M, K)).astype(np.float32), dtype)
+    w = dev((g.standard_normal((N, K)) * 0.05).astype(np.float32), dtype)
     y = akvs.op_linear(x, w, algo)
     torch.cuda.synchronize()
     ref = n64(x) @ n64(w).T
-    assert orc.rel_l2(n64(y), ref) < 4e-3            # only the output rounding to bf16 (2^-9) remains
-    assert np.abs(n64(y) - ref).max() <= 2.0 ** -8 * np.abs(ref).max() + 1e-6
+    ulp = EPS[dtype]                                 # only the output rounding remains
+    assert orc.rel_l2(n64(y), ref) < 2 * ulp
+    assert np.abs(n64(y) - ref).max() <= ulp * np.abs(ref).max() + 1e-5
 
 
 @pytest.mark.parametrize("M,N,K", [(1, 1, 1), (65, 130, 33), (200, 688, 256)])
@@ -49,12 +55,13 @@ def test_linear_f32(akvs, M, N, K):
     assert orc.rel_l2(n64(y), n64(x) @ n64(w).T) < 1e-6
 
 
-def test_linear_bf16_full_size_sampled(akvs):
+@pytest.mark.parametrize("dtype", H16)
+def test_linear_16bit_full_size_sampled(akvs, dtype):
     """Config-3 MLP shape; the oracle checks sampled outputs one by one."""
     g = torch.Generator(device="cuda").manual_seed(5)
     M, N, K = 2586, 4096, 14336
-    x = torch.randn((M, K), generator=g, device="cuda").to(torch.bfloat16)
-    w = (torch.randn((N, K), generator=g, device="cuda") * 0.02).to(torch.bfloat16)
+    x = torch.randn((M, K), generator=g, device="cuda").to(dtype)
+    w = (torch.randn((N, K), generator=g, device="cuda") * 0.02).to(dtype)
     y = akvs.op_linear(x, w, 0)
     torch.cuda.synchronize()
     rs = np.random.default_rng(0)
@@ -63,12 +70,13 @@ def test_linear_bf16_full_size_sampled(akvs):
     xr, wc = n64(x[rows]), n64(w[cols])
     ref = xr @ wc.T
     got = n64(y[rows][:, cols])
-    assert np.abs(got - ref).max() <= 2.0 ** -8 * np.abs(ref).max() + 1e-6
+    assert np.abs(got - ref).max() <= EPS[dtype] * np.abs(ref).max() + 1e-4
 
 
 # ----------------------------------------------------------------------------- RoPE
 
-@pytest.mark.parametrize("dtype,hd", [(torch.float32, 64), (torch.bfloat16, 128), (torch.float32, 128)])
+@pytest.mark.parametrize("dtype,hd", [(torch.float32, 64), (torch.float16, 128), (torch.bfloat16, 128),
+                                      (torch.float32, 128)])
 def test_rope(akvs, dtype, hd):
     g = np.random.default_rng(1)
     n, H = 37, 3
@@ -78,14 +86,14 @@ def test_rope(akvs, dtype, hd):
     ref = orc.rope_rotate(n64(xt), pos, 1e4)
     akvs.op_rope(xt, dev(pos), 1e4)
     torch.cuda.synchronize()
-    tol = 1e-6 if dtype == torch.float32 else 4e-3
-    assert orc.rel_l2(n64(xt), ref) < tol
+    assert orc.rel_l2(n64(xt), ref) < max(1e-6, EPS[dtype])
 
 
 # ----------------------------------------------------------------------------- attention
 
-@pytest.mark.parametrize("dtype,hd,nq,nkv", [(torch.float32, 64, 4, 2), (torch.bfloat16, 128, 8, 2),
-                                             (torch.bfloat16, 128, 5, 1), (torch.bfloat16, 64, 2, 2)])
+@pytest.mark.parametrize("dtype,hd,nq,nkv", [(torch.float32, 64, 4, 2), (torch.float16, 128, 8, 2),
+                                             (torch.bfloat16, 128, 4, 1), (torch.float16, 128, 5, 1),
+                                             (torch.bfloat16, 64, 2, 2)])
 def test_attention_sparse_rows_and_block_diagonal(akvs, dtype, hd, nq, nkv):
     g = np.random.default_rng(2)
     T = 300
@@ -94,7 +102,7 @@ def test_attention_sparse_rows_and_block_diagonal(akvs, dtype, hd, nq, nkv):
     rows = np.sort(g.choice(T, 45, replace=False)).astype(np.int32)
     rows[0] = 0
     q = dev(g.standard_normal((len(rows), nq, hd)).astype(np.float32), dtype)
-    tol = 1e-5 if dtype == torch.float32 else 6e-3
+    tol = max(1e-5, 2 * EPS[dtype])
     out = akvs.op_attention(q, k, v, dev(np.zeros_like(rows)), dev(rows))
     torch.cuda.synchronize()
     ref = orc.attention(n64(q), n64(k), n64(v), rows, np.arange(T))
@@ -152,7 +160,7 @@ def test_select_nan_is_reported(akvs):
 # ----------------------------------------------------------------------------- quantiser (bit-exact)
 
 @pytest.mark.parametrize("bits", [2, 4])
-@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("dtype", [torch.float32, torch.float16, torch.bfloat16])
 def test_quantize_bit_exact(akvs, bits, dtype):
     g = np.random.default_rng(bits)
     x = g.standard_normal((203, 2, 128)).astype(np.float32) * 3
@@ -191,7 +199,7 @@ def _correct_case(akvs, dtype_t, kv_format, N_units, len_lo, len_hi, nkv, hd, nq
     R = probes.n_rows
     fk = g.standard_normal((R, nkv, hd)).astype(np.float32)
     fv = g.standard_normal((R, nkv, hd)).astype(np.float32)
-    dt = akvs.F32 if dtype_t == torch.float32 else akvs.BF16
+    dt = {torch.float32: akvs.F32, torch.bfloat16: akvs.BF16, torch.float16: akvs.F16}[dtype_t]
     fk_t, fv_t = dev(fk, dtype_t), dev(fv, dtype_t)
     if kv_format == 0:
         ck_t, cv_t = dev(ck, dtype_t), dev(cv, dtype_t)
@@ -225,7 +233,7 @@ def _correct_case(akvs, dtype_t, kv_format, N_units, len_lo, len_hi, nkv, hd, nq
     rmu_v = orc.probe_offsets(v_f, cv_ref, ref_p["sv_idx"], ref_p["probe_off"])
     rk = np.concatenate([orc.apply_correction(k_f, kr, ref_p["sk_idx"], ref_p["w_k"], rmu_k, off), n64(fk_t)[P:]])
     rv = np.concatenate([orc.apply_correction(v_f, cv_ref, ref_p["sv_idx"], ref_p["w_v"], rmu_v, off), n64(fv_t)[P:]])
-    tol = 2e-6 if dtype_t == torch.float32 else 3e-3
+    tol = max(2e-6, EPS[dtype_t])
     assert orc.rel_l2(n64(mu_k).reshape(rmu_k.shape), rmu_k) < 2e-6 * (1 if dtype_t == torch.float32 else 10)
     assert orc.rel_l2(n64(mu_v).reshape(rmu_v.shape), rmu_v) < 2e-6 * (1 if dtype_t == torch.float32 else 10)
     assert orc.rel_l2(n64(out_k), rk) < tol and orc.rel_l2(n64(out_v), rv) < tol
@@ -236,8 +244,9 @@ def _correct_case(akvs, dtype_t, kv_format, N_units, len_lo, len_hi, nkv, hd, nq
     return N
 
 
-@pytest.mark.parametrize("dtype_t,kv_format,hd", [(torch.float32, 0, 64), (torch.bfloat16, 0, 128),
-                                                  (torch.bfloat16, 4, 128), (torch.bfloat16, 2, 128),
+@pytest.mark.parametrize("dtype_t,kv_format,hd", [(torch.float32, 0, 64), (torch.float16, 0, 128),
+                                                  (torch.bfloat16, 0, 128), (torch.bfloat16, 4, 64),
+                                                  (torch.float16, 4, 128), (torch.float16, 2, 128),
                                                   (torch.float32, 4, 64), (torch.float32, 2, 128)])
 def test_correct_layer_small_ragged(akvs, dtype_t, kv_format, hd):
     _correct_case(akvs, dtype_t, kv_format, 5, 3, 41, 2, hd, 7, 2500)
@@ -249,7 +258,7 @@ def test_correct_layer_small_ragged(akvs, dtype_t, kv_format, hd):
 def test_correct_layer_full_size(akvs, kv_format):
     """One layer at the 8B-class shapes (8 kv heads x 128, ~8k / ~12k context tokens)."""
     if kv_format == 0:
-        N = _correct_case(akvs, torch.bfloat16, 0, 32, 128, 384, 8, 128, 128, 1500, seed=3)
+        N = _correct_case(akvs, torch.float16, 0, 32, 128, 384, 8, 128, 128, 1500, seed=3)
     else:
-        N = _correct_case(akvs, torch.bfloat16, kv_format, 48, 256, 256, 8, 128, 128, 2000, seed=4)
+        N = _correct_case(akvs, torch.float16, kv_format, 48, 256, 256, 8, 128, 128, 2000, seed=4)
     assert N > 6000
