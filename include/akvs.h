@@ -46,6 +46,7 @@ extern "C" {
 #define AKVS_ERR_CUDA        (-5)  /* a CUDA runtime or driver call failed                    */
 #define AKVS_ERR_TIMEOUT     (-6)  /* a bounded device-side wait ran out (no hang, no trap)  */
 #define AKVS_ERR_NAN_SCORE   (-7)  /* a divergence score was NaN                             */
+#define AKVS_ERR_TOO_LARGE   (-8)  /* request exceeds a fixed capacity of the entry point    */
 
 #define AKVS_F32   0
 #define AKVS_BF16  1
@@ -211,6 +212,32 @@ int64_t akvs_op_scratch_bytes(int32_t n_ctx, int32_t n_query, int32_t n_units, i
  * scratch: device, 256-byte aligned, akvs_op_scratch_bytes(...) bytes.  Synchronises the stream. */
 int32_t akvs_op_select(const float* d_k, const float* d_v, const int32_t* ctx_off_host, int32_t n_units,
                        int32_t n_query, int32_t refresh_bp, akvs_probes* out, void* scratch, void* stream);
+
+/* akvs_op_select for callers that cannot allocate device memory.  (The paper has no
+ * counterpart to this entry point; it exists for deployment reasons only.)
+ *
+ * Who needs it: code that runs where cudaMalloc is not an option -- a serving loop whose
+ * device memory pool is carved up at start-up, a process whose remaining memory belongs to
+ * another allocator, a request path on which allocation is forbidden -- and that therefore
+ * has no scratch buffer to hand to akvs_op_select.  Here the scratch (sort keys, selection
+ * flags, counters; about 0.3 MB) is a fixed array inside the library's device image, held
+ * on every GPU that loads the library until the process exits.  The call itself allocates
+ * nothing on the device or on the host heap.
+ *
+ * Same arguments, outputs and bit-exact results as akvs_op_select, minus `scratch`.
+ * Limits: ctx_off_host[n_units] <= AKVS_STATIC_MAX_CTX context tokens and
+ * n_units <= AKVS_STATIC_MAX_UNITS; beyond either the call returns AKVS_ERR_TOO_LARGE and
+ * launches nothing.
+ * First call per device: it resolves the device address of the array (with that device
+ * current); make that first call outside any stream capture.
+ * Sharing: every call on a device uses the one array, which keeps the previous call's
+ * contents; the call clears what has to start at zero itself.  Two calls that overlap on the
+ * GPU (different streams, different host threads) race on it: run them one after another.
+ * Synchronises `stream` once, like akvs_op_select. */
+#define AKVS_STATIC_MAX_CTX   16384
+#define AKVS_STATIC_MAX_UNITS 1024
+int32_t akvs_op_select_static(const float* d_k, const float* d_v, const int32_t* ctx_off_host, int32_t n_units,
+                              int32_t n_query, int32_t refresh_bp, akvs_probes* out, void* stream);
 
 /* One layer of Algorithm 1 lines 5-8 (mean estimation + correction) over a whole context.
  * fresh_k/fresh_v [n_rows][n_kv][hd] hold the recomputed rows listed in probes->rows (K

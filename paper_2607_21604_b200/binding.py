@@ -16,7 +16,8 @@ LIB_PATH = os.path.join(_HERE, "libakvs.so")
 
 OK = 0
 ERR = {0: "AKVS_OK", -1: "AKVS_ERR_INVALID_ARG", -2: "AKVS_ERR_SHAPE", -3: "AKVS_ERR_WORKSPACE",
-       -4: "AKVS_ERR_UNSUPPORTED", -5: "AKVS_ERR_CUDA", -6: "AKVS_ERR_TIMEOUT", -7: "AKVS_ERR_NAN_SCORE"}
+       -4: "AKVS_ERR_UNSUPPORTED", -5: "AKVS_ERR_CUDA", -6: "AKVS_ERR_TIMEOUT", -7: "AKVS_ERR_NAN_SCORE",
+       -8: "AKVS_ERR_TOO_LARGE"}
 F32, BF16, F16 = 0, 1, 2
 KV_NATIVE, KV_Q2, KV_Q4 = 0, 2, 4
 MODE_CORRECTED, MODE_NAIVE, MODE_FULL = 0, 1, 2
@@ -24,7 +25,9 @@ MODE_CORRECTED, MODE_NAIVE, MODE_FULL = 0, 1, 2
 EXPORTS = ["akvs_workspace_bytes", "akvs_debug_set_linear_algo", "akvs_launch_count", "akvs_prof_enable",
            "akvs_prof_reset", "akvs_prof_read", "akvs_encode_units", "akvs_select_probes", "akvs_prefill_corrected",
            "akvs_free", "akvs_check", "akvs_op_linear", "akvs_op_rope", "akvs_op_attention",
-           "akvs_op_scratch_bytes", "akvs_op_select", "akvs_op_correct_layer", "akvs_op_quantize"]
+           "akvs_op_scratch_bytes", "akvs_op_select", "akvs_op_select_static", "akvs_op_correct_layer",
+           "akvs_op_quantize"]
+STATIC_MAX_CTX, STATIC_MAX_UNITS = 16384, 1024
 
 
 class AkvsError(RuntimeError):
@@ -311,6 +314,20 @@ def op_select(d_k, d_v, ctx_off, n_query, refresh_bp):
     scratch = op_scratch(N, n_query, M, 128, d_k.device)
     _chk(lib.akvs_op_select(_ptr(d_k), _ptr(d_v), off, M, n_query, refresh_bp, C.byref(probes.desc), _ptr(scratch),
                             _stream()), "akvs_op_select")
+    return probes
+
+
+def op_select_static(d_k, d_v, ctx_off, n_query, refresh_bp, probes=None):
+    """Selection without a scratch buffer, for callers that must not allocate device memory:
+    the library's built-in array is used (limits STATIC_MAX_CTX / STATIC_MAX_UNITS).  Pass
+    `probes` to reuse output arrays; this wrapper only allocates them when none are given."""
+    M = len(ctx_off) - 1
+    N = int(ctx_off[-1])
+    if probes is None:
+        probes = Probes(N, M, n_query, d_k.device)
+    off = (C.c_int32 * (M + 1))(*[int(x) for x in ctx_off])
+    _chk(lib.akvs_op_select_static(_ptr(d_k), _ptr(d_v), off, M, n_query, refresh_bp, C.byref(probes.desc),
+                                   _stream()), "akvs_op_select_static")
     return probes
 
 
