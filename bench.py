@@ -214,7 +214,7 @@ def main():
         return ms / steps
 
     # ---------------------------------------------------------------- device-resident timing
-    akvs.prof_enable(1, 4096)
+    akvs.prof_enable((1 << 1) | (1 << 2) | (1 << 3), 8192)
     for _ in range(args.warmup):
         step()
     barrier()
@@ -231,17 +231,35 @@ def main():
     P = probes.n_probe_rows
 
     pk = peaks()
-    g_ms = sum(r[0] for r in recs)
-    g_fl = sum(r[1] for r in recs)
+    gemm = [r for r in recs if r[2] >> 8 == 1]
+    corr = [r for r in recs if r[2] >> 8 == 2]
+    attn = [r for r in recs if r[2] >> 8 == 3]
+    g_ms = sum(r[0] for r in gemm)
+    g_fl = sum(r[1] for r in gemm)
     by_epi = {}
-    for ms_, fl, sub in recs:
-        a = by_epi.setdefault(sub, [0.0, 0.0, 0])
+    for ms_, fl, sub in gemm:
+        a = by_epi.setdefault(sub & 255, [0.0, 0.0, 0])
         a[0] += ms_; a[1] += fl; a[2] += 1
+    # attention flops of one step from the recomputed rows: 4 * dq * sum_r (keys visible to r);
+    # the dense first layer sees every row, the selective layers the probe and query rows
+    rows = probes.rows[:probes.n_rows].cpu().numpy().astype(np.float64)
+    a_fl = 4.0 * m.dq * ((CHECK_LAYER - 1) * (T * (T + 1) / 2.0) + (m.n_layers - CHECK_LAYER + 1) * float((rows + 1).sum()))
+    a_ms = sum(r[0] for r in attn) / args.steps
+    c_ms = sum(r[0] for r in corr)
+    c_by = sum(r[1] for r in corr)
     achieved = g_fl / (g_ms * 1e-3) / 1e12 if g_ms > 0 else 0.0
+    other = {
+        "attention_tc_kernel": {"bound": "tensor", "tflops": a_fl / (a_ms * 1e-3) / 1e12 if a_ms > 0 else None,
+                                "frac": a_fl / (a_ms * 1e-3) / 1e12 / pk["tensor"] if a_ms > 0 else None,
+                                "ms_per_step": a_ms, "launches_per_step": len(attn) / args.steps},
+        "correct_kernel": {"bound": "hbm", "gbs": c_by / (c_ms * 1e-3) / 1e9 if c_ms > 0 else None,
+                           "frac": c_by / (c_ms * 1e-3) / 1e9 / pk["hbm"] if c_ms > 0 else None,
+                           "ms_per_step": c_ms / args.steps, "launches_per_step": len(corr) / args.steps,
+                           "bytes_per_launch": c_by / max(1, len(corr))}}
     roofline = {"bound": "tensor", "kernel": "gemm_tc_kernel (all linear layers of the step)",
                 "achieved": achieved, "peak": pk["tensor"], "unit": "TFLOP/s", "frac": achieved / pk["tensor"],
                 "peak_source": pk["src"] + " bf16 cuBLAS sustained (f16 and bf16 MMAs run at the same rate)",
-                "traffic": None, "launches": len(recs), "share_of_step": g_ms / (ms_step * args.steps),
+                "traffic": None, "launches": len(gemm), "share_of_step": g_ms / (ms_step * args.steps),
                 "by_epilogue": {{0: "qkv_store", 1: "residual", 2: "swiglu"}.get(k, str(k)):
                                 {"tflops": v[1] / (v[0] * 1e-3) / 1e12, "ms_per_step": v[0] / args.steps,
                                  "launches": v[2]} for k, v in sorted(by_epi.items())}}
@@ -302,6 +320,7 @@ def main():
                 "what": "unit cache + ids from pinned host memory each step, query hidden state back"},
         "gpu_launches": int(launches),
         "roofline": roofline,
+        "other_kernels": other,
         "cpu_baseline": cpu,
         "context": {"full_recompute_ms": full_ms, "speedup_vs_full_recompute": full_ms / ms_step,
                     "encode_units_ms": encode_ms, "setup_s": setup_s,

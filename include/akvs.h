@@ -167,20 +167,23 @@ void akvs_free(void* ctx);
  * (AKVS_OK, AKVS_ERR_TIMEOUT, AKVS_ERR_NAN_SCORE), then clears it. */
 int32_t akvs_check(void* workspace, void* stream);
 
-/* Cross-check switch for the tests: 0 (default) routes 16-bit linear layers to the tcgen05
- * kernels, 1 to the CUDA-core kernels.  Process-wide; not part of the serving surface. */
+/* Cross-check switch for the tests: bit 0 set routes the 16-bit linear layers, bit 1 set the
+ * 16-bit attention, to the CUDA-core kernels instead of the tcgen05 ones (default 0: tensor
+ * cores for both).  Process-wide; not part of the serving surface. */
 int32_t akvs_debug_set_linear_algo(int32_t algo);
 
 /* Number of kernels this library has launched in this process so far. */
 int64_t akvs_launch_count(void);
 
-/* Per-launch device timing of one kernel class with CUDA events recorded on the launching
- * stream: kind 1 = tensor-core linear layers (sub = epilogue: 0 store, 1 residual, 2 SwiGLU;
- * work = flops), kind 2 = correction pass (sub = kv format; work = algorithmic bytes),
- * kind 0 = off.  akvs_prof_enable allocates max_records event pairs (host objects only);
- * akvs_prof_read waits for the recorded events and returns elapsed ms, work and sub per
- * launch; akvs_prof_reset forgets the records but keeps the events.  Not thread-safe. */
-int32_t akvs_prof_enable(int32_t kind, int32_t max_records);
+/* Per-launch device timing of kernel classes with CUDA events recorded on the launching
+ * stream.  kind_mask has bit k set for class k: 1 = tensor-core linear layers (sub =
+ * epilogue: 0 store, 1 residual, 2 SwiGLU; work = flops), 2 = correction pass (sub = kv
+ * format; work = algorithmic bytes), 3 = tensor-core attention (work not filled in);
+ * 0 = off.  akvs_prof_enable allocates max_records event pairs (host objects only);
+ * akvs_prof_read waits for the recorded events and returns per launch the elapsed ms, the
+ * work and (class << 8 | sub); akvs_prof_reset forgets the records but keeps the events.
+ * Not thread-safe. */
+int32_t akvs_prof_enable(int32_t kind_mask, int32_t max_records);
 int32_t akvs_prof_reset(void);
 int32_t akvs_prof_read(int32_t capacity, float* ms, double* work, int32_t* sub, int32_t* n_out);
 
@@ -199,7 +202,9 @@ int32_t akvs_op_rope(int32_t dtype, void* x, const int32_t* pos, int32_t n, int3
                      int32_t head_dim, float rope_base, void* stream);
 
 /* GQA attention: query row r sees key j iff k_lo[r] <= j <= k_hi[r] (device arrays, both
- * non-decreasing in r).  q [R][n_q][hd], k/v [T][n_kv][hd], out [R][n_q][hd]. */
+ * non-decreasing in r).  q [R][n_q][hd], k/v [T][n_kv][hd], out [R][n_q][hd].
+ * algo 0: the path's default (tcgen05 for 16-bit types with head_dim 128, else CUDA cores);
+ * algo 1: CUDA cores. */
 int32_t akvs_op_attention(int32_t dtype, const void* q, const void* k, const void* v, void* out,
                           const int32_t* k_lo, const int32_t* k_hi, int32_t R, int32_t T,
                           int32_t n_q_heads, int32_t n_kv_heads, int32_t head_dim, int32_t algo, void* stream);

@@ -18,10 +18,10 @@ size_t g_prof_used = 0;
 }  // namespace
 
 void akvs_prof_mark(int kind, int sub, double work, bool begin, cudaStream_t st) {
-  if (kind != g_prof_kind || g_prof_used >= g_prof.size()) return;
+  if (!((g_prof_kind >> kind) & 1) || g_prof_used >= g_prof.size()) return;
   ProfRec& r = g_prof[g_prof_used];
   if (begin) {
-    r.sub = sub;
+    r.sub = (kind << 8) | sub;
     r.work = work;
     cudaEventRecord(r.a, st);
   } else {
@@ -186,9 +186,18 @@ int32_t linear_swiglu(const Dims& D, const void* x, int M, int K, const void* wg
 // (rotated at `pos`) and V; `between` runs after RoPE and before attention (store to the
 // cache, or estimate offsets and assemble the corrected K/V); attention then reads
 // attn_k/attn_v with per-row key ranges [lo, hi].
+int g_attention_algo = 0;       // 16-bit models with head_dim 128: 0 = tcgen05; 1 = CUDA cores
+
+int32_t attention(const Dims& D, const void* q, const void* k, const void* v, void* out, const int32_t* lo,
+                  const int32_t* hi, int n, int n_keys, int32_t* status, cudaStream_t st) {
+  if (D.dtype != AKVS_F32 && D.hd == 128 && g_attention_algo == 0)
+    return launch_attention_tc(D.dtype, q, k, v, out, lo, hi, n, n_keys, D.nq, D.nkv, status, st);
+  return launch_attention_simt(D.dtype, q, k, v, out, lo, hi, n, D.nq, D.nkv, D.hd, st);
+}
+
 int32_t run_layer(const akvs_model_desc* m, const Dims& D, int l, const Workspace& ws, int n, const int32_t* pos,
                   const int32_t* lo, const int32_t* hi, void* k_dst, void* v_dst, const void* attn_k,
-                  const void* attn_v, const std::function<int32_t()>& between, cudaStream_t st) {
+                  const void* attn_v, int n_keys, const std::function<int32_t()>& between, cudaStream_t st) {
   if (n == 0) return between ? between() : AKVS_OK;
   AKVS_TRY(launch_rmsnorm(D.dtype, ws.h, m->attn_norm[l], m->rms_eps, n, D.d, ws.x, st));
   {
@@ -200,7 +209,7 @@ int32_t run_layer(const akvs_model_desc* m, const Dims& D, int l, const Workspac
   AKVS_TRY(launch_rope(D.dtype, ws.q, pos, n, D.nq, D.hd, D.dq, ws.rope, m->rope_base, st));
   AKVS_TRY(launch_rope(D.dtype, k_dst, pos, n, D.nkv, D.hd, D.dkv, ws.rope, m->rope_base, st));
   if (between) AKVS_TRY(between());
-  AKVS_TRY(launch_attention_simt(D.dtype, ws.q, attn_k, attn_v, ws.ao, lo, hi, n, D.nq, D.nkv, D.hd, st));
+  AKVS_TRY(attention(D, ws.q, attn_k, attn_v, ws.ao, lo, hi, n, n_keys, ws.status, st));
   AKVS_TRY(linear_resid(D, ws.ao, n, D.dq, m->wo[l], D.d, ws.h, ws.status, st));
   AKVS_TRY(launch_rmsnorm(D.dtype, ws.h, m->mlp_norm[l], m->rms_eps, n, D.d, ws.x, st));
   AKVS_TRY(linear_swiglu(D, ws.x, n, D.d, m->w_gate[l], m->w_up[l], D.f, ws.act, ws.status, st));
@@ -307,7 +316,8 @@ int32_t embed_all(const akvs_model_desc* m, const Dims& D, const akvs_cache* c, 
 extern "C" {
 
 int32_t akvs_debug_set_linear_algo(int32_t algo) {
-  g_bf16_linear_algo = algo;
+  g_bf16_linear_algo = algo & 1;
+  g_attention_algo = (algo >> 1) & 1;
   return AKVS_OK;
 }
 
@@ -392,7 +402,7 @@ int32_t akvs_encode_units(const akvs_model_desc* model, akvs_cache* cache, void*
                                reinterpret_cast<char*>(cache->v) + l * lstride,
                                reinterpret_cast<char*>(cache->v_meta) + l * mstride, st);
       };
-    AKVS_TRY(run_layer(model, D, l, ws, N, local_pos, ws.lo, ws.pos, k_dst, v_dst, k_dst, v_dst, store, st));
+    AKVS_TRY(run_layer(model, D, l, ws, N, local_pos, ws.lo, ws.pos, k_dst, v_dst, k_dst, v_dst, N, store, st));
   }
   return AKVS_OK;
 }
@@ -435,7 +445,7 @@ int32_t akvs_select_probes(const akvs_model_desc* model, const akvs_cache* cache
   for (int l = 0; l < check_layer - 1; ++l) {
     void* kd = reinterpret_cast<char*>(ws.stash_k) + l * kv_l;
     void* vd = reinterpret_cast<char*>(ws.stash_v) + l * kv_l;
-    AKVS_TRY(run_layer(model, D, l, ws, T, ws.pos, ws.zeros, ws.pos, kd, vd, kd, vd, nullptr, st));
+    AKVS_TRY(run_layer(model, D, l, ws, T, ws.pos, ws.zeros, ws.pos, kd, vd, kd, vd, T, nullptr, st));
   }
   if (T > 0)
     AKVS_CUDA(cudaMemcpyAsync(ws.stash_h, ws.h, (size_t)T * D.d * sizeof(float), cudaMemcpyDeviceToDevice, st));
@@ -499,7 +509,7 @@ int32_t akvs_prefill_corrected(const akvs_model_desc* model, const akvs_cache* c
     AKVS_TRY(embed_all(model, D, cache, req, ws, N, st));
     for (int l = 0; l < D.L; ++l)
       AKVS_TRY(run_layer(model, D, l, ws, T, ws.pos, ws.zeros, ws.pos, ok + l * kv_l, ov + l * kv_l, ok + l * kv_l,
-                         ov + l * kv_l, nullptr, st));
+                         ov + l * kv_l, T, nullptr, st));
     return launch_rmsnorm(AKVS_F32, ws.h + (size_t)N * D.d, model->final_norm, model->rms_eps, nq, D.d, out_hidden, st);
   }
 
@@ -552,8 +562,8 @@ int32_t akvs_prefill_corrected(const akvs_model_desc* model, const akvs_cache* c
                             corrected ? probes->w_v : nullptr, ws.mu_k, ws.mu_v, N, nq, P, D.nkv, D.hd, ws.rope,
                             ok + l * kv_l, ov + l * kv_l, st);
     };
-    AKVS_TRY(run_layer(model, D, l, ws, R, rows, ws.zeros, rows, ws.k, ws.v, ok + l * kv_l, ov + l * kv_l, assemble,
-                       st));
+    AKVS_TRY(run_layer(model, D, l, ws, R, rows, ws.zeros, rows, ws.k, ws.v, ok + l * kv_l, ov + l * kv_l, T,
+                       assemble, st));
   }
   return launch_rmsnorm(AKVS_F32, ws.h + (size_t)P * D.d, model->final_norm, model->rms_eps, nq, D.d, out_hidden, st);
 }
@@ -604,9 +614,10 @@ int32_t akvs_op_attention(int32_t dtype, const void* q, const void* k, const voi
                           int32_t head_dim, int32_t algo, void* stream) {
   if (!q || !k || !v || !out || !k_lo || !k_hi || R < 0 || T < 0) return AKVS_ERR_INVALID_ARG;
   if (dtype != AKVS_F32 && dtype != AKVS_BF16 && dtype != AKVS_F16) return AKVS_ERR_UNSUPPORTED;
-  (void)algo;
-  return launch_attention_simt(dtype, q, k, v, out, k_lo, k_hi, R, n_q_heads, n_kv_heads, head_dim,
-                               reinterpret_cast<cudaStream_t>(stream));
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  if (dtype != AKVS_F32 && head_dim == 128 && algo == 0)
+    return launch_attention_tc(dtype, q, k, v, out, k_lo, k_hi, R, T, n_q_heads, n_kv_heads, nullptr, st);
+  return launch_attention_simt(dtype, q, k, v, out, k_lo, k_hi, R, n_q_heads, n_kv_heads, head_dim, st);
 }
 
 int64_t akvs_op_scratch_bytes(int32_t n_ctx, int32_t n_query, int32_t n_units, int32_t head_dim) {

@@ -208,6 +208,10 @@ int32_t launch_linear_simt(int dtype, const void* x, const void* w, const void* 
 int32_t launch_linear_tc(int dtype, int epi, const void* x, int M, int K, int n_seg, const void* const* w, const int* n,
                          void* const* out, const int* ldc, int32_t* status, cudaStream_t st);
 
+// tcgen05 attention (attn_tc.cu): 16-bit types, head_dim 128.
+int32_t launch_attention_tc(int dtype, const void* q, const void* k, const void* v, void* out, const int32_t* k_lo,
+                            const int32_t* k_hi, int R, int T, int n_q, int n_kv, int32_t* status, cudaStream_t st);
+
 int32_t launch_attention_simt(int dtype, const void* q, const void* k, const void* v, void* out,
                               const int32_t* k_lo, const int32_t* k_hi, int R, int n_q, int n_kv, int hd,
                               cudaStream_t st);
