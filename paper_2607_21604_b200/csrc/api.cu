@@ -83,6 +83,7 @@ struct Workspace {
   int32_t* tok_unit;        // [N]
   int32_t* tok_src;         // [N]
   int32_t* row_of_pos;      // [T]
+  int4* tok_meta;           // [T]
   uint8_t* flags;           // [2N]: kflag, vflag
   uint64_t* keys;           // [2N]
   int32_t* pos;             // [T] 0..T-1 (or unit-local positions while encoding)
@@ -115,6 +116,7 @@ Workspace carve(const Dims& D, int N, int nq, int M, int check_layer, void* base
   w.tok_unit = c.take<int32_t>(N);
   w.tok_src = c.take<int32_t>(N);
   w.row_of_pos = c.take<int32_t>(T);
+  w.tok_meta = c.take<int4>(T);
   w.flags = c.take<uint8_t>(2 * (int64_t)N);
   w.keys = c.take<uint64_t>(2 * (int64_t)N);
   w.pos = c.take<int32_t>(T);
@@ -299,6 +301,7 @@ ReqMaps req_maps(const Workspace& ws, int N) {
   mp.row_of_pos = ws.row_of_pos;
   mp.kflag = ws.flags;
   mp.vflag = ws.flags + N;
+  mp.tok_meta = ws.tok_meta;
   return mp;
 }
 
@@ -523,6 +526,7 @@ int32_t akvs_prefill_corrected(const akvs_model_desc* model, const akvs_cache* c
     AKVS_TRY(launch_rope_table(model->rope_base, D.hd, T, ws.rope, st));
     rows = ws.pos + N;                                   // the query positions N..T-1
     AKVS_TRY(launch_row_maps(rows, nq, nullptr, nullptr, 0, N, T, ws.row_of_pos, ws.flags, ws.flags + N, st));
+    AKVS_TRY(launch_tok_meta(ws.tok_unit, ws.tok_src, ws.row_of_pos, ws.flags, ws.flags + N, N, T, 0, ws.tok_meta, st));
     AKVS_TRY(launch_embed(D.dtype, model->tok_emb, req->query_ids, nullptr, nq, D.d, ws.h, st));
   } else {
     const Ctx* ctx = reinterpret_cast<const Ctx*>(ctx_v);
@@ -541,6 +545,7 @@ int32_t akvs_prefill_corrected(const akvs_model_desc* model, const akvs_cache* c
     rows = probes->rows;
     AKVS_TRY(launch_row_maps(rows, R, probes->sk_idx, probes->sv_idx, ctx->n_probe_total, N, T, ws.row_of_pos,
                              ws.flags, ws.flags + N, st));
+    AKVS_TRY(launch_tok_meta(ws.tok_unit, ws.tok_src, ws.row_of_pos, ws.flags, ws.flags + N, N, T, P, ws.tok_meta, st));
     for (int l = 0; l < first_layer; ++l) {
       AKVS_CUDA(cudaMemcpyAsync(ok + l * kv_l, reinterpret_cast<char*>(ws.stash_k) + l * kv_l, kv_l,
                                 cudaMemcpyDeviceToDevice, st));
@@ -622,7 +627,7 @@ int32_t akvs_op_attention(int32_t dtype, const void* q, const void* k, const voi
 
 int64_t akvs_op_scratch_bytes(int32_t n_ctx, int32_t n_query, int32_t n_units, int32_t head_dim) {
   const int64_t T = (int64_t)n_ctx + n_query;
-  return 4096 + 256 * 12 + T * (4 + head_dim * 4) + (int64_t)n_ctx * (4 + 2 + 16) + (int64_t)(n_units + 1) * 8;
+  return 4096 + 256 * 12 + T * (4 + 16 + head_dim * 4) + (int64_t)n_ctx * (4 + 2 + 16) + (int64_t)(n_units + 1) * 8;
 }
 
 int32_t akvs_op_select(const float* d_k, const float* d_v, const int32_t* ctx_off_host, int32_t n_units,
@@ -682,6 +687,7 @@ int32_t akvs_op_correct_layer(int32_t dtype, int32_t kv_format, const void* cach
   int32_t* zero_src = c.take<int32_t>(M + 1);
   int32_t* dummy_src = c.take<int32_t>(N);
   float2* table = c.take<float2>((int64_t)T * (head_dim / 2));
+  int4* tok_meta = c.take<int4>(T);
   (void)poff_host_dev;
   // the number of probe indices is probe_off[M]; read it back (this helper may synchronise)
   int32_t n_probe = 0;
@@ -693,8 +699,9 @@ int32_t akvs_op_correct_layer(int32_t dtype, int32_t kv_format, const void* cach
   AKVS_TRY(launch_row_maps(probes->rows, probes->n_rows, probes->sk_idx, probes->sv_idx, n_probe, N, T, row_of_pos,
                            flags, flags + N, st));
   AKVS_TRY(launch_rope_table(rope_base, head_dim, T, table, st));
+  AKVS_TRY(launch_tok_meta(tok_unit, src_tok, row_of_pos, flags, flags + N, N, T, probes->n_probe_rows, tok_meta, st));
   KvLayer kv{cache_k, cache_v, k_meta, v_meta, kv_format};
-  ReqMaps maps{probes->ctx_off, tok_unit, src_tok, row_of_pos, flags, flags + N};
+  ReqMaps maps{probes->ctx_off, tok_unit, src_tok, row_of_pos, flags, flags + N, tok_meta};
   AKVS_TRY(launch_offsets(dtype, kv, maps, probes->probe_off, probes->sk_idx, probes->sv_idx, fresh_k, fresh_v, M,
                           n_kv_heads, head_dim, table, mu_k, mu_v, st));
   return launch_correct(dtype, kv, maps, fresh_k, fresh_v, probes->w_k, probes->w_v, mu_k, mu_v, N, n_query,

@@ -14,7 +14,7 @@
 // by TMA (two stages each), warp 1 issues the MMAs, warps 2-5 do the softmax (a whole S row
 // is pulled into registers with one wait), warps 6-9 fold the P V products into the output
 // rows they keep in registers; the per-tile rescale factors travel through shared memory.
-// Row blocks are taken longest first (the last rows see the most keys).
+// Row blocks are taken longest first across all kv heads (the last rows see the most keys).
 // Query row r sees keys k_lo[r] <= j <= k_hi[r]; both arrays are non-decreasing in r.
 #include "tc_common.cuh"
 
@@ -32,7 +32,7 @@ constexpr int ATT_SMEM = OFF_CORR + 5 * 128 * 4;   // 232192 of the 232448 bytes
                                                    // re-aligning, the buffer itself is declared 1024-byte aligned
 
 struct AttnParams {
-  int R, T, n_q, n_kv, g, BR;
+  int R, T, n_q, n_kv, g, BR, row_blocks;
   const int32_t* k_lo;
   const int32_t* k_hi;
   void* out;
@@ -64,8 +64,10 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int hk = blockIdx.y;
-  const int r0 = (gridDim.x - 1 - blockIdx.x) * p.BR;       // longest row blocks first
+  // 1-D grid, kv head fastest: CTAs are handed out longest row block first across ALL heads
+  // (the last rows see the most keys), so the tail of the launch is made of short CTAs
+  const int hk = blockIdx.x % p.n_kv;
+  const int r0 = (p.row_blocks - 1 - blockIdx.x / p.n_kv) * p.BR;
   const int n_rows = min(p.BR, p.R - r0);
   const int key_lo = p.k_lo[r0];
   const int key_hi = p.k_hi[r0 + n_rows - 1];
@@ -313,7 +315,8 @@ int32_t launch_attention_tc(int dtype, const void* q, const void* k, const void*
   AKVS_TRY(encode_tmap_3d_16bit(&tmQ, q, HD, n_q, R, HD, (uint64_t)n_q * HD, p.g, p.BR));
   AKVS_TRY(encode_tmap_2d_16bit(&tmK, k, T, (uint64_t)n_kv * HD, (uint64_t)n_kv * HD, BN));
   AKVS_TRY(encode_tmap_2d_16bit(&tmV, v, T, (uint64_t)n_kv * HD, (uint64_t)n_kv * HD, BN));
-  const dim3 grid(akvs_cdiv(R, p.BR), n_kv);
+  p.row_blocks = akvs_cdiv(R, p.BR);
+  const dim3 grid((unsigned)p.row_blocks * n_kv);
   double flops = 0;   // filled by the caller's accounting when profiling attention
   ProfScope prof(3, 0, flops, st);
   if (dtype == AKVS_BF16) attention_tc_kernel<bf16><<<grid, ATT_THREADS, ATT_SMEM, st>>>(tmQ, tmK, tmV, p);

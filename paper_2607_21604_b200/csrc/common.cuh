@@ -186,6 +186,7 @@ struct ReqMaps {            // per-request index maps (device)
   const int32_t* row_of_pos;// [T] index into the recomputed rows, or -1
   const uint8_t* kflag;     // [N] 1 if j in S^K
   const uint8_t* vflag;     // [N]
+  const int4* tok_meta;     // [T] (store row, fresh K row or -1, fresh V row or -1, unit slot)
 };
 
 int32_t launch_embed(int dtype, const void* tok_emb, const int32_t* ids, const int32_t* gather, int n, int d,
@@ -220,6 +221,9 @@ int32_t launch_tok_maps(const int32_t* ctx_off, const int32_t* slot_src_off, int
                         int32_t* tok_src, cudaStream_t st);
 int32_t launch_row_maps(const int32_t* rows, int n_rows, const int32_t* sk_idx, const int32_t* sv_idx, int n_probe,
                         int N, int T, int32_t* row_of_pos, uint8_t* kflag, uint8_t* vflag, cudaStream_t st);
+int32_t launch_tok_meta(const int32_t* tok_unit, const int32_t* tok_src, const int32_t* row_of_pos,
+                        const uint8_t* kflag, const uint8_t* vflag, int N, int T, int n_probe_rows, int4* tok_meta,
+                        cudaStream_t st);
 int32_t launch_scores(int dtype, const KvLayer& kv, const ReqMaps& maps, const void* k_fresh, const void* v_fresh,
                       int N, int n_kv, int hd, const float2* table, float* d_k, float* d_v, cudaStream_t st);
 int32_t launch_select(const float* d_k, const float* d_v, const int32_t* ctx_off, const int32_t* probe_off, int M,

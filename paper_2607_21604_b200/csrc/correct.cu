@@ -81,6 +81,33 @@ __global__ void row_maps_fill_kernel(const int32_t* __restrict__ rows, int n_row
   }
 }
 
+// Per-token record of the correction pass: (store row, fresh row for K or -1, fresh row for V
+// or -1, unit slot).  Query tokens take both from the fresh rows that follow the probes.
+__global__ void tok_meta_kernel(const int32_t* __restrict__ tok_unit, const int32_t* __restrict__ tok_src,
+                                const int32_t* __restrict__ row_of_pos, const uint8_t* __restrict__ kflag,
+                                const uint8_t* __restrict__ vflag, int N, int T, int n_probe_rows,
+                                int4* __restrict__ tok_meta) {
+  const int j = blockIdx.x * blockDim.x + threadIdx.x;
+  if (j >= T) return;
+  if (j >= N) {
+    const int r = n_probe_rows + (j - N);
+    tok_meta[j] = make_int4(-1, r, r, 0);
+  } else {
+    const int r = row_of_pos[j];
+    tok_meta[j] = make_int4(tok_src[j], kflag[j] ? r : -1, vflag[j] ? r : -1, tok_unit[j]);
+  }
+}
+
+int32_t launch_tok_meta(const int32_t* tok_unit, const int32_t* tok_src, const int32_t* row_of_pos,
+                        const uint8_t* kflag, const uint8_t* vflag, int N, int T, int n_probe_rows, int4* tok_meta,
+                        cudaStream_t st) {
+  if (T == 0) return AKVS_OK;
+  tok_meta_kernel<<<akvs_cdiv(T, 256), 256, 0, st>>>(tok_unit, tok_src, row_of_pos, kflag, vflag, N, T, n_probe_rows,
+                                                    tok_meta);
+  AKVS_LAUNCHED();
+  return AKVS_OK;
+}
+
 int32_t launch_row_maps(const int32_t* rows, int n_rows, const int32_t* sk_idx, const int32_t* sv_idx, int n_probe,
                         int N, int T, int32_t* row_of_pos, uint8_t* kflag, uint8_t* vflag, cudaStream_t st) {
   if (T == 0) return AKVS_OK;
@@ -385,80 +412,182 @@ int32_t launch_offsets(int dtype, const KvLayer& kv, const ReqMaps& maps, const 
 //   context token j of unit u, not in S^K:  K_out = Rot(off_u) deq(K_cached) + w_K[j] mu_K[u]
 //                              in S^K:      K_out = fresh K of its recomputed row
 //   V likewise with S^V (no rotation);  query token i: fresh K/V of row P + i.
-// One thread per pair chunk; it moves 4 x 16 B in and 4 x 16 B out.
+// One thread owns one pair chunk (16 B of the lower half of a head + its RoPE partner in the
+// upper half) of COR_TOK consecutive tokens: it first issues all of their 16-byte loads
+// (4 per token: K lo/hi, V lo/hi), then decodes, rotates, corrects and stores.  The unit's
+// rotation row and offsets are fetched once per run of tokens of the same unit, so that the
+// L1 traffic per token is little more than the data itself.
 // ---------------------------------------------------------------------------------------
+constexpr int COR_TOK = 2;
+
+template <typename TW, int FMT> struct RawChunk;
+template <typename TW> struct RawChunk<TW, AKVS_KV_NATIVE> { uint4 v; };
+template <typename TW> struct RawChunk<TW, AKVS_KV_Q4> { uint32_t packed; __half2 sm; };
+template <typename TW> struct RawChunk<TW, AKVS_KV_Q2> { uint32_t packed; __half2 sm; };
+
+__device__ __forceinline__ void unpack16(const uint4& r, float (&o)[4], const float*) {
+  o[0] = __uint_as_float(r.x); o[1] = __uint_as_float(r.y); o[2] = __uint_as_float(r.z); o[3] = __uint_as_float(r.w);
+}
+__device__ __forceinline__ void unpack16(const uint4& r, float (&o)[8], const bf16*) {
+  const uint32_t w[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) { o[2 * i] = __uint_as_float(w[i] << 16); o[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u); }
+}
+__device__ __forceinline__ void unpack16(const uint4& r, float (&o)[8], const f16*) {
+  const uint32_t w[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&w[i]));
+    o[2 * i] = f.x; o[2 * i + 1] = f.y;
+  }
+}
+
+// Issues the load of one 16-byte-equivalent chunk: either from the fresh rows (T) or from
+// the cache in its own format.  A native cache of the same element type shares the register
+// with the fresh row (one pointer select, one load).
 template <typename T, typename TW, int FMT>
-__global__ void __launch_bounds__(256)
+__device__ __forceinline__ void issue_chunk(bool from_fresh, const T* fresh_p, const void* base, const void* meta,
+                                            int64_t src, int n_kv, int hd, int h, int dim0, uint4& fresh_raw,
+                                            RawChunk<TW, FMT>& raw) {
+  constexpr int V = VecOf<T>::N;
+  if constexpr (FMT == AKVS_KV_NATIVE && std::is_same<T, TW>::value) {
+    const T* cp = reinterpret_cast<const T*>(base) + ((size_t)(from_fresh ? 0 : src) * n_kv + h) * hd + dim0;
+    fresh_raw = *reinterpret_cast<const uint4*>(from_fresh ? fresh_p : cp);
+  } else if (from_fresh) {
+    fresh_raw = *reinterpret_cast<const uint4*>(fresh_p);
+  } else if constexpr (FMT == AKVS_KV_NATIVE) {
+    raw.v = *reinterpret_cast<const uint4*>(reinterpret_cast<const TW*>(base) + ((size_t)src * n_kv + h) * hd + dim0);
+  } else {
+    constexpr int BYTES = V * FMT / 8;
+    raw.packed = ld_codes<BYTES>(reinterpret_cast<const uint8_t*>(base) + (((size_t)src * n_kv + h) * hd + dim0) * FMT / 8);
+    raw.sm = reinterpret_cast<const __half2*>(meta)[((size_t)src * n_kv + h) * (hd / 64) + dim0 / 64];
+  }
+}
+template <typename T, typename TW, int FMT>
+__device__ __forceinline__ void decode_chunk(bool from_fresh, const uint4& fresh_raw, const RawChunk<TW, FMT>& raw,
+                                             float (&out)[VecOf<T>::N]) {
+  constexpr int V = VecOf<T>::N;
+  if constexpr (FMT == AKVS_KV_NATIVE && std::is_same<T, TW>::value) {
+    unpack16(fresh_raw, out, (const T*)nullptr);
+  } else if (from_fresh) {
+    unpack16(fresh_raw, out, (const T*)nullptr);
+  } else if constexpr (FMT == AKVS_KV_NATIVE) {
+    unpack16(raw.v, out, (const TW*)nullptr);
+  } else {
+    const float s = __low2float(raw.sm), mn = __high2float(raw.sm);
+#pragma unroll
+    for (int i = 0; i < V; ++i) out[i] = __fmaf_rn((float)((raw.packed >> (FMT * i)) & ((1u << FMT) - 1u)), s, mn);
+  }
+}
+
+// V consecutive floats / float2 as 16-byte loads (the addresses are 16-byte aligned by layout)
+template <int V>
+__device__ __forceinline__ void ld_f(const float* p, float (&o)[V]) {
+#pragma unroll
+  for (int i = 0; i < V; i += 4) {
+    const float4 t = *reinterpret_cast<const float4*>(p + i);
+    o[i] = t.x; o[i + 1] = t.y; o[i + 2] = t.z; o[i + 3] = t.w;
+  }
+}
+template <int V>
+__device__ __forceinline__ void ld_f2(const float2* p, float2 (&o)[V]) {
+#pragma unroll
+  for (int i = 0; i < V; i += 2) {
+    const float4 t = *reinterpret_cast<const float4*>(p + i);
+    o[i] = make_float2(t.x, t.y); o[i + 1] = make_float2(t.z, t.w);
+  }
+}
+
+template <typename T, typename TW, int FMT>
+__global__ void __launch_bounds__(256, 2)
 correct_kernel(KvLayer kv, ReqMaps maps, const T* __restrict__ k_fresh, const T* __restrict__ v_fresh,
                const float* __restrict__ w_k, const float* __restrict__ w_v, const float* __restrict__ mu_k,
                const float* __restrict__ mu_v, int N, int T_tok, int n_probe_rows, int n_kv, int hd,
                const float2* __restrict__ table, T* __restrict__ out_k, T* __restrict__ out_v) {
   constexpr int V = VecOf<T>::N;
   const int half = hd / 2, ch = half / V;
-  const int64_t total = (int64_t)T_tok * n_kv * ch;
-  for (int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
-       idx += (int64_t)gridDim.x * blockDim.x) {
-    const int c = (int)(idx % ch);
-    const int h = (int)((idx / ch) % n_kv);
-    const int j = (int)(idx / ((int64_t)ch * n_kv));
-    const size_t o = ((size_t)j * n_kv + h) * hd + c * V;
-    float lo[V], hi[V];
-    int row_k = -1, row_v = -1, u = 0;
-    int64_t src = 0;
-    float wk = 0.f, wv = 0.f;
-    if (j >= N) {
-      row_k = row_v = n_probe_rows + (j - N);
-    } else {
-      const int row = maps.row_of_pos[j];
-      if (maps.kflag[j]) row_k = row;
-      if (maps.vflag[j]) row_v = row;
-      u = maps.tok_unit[j];
-      src = maps.tok_src[j];
-      if (w_k) { wk = w_k[j]; wv = w_v[j]; }
-    }
-    // ---- K
-    if (row_k >= 0) {
-      const T* fp = k_fresh + ((size_t)row_k * n_kv + h) * hd + c * V;
-      ld16(fp, lo);
-      ld16(fp + half, hi);
-    } else {
-      float clo[V], chi[V];
-      load_cached_chunk<TW, FMT>(kv.k, kv.k_meta, src, n_kv, hd, h, c * V, clo);
-      load_cached_chunk<TW, FMT>(kv.k, kv.k_meta, src, n_kv, hd, h, half + c * V, chi);
-      const float2* rot = table + (size_t)maps.ctx_off[u] * half + c * V;
-      const float* mu = mu_k + ((size_t)u * n_kv + h) * hd + c * V;
+  const int groups = (T_tok + COR_TOK - 1) / COR_TOK;
+  const int total = groups * n_kv * ch;                 // < 2^31: checked by the launcher
+  const bool weighted = w_k != nullptr;
+  for (int idx = blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += gridDim.x * blockDim.x) {
+    const int c = idx % ch;
+    const int h = (idx / ch) % n_kv;
+    const int j0 = (idx / (ch * n_kv)) * COR_TOK;
+    int4 meta[COR_TOK];
+    float wk[COR_TOK], wv[COR_TOK];
 #pragma unroll
-      for (int i = 0; i < V; ++i) {
-        const float2 t = rot[i];
-        lo[i] = clo[i] * t.x - chi[i] * t.y;
-        hi[i] = chi[i] * t.x + clo[i] * t.y;
-        if (w_k) {
-          lo[i] = fmaf(wk, mu[i], lo[i]);
-          hi[i] = fmaf(wk, mu[half + i], hi[i]);
+    for (int t = 0; t < COR_TOK; ++t) {
+      const int j = j0 + t;
+      meta[t] = j < T_tok ? maps.tok_meta[j] : make_int4(-1, -1, -1, -1);
+      const bool ctx = j < N && weighted;
+      wk[t] = ctx ? w_k[j] : 0.f;
+      wv[t] = ctx ? w_v[j] : 0.f;
+    }
+    // ---- all loads first
+    uint4 fk_lo[COR_TOK], fk_hi[COR_TOK], fv_lo[COR_TOK], fv_hi[COR_TOK];
+    RawChunk<TW, FMT> ck_lo[COR_TOK], ck_hi[COR_TOK], cv_lo[COR_TOK], cv_hi[COR_TOK];
+#pragma unroll
+    for (int t = 0; t < COR_TOK; ++t) {
+      if (j0 + t >= T_tok) continue;
+      const bool kf = meta[t].y >= 0, vf = meta[t].z >= 0;
+      const T* fkp = k_fresh + ((size_t)(kf ? meta[t].y : 0) * n_kv + h) * hd + c * V;
+      const T* fvp = v_fresh + ((size_t)(vf ? meta[t].z : 0) * n_kv + h) * hd + c * V;
+      issue_chunk<T, TW, FMT>(kf, fkp, kv.k, kv.k_meta, meta[t].x, n_kv, hd, h, c * V, fk_lo[t], ck_lo[t]);
+      issue_chunk<T, TW, FMT>(kf, fkp + half, kv.k, kv.k_meta, meta[t].x, n_kv, hd, h, half + c * V, fk_hi[t], ck_hi[t]);
+      issue_chunk<T, TW, FMT>(vf, fvp, kv.v, kv.v_meta, meta[t].x, n_kv, hd, h, c * V, fv_lo[t], cv_lo[t]);
+      issue_chunk<T, TW, FMT>(vf, fvp + half, kv.v, kv.v_meta, meta[t].x, n_kv, hd, h, half + c * V, fv_hi[t], cv_hi[t]);
+    }
+    // ---- decode, re-align, correct, store
+    float2 rot[V];
+    float muk_lo[V], muk_hi[V], muv_lo[V], muv_hi[V];
+    int cur_unit = -1;
+#pragma unroll
+    for (int t = 0; t < COR_TOK; ++t) {
+      const int j = j0 + t;
+      if (j >= T_tok) continue;
+      const bool kf = meta[t].y >= 0, vf = meta[t].z >= 0;
+      const int u = meta[t].w;
+      if ((!kf || !vf) && u != cur_unit) {
+        cur_unit = u;
+        ld_f2<V>(table + (size_t)maps.ctx_off[u] * half + c * V, rot);
+        if (weighted) {
+          const float* mk = mu_k + ((size_t)u * n_kv + h) * hd + c * V;
+          const float* mv = mu_v + ((size_t)u * n_kv + h) * hd + c * V;
+          ld_f<V>(mk, muk_lo);
+          ld_f<V>(mk + half, muk_hi);
+          ld_f<V>(mv, muv_lo);
+          ld_f<V>(mv + half, muv_hi);
+        } else {
+#pragma unroll
+          for (int i = 0; i < V; ++i) muk_lo[i] = muk_hi[i] = muv_lo[i] = muv_hi[i] = 0.f;
         }
       }
-    }
-    st16(out_k + o, lo);
-    st16(out_k + o + half, hi);
-    // ---- V
-    if (row_v >= 0) {
-      const T* fp = v_fresh + ((size_t)row_v * n_kv + h) * hd + c * V;
-      ld16(fp, lo);
-      ld16(fp + half, hi);
-    } else {
-      load_cached_chunk<TW, FMT>(kv.v, kv.v_meta, src, n_kv, hd, h, c * V, lo);
-      load_cached_chunk<TW, FMT>(kv.v, kv.v_meta, src, n_kv, hd, h, half + c * V, hi);
-      if (w_k) {
-        const float* mu = mu_v + ((size_t)u * n_kv + h) * hd + c * V;
+      const size_t o = ((size_t)j * n_kv + h) * hd + c * V;
+      float lo[V], hi[V];
+      decode_chunk<T, TW, FMT>(kf, fk_lo[t], ck_lo[t], lo);
+      decode_chunk<T, TW, FMT>(kf, fk_hi[t], ck_hi[t], hi);
+      if (!kf) {
 #pragma unroll
         for (int i = 0; i < V; ++i) {
-          lo[i] = fmaf(wv, mu[i], lo[i]);
-          hi[i] = fmaf(wv, mu[half + i], hi[i]);
+          const float a = lo[i], b = hi[i];
+          lo[i] = fmaf(wk[t], muk_lo[i], a * rot[i].x - b * rot[i].y);
+          hi[i] = fmaf(wk[t], muk_hi[i], b * rot[i].x + a * rot[i].y);
         }
       }
+      st16(out_k + o, lo);
+      st16(out_k + o + half, hi);
+      decode_chunk<T, TW, FMT>(vf, fv_lo[t], cv_lo[t], lo);
+      decode_chunk<T, TW, FMT>(vf, fv_hi[t], cv_hi[t], hi);
+      if (!vf) {
+#pragma unroll
+        for (int i = 0; i < V; ++i) {
+          lo[i] = fmaf(wv[t], muv_lo[i], lo[i]);
+          hi[i] = fmaf(wv[t], muv_hi[i], hi[i]);
+        }
+      }
+      st16(out_v + o, lo);
+      st16(out_v + o + half, hi);
     }
-    st16(out_v + o, lo);
-    st16(out_v + o + half, hi);
   }
 }
 
@@ -470,9 +599,10 @@ int32_t launch_correct(int dtype, const KvLayer& kv, const ReqMaps& maps, const 
   if (T_tok == 0) return AKVS_OK;
   AKVS_TRY(check_kv_shape(dtype, kv, hd));
   const int V = dtype == AKVS_F32 ? 4 : 8;
-  const int64_t total = (int64_t)T_tok * n_kv * (hd / 2 / V);
+  const int64_t total = (int64_t)((T_tok + COR_TOK - 1) / COR_TOK) * n_kv * (hd / 2 / V);
+  if (total >= (1ll << 31) - (1 << 20)) return AKVS_ERR_SHAPE;
   int64_t want = (total + 255) / 256;
-  const int grid = (int)(want < 148 * 8 ? want : 148 * 8);   // grid-stride; 8 CTAs of 256 threads per SM
+  const int grid = (int)(want < 148 * 4 ? want : 148 * 4);   // grid-stride; two resident CTAs of 256 threads per SM
   // algorithmic bytes: every context K and V element read once in its cache format and
   // written once; fresh rows and query rows copied; 8 bytes of weights per context token
   const double in_b = kv.fmt == AKVS_KV_NATIVE ? (double)dtype_size(dtype) : kv.fmt / 8.0 + 4.0 / 64.0;
