@@ -40,12 +40,6 @@ def peaks():
         return {"hbm": 6650.0, "tensor": 1400.0, "src": "fallback"}
 
 
-def make_layers(m, n_threads):
-    from concurrent.futures import ThreadPoolExecutor
-    with ThreadPoolExecutor(n_threads) as ex:
-        return list(ex.map(lambda l: testgen.layer_weights(m, SEED_W, l), range(m.n_layers)))
-
-
 class ClockSampler:
     """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
     Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
@@ -78,6 +72,23 @@ class ClockSampler:
         busy = sorted(sm)[len(sm) // 2:] if sm else []
         return {"sm_mhz": float(np.median(busy)) if busy else None, "sm_max_mhz": max(mx) if mx else None,
                 "reasons": reasons, "samples": len(sm)}
+
+
+def max_over_ranks(value, world, device="cuda"):
+    """Multi-GPU numbers are the slowest rank's: all-reduce MAX over the process group."""
+    if world <= 1:
+        return float(value)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([float(value)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_rate(tokens_per_rank, world, ms):
+    """Replicas: every rank prefills its own request; the job's rate is the sum over ranks
+    divided by the slowest rank's time."""
+    return world * tokens_per_rank / (ms * 1e-3)
 
 
 def reference_arm(args, w):
@@ -162,9 +173,8 @@ def main():
     # ---------------------------------------------------------------- synthetic inputs
     t_setup = time.time()
     cores = len(os.sched_getaffinity(0))
-    layers = make_layers(m, max(1, min(16, cores // max(1, world))))
-    gmodel = akvs.Model.from_numpy(m, testgen.embedding(m, SEED_W), layers)
-    del layers
+    gmodel = akvs.Model.from_layer_fn(m, testgen.embedding(m, SEED_W), lambda l: testgen.layer_weights(m, SEED_W, l),
+                                      n_threads=max(1, min(12, cores // max(1, world))))
     lens = testgen.unit_lengths(w, SEED_LEN)
     ctx_ids, qry_ids = testgen.token_ids(w, SEED_IDS, lens)
     kvf = {"native": akvs.KV_NATIVE, "q4": akvs.KV_Q4, "q2": akvs.KV_Q2}[w.kv_format]
@@ -206,12 +216,7 @@ def main():
             fn()
         b.record()
         barrier()
-        ms = a.elapsed_time(b)
-        if world > 1:
-            t = torch.tensor([ms], device="cuda")
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
-        return ms / steps
+        return max_over_ranks(a.elapsed_time(b), world) / steps
 
     # ---------------------------------------------------------------- device-resident timing
     akvs.prof_enable((1 << 1) | (1 << 2) | (1 << 3), 8192)
@@ -301,7 +306,7 @@ def main():
         val, _, ccores, sample = reference_arm(a2, w)
         cpu = {"value": val, "unit": UNIT, "cores": ccores, "kind": "oracle", "sample": sample}
     out = {
-        "metric": metric, "value": world * T / (ms_step * 1e-3), "unit": UNIT, "n_gpus": world,
+        "metric": metric, "value": whole_job_rate(T, world, ms_step), "unit": UNIT, "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None,
         "dtype": {"f16": "f16 storage (bf16-valued random-init weights), f32 accumulate",
@@ -315,7 +320,7 @@ def main():
                          f"({sum(p.numel() * p.element_size() for l in gmodel.layers for p in l.values()) / 1e9:.1f} GB)",
                    "seeds": [SEED_W, SEED_IDS, SEED_LEN]},
         "clocks": clocks,
-        "e2e": {"value": world * T / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
+        "e2e": {"value": whole_job_rate(T, world, e2e_ms), "unit": UNIT, "ms_per_step": e2e_ms,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "what": "unit cache + ids from pinned host memory each step, query hidden state back"},
         "gpu_launches": int(launches),

@@ -124,6 +124,29 @@ class Model:
         self.desc = d
 
     @classmethod
+    def from_layer_fn(cls, cfg, tok_emb, layer_fn, n_threads=8, device="cuda"):
+        """Uploads a model layer by layer: `layer_fn(l)` returns the host arrays of layer l.  At
+        most `n_threads` layers are resident on the host at a time (the 32B-class model does
+        not fit in host memory as float32)."""
+        from concurrent.futures import ThreadPoolExecutor
+        dtype = {"f32": F32, "bf16": BF16, "f16": F16}[cfg.dtype]
+        td = _tdtype(dtype)
+        up = lambda a, t: torch.from_numpy(a).to(device=device, dtype=t).contiguous()
+        dl = [None] * cfg.n_layers
+        with ThreadPoolExecutor(n_threads) as ex:
+            pending = {}
+            nxt = 0
+            for l in range(cfg.n_layers):
+                while nxt < cfg.n_layers and len(pending) < n_threads:
+                    pending[nxt] = ex.submit(layer_fn, nxt)
+                    nxt += 1
+                lw = pending.pop(l).result()
+                dl[l] = {n: up(lw[n], torch.float32 if "norm" in n else td) for n in cls.NAMES}
+                del lw
+        fn = torch.ones(cfg.d_model, dtype=torch.float32, device=device)
+        return cls(cfg, up(tok_emb, td), dl, fn, dtype)
+
+    @classmethod
     def from_numpy(cls, cfg, tok_emb, layers, final_norm=None, device="cuda"):
         """Uploads host arrays (float32 values, bf16-representable for bf16 models)."""
         dtype = {"f32": F32, "bf16": BF16, "f16": F16}[cfg.dtype]
