@@ -91,6 +91,11 @@ typedef struct akvs_cache {
   void* v;                   /* same layout                                                    */
   void* k_meta;              /* device half2 (scale, min) [L][n_tokens][n_kv][head_dim/64]; NULL if native */
   void* v_meta;
+  void* const* layer_ready;  /* host [L] of cudaEvent_t, or NULL.  When set, the library makes its stream wait
+                                for layer_ready[l] before the first read of layer l of k/v/meta, so a caller
+                                that streams an offloaded cache in over PCIe (one copy + event record per layer,
+                                on its own stream, enqueued before the call) overlaps the transfer with the
+                                prefill.  Ignored by akvs_encode_units. */
 } akvs_cache;
 
 /* One request: which units, in which order (retrieval order differs per query), and the query. */

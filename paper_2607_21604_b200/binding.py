@@ -48,7 +48,8 @@ class ModelDesc(C.Structure):
 class CacheDesc(C.Structure):
     _fields_ = [("n_units", C.c_int32), ("n_tokens", C.c_int32), ("kv_format", C.c_int32),
                 ("unit_off", C.POINTER(C.c_int32)), ("token_ids", C.c_void_p), ("k", C.c_void_p),
-                ("v", C.c_void_p), ("k_meta", C.c_void_p), ("v_meta", C.c_void_p)]
+                ("v", C.c_void_p), ("k_meta", C.c_void_p), ("v_meta", C.c_void_p),
+                ("layer_ready", C.POINTER(C.c_void_p))]
 
 
 class RequestDesc(C.Structure):
@@ -188,6 +189,18 @@ class UnitStore:
         d.k_meta = self.k_meta.data_ptr() if self.k_meta is not None else None
         d.v_meta = self.v_meta.data_ptr() if self.v_meta is not None else None
         self.desc = d
+        self._events = None
+
+    def set_layer_events(self, events):
+        """`events`: one recorded torch.cuda.Event per layer (or None to clear).  The library then
+        waits for events[l] before it first reads layer l (a cache streamed in from the host)."""
+        if events is None:
+            self._events = None
+            self.desc.layer_ready = None
+            return
+        arr = (C.c_void_p * len(events))(*[e.cuda_event for e in events])
+        self._events = (arr, events)
+        self.desc.layer_ready = C.cast(arr, C.POINTER(C.c_void_p))
 
 
 class Probes:

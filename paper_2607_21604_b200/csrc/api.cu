@@ -239,6 +239,13 @@ KvLayer cache_layer(const akvs_cache* c, const Dims& D, int l) {
   return kv;
 }
 
+// The caller may be streaming layer l of the cache in on another stream: wait for its event.
+int32_t wait_layer(const akvs_cache* c, int l, cudaStream_t st) {
+  if (c->layer_ready && c->layer_ready[l])
+    AKVS_CUDA(cudaStreamWaitEvent(st, reinterpret_cast<cudaEvent_t>(c->layer_ready[l]), 0));
+  return AKVS_OK;
+}
+
 int32_t check_cache(const akvs_cache* c, const Dims& D, bool need_kv) {
   if (!c || !c->unit_off || !c->token_ids) return AKVS_ERR_INVALID_ARG;
   if (c->n_units < 0 || c->n_tokens < 0) return AKVS_ERR_INVALID_ARG;
@@ -462,6 +469,7 @@ int32_t akvs_select_probes(const akvs_model_desc* model, const akvs_cache* cache
     void* o[2] = {ws.k, ws.v};
     AKVS_TRY(linear_multi(D, ws.x, N, D.d, 2, w, ns, o, ns, ws.status, st));
     AKVS_TRY(launch_rope(D.dtype, ws.k, ws.pos, N, D.nkv, D.hd, D.dkv, ws.rope, model->rope_base, st));
+    AKVS_TRY(wait_layer(cache, lc, st));
     AKVS_TRY(launch_scores(D.dtype, cache_layer(cache, D, lc), req_maps(ws, N), ws.k, ws.v, N, D.nkv, D.hd, ws.rope,
                            out->d_k, out->d_v, st));
   }
@@ -560,6 +568,7 @@ int32_t akvs_prefill_corrected(const akvs_model_desc* model, const akvs_cache* c
   for (int l = first_layer; l < D.L; ++l) {
     const KvLayer kv = cache_layer(cache, D, l);
     auto assemble = [&, l]() -> int32_t {
+      AKVS_TRY(wait_layer(cache, l, st));
       if (corrected)
         AKVS_TRY(launch_offsets(D.dtype, kv, maps, probes->probe_off, probes->sk_idx, probes->sv_idx, ws.k, ws.v, M,
                                 D.nkv, D.hd, ws.rope, ws.mu_k, ws.mu_v, st));

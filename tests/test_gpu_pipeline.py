@@ -197,3 +197,34 @@ def test_empty_edges():
     case = Case(w, std_scale=6.0, order=[1])
     units = _check_encode(case, case.tol)
     _run_all_modes(case, 5000, 2, units)
+
+
+def test_cache_streamed_in_behind_layer_events():
+    """An offloaded cache copied in on a side stream, one event per layer: the library waits for
+    each layer's event before it reads that layer, so the result equals the resident-cache run."""
+    case = Case(small16("f16"), std_scale=4.0)
+    case.encode()
+    a = case.akvs
+    probes, ctx, ws = case.gpu_select(2500, 2)
+    want = case.gpu_prefill(a.MODE_CORRECTED, ws, probes, ctx, 2)
+    a.free(ctx)
+    h_k, h_v = case.store.k.cpu().pin_memory(), case.store.v.cpu().pin_memory()
+    case.store.k.zero_()
+    case.store.v.zero_()
+    torch.cuda.synchronize()
+    side = torch.cuda.Stream()
+    L = case.cfg.n_layers
+    events = [torch.cuda.Event() for _ in range(L)]
+    with torch.cuda.stream(side):
+        torch.cuda._sleep(20_000_000)                      # the copies start late on purpose
+        for l in range(L):
+            case.store.k[l].copy_(h_k[l], non_blocking=True)
+            case.store.v[l].copy_(h_v[l], non_blocking=True)
+            events[l].record(side)
+    case.store.set_layer_events(events)
+    probes, ctx, ws = case.gpu_select(2500, 2)
+    got = case.gpu_prefill(a.MODE_CORRECTED, ws, probes, ctx, 2)
+    a.free(ctx)
+    case.store.set_layer_events(None)
+    for x, y in zip(got, want):
+        assert np.array_equal(x, y)
