@@ -4,16 +4,20 @@
 // One CTA = one kv head x a block of BR = 128 / g query rows (g = q heads per kv head): the
 // g heads of a row that share the kv head are stacked along M, so one K/V tile in shared
 // memory serves all of them.  Per key tile of 128 keys:
-//     S  = Q K^T          tcgen05.mma 128x128x16 x8,  float in tensor memory
-//     P  = exp2(S*c - m)  4 softmax warps, one M row per thread (no shuffles), written to
-//                         shared memory as the 16-bit A operand in the 128-byte-swizzled layout
-//     O_j = P V           tcgen05.mma 128x128x16 x8 with V as an MN-major B operand
+//     S  = Q K^T          tcgen05.mma 128x128x16 x8, float in tensor memory
+//     P  = exp2(S*c - m)  4 softmax warps, one M row per thread (no shuffles); the 16-bit
+//                         probabilities go back into the first 64 columns of the S buffer
+//                         (tcgen05.st), two per 32-bit column
+//     O_j = P V           tcgen05.mma 128x128x16 x8 with P read from tensor memory as the A
+//                         operand and V from shared memory as an MN-major B operand
 //     O  = O*corr + O_j   accumulated in registers by 4 more warps (no TMEM read-modify-write)
-// S and O_j are double-buffered in tensor memory (4 x 128 columns) so that the tensor pipe
-// computes S(j+1) and O(j-1) while the softmax of tile j runs.  Warp 0 feeds K and V tiles
-// by TMA (two stages each), warp 1 issues the MMAs, warps 2-5 do the softmax (a whole S row
-// is pulled into registers with one wait), warps 6-9 fold the P V products into the output
-// rows they keep in registers; the per-tile rescale factors travel through shared memory.
+// S/P and O_j are double-buffered in tensor memory (4 x 128 columns): the tensor pipe computes
+// S(j+1) and O(j-1) while the softmax of tile j runs; the in-order tensor pipe itself keeps
+// S(j+2) from overwriting P(j) before P(j) V(j) has read it.  Keeping P out of shared memory
+// leaves room for three K and three V stages and halves the shared-memory traffic of P V.
+// Warp 0 feeds K and V tiles by TMA, warp 1 issues the MMAs, warps 2-5 do the softmax,
+// warps 6-9 fold the P V products into the output rows they keep in registers; the per-tile
+// rescale factors travel through shared memory.
 // Row blocks are taken longest first across all kv heads (the last rows see the most keys).
 // Query row r sees keys k_lo[r] <= j <= k_hi[r]; both arrays are non-decreasing in r.
 #include "tc_common.cuh"
@@ -25,8 +29,9 @@ constexpr int BN = 128;              // keys per tile
 constexpr int SLAB = 128 * 64 * 2;   // one 64-wide slab of a 128-row tile: 16 KB
 constexpr int TILE = 2 * SLAB;       // 32 KB
 constexpr int ATT_THREADS = 320;
-// shared memory: Q | K[2] | V[2] | P[2] | barriers
-constexpr int OFF_Q = 0, OFF_K = TILE, OFF_V = 3 * TILE, OFF_P = 5 * TILE, OFF_BAR = 7 * TILE;
+constexpr int KV_STAGES = 3;
+// shared memory: Q | K[3] | V[3] | barriers | rescale factors
+constexpr int OFF_Q = 0, OFF_K = TILE, OFF_V = 4 * TILE, OFF_BAR = 7 * TILE;
 constexpr int OFF_CORR = OFF_BAR + 256;      // float corr[4][128], float l_final[128]
 constexpr int ATT_SMEM = OFF_CORR + 5 * 128 * 4;   // 232192 of the 232448 bytes a CTA may own: no slack for
                                                    // re-aligning, the buffer itself is declared 1024-byte aligned
@@ -47,8 +52,8 @@ __device__ __forceinline__ float ex2(float x) {
   return y;
 }
 
-enum { B_QFULL = 0, B_KFULL = 1, B_KEMPTY = 3, B_VFULL = 5, B_VEMPTY = 7, B_SFULL = 9, B_SEMPTY = 11, B_PFULL = 13,
-       B_PEMPTY = 15, B_OFULL = 17, B_OEMPTY = 19, B_COUNT = 21 };
+enum { B_QFULL = 0, B_KFULL = 1, B_KEMPTY = 4, B_VFULL = 7, B_VEMPTY = 10, B_SFULL = 13, B_PFULL = 15, B_OFULL = 17,
+       B_OEMPTY = 19, B_COUNT = 21 };
 
 template <typename T>
 __global__ void __launch_bounds__(ATT_THREADS, 1)
@@ -75,8 +80,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < B_COUNT; ++i) {
-      const bool four = (i >= B_SEMPTY && i < B_SEMPTY + 2) || (i >= B_PFULL && i < B_PFULL + 2) ||
-                        (i >= B_OEMPTY && i < B_OEMPTY + 2);
+      const bool four = (i >= B_PFULL && i < B_PFULL + 2) || (i >= B_OEMPTY && i < B_OEMPTY + 2);
       tc::mbar_init(&bar[i], four ? 4 : 1);
     }
     *abort_flag = 0;
@@ -105,8 +109,8 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
       tc::tma_load_3d(smem + OFF_Q + SLAB, &tmQ, 64, hk * p.g, r0, &bar[B_QFULL]);
       bool ok = true;
       for (int j = 0; j < n_tiles && ok; ++j) {
-        const int s = j & 1;
-        const uint32_t ph = ((j >> 1) & 1) ^ 1;
+        const int s = j % KV_STAGES;
+        const uint32_t ph = ((j / KV_STAGES) & 1) ^ 1;
         const int y = key_lo + j * BN;
         if (!tc::mbar_wait(&bar[B_KEMPTY + s], ph, abort_flag)) { ok = false; break; }
         tc::mbar_expect_tx(&bar[B_KFULL + s], TILE);
@@ -124,13 +128,13 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     if (lane == 0 && n_tiles > 0) {
       bool ok = tc::mbar_wait(&bar[B_QFULL], 0, abort_flag);
       const uint32_t q_addr = tc::smem_u32(smem + OFF_Q);
+      // S(j) may overwrite the buffer that held S(j-2)/P(j-2): the tensor pipe runs the MMAs of
+      // this thread in order and P(j-2) V(j-2) was issued before, so no barrier is needed
       auto issue_qk = [&](int j) -> bool {
-        const int s = j & 1;
-        const uint32_t ph = (j >> 1) & 1;
-        if (!tc::mbar_wait(&bar[B_KFULL + s], ph, abort_flag)) return false;
-        if (!tc::mbar_wait(&bar[B_SEMPTY + s], ph ^ 1, abort_flag)) return false;
+        const int s = j & 1, ks = j % KV_STAGES;
+        if (!tc::mbar_wait(&bar[B_KFULL + ks], (j / KV_STAGES) & 1, abort_flag)) return false;
         tc::fence_after_sync();
-        const uint32_t k_addr = tc::smem_u32(smem + OFF_K + s * TILE);
+        const uint32_t k_addr = tc::smem_u32(smem + OFF_K + ks * TILE);
 #pragma unroll
         for (int k = 0; k < HD / 16; ++k) {
           const uint32_t off = (k >> 2) * SLAB + (k & 3) * 32;
@@ -138,7 +142,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                       p.idesc_qk, k != 0);
         }
         tc::mma_commit(&bar[B_SFULL + s]);
-        tc::mma_commit(&bar[B_KEMPTY + s]);
+        tc::mma_commit(&bar[B_KEMPTY + ks]);
         return true;
       };
       if (ok) ok = issue_qk(0);
@@ -146,21 +150,20 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         const int s = j & 1;
         const uint32_t ph = (j >> 1) & 1;
         if (j + 1 < n_tiles && !issue_qk(j + 1)) { ok = false; break; }
-        if (!tc::mbar_wait(&bar[B_VFULL + s], ph, abort_flag)) { ok = false; break; }
+        const int vs = j % KV_STAGES;
+        if (!tc::mbar_wait(&bar[B_VFULL + vs], (j / KV_STAGES) & 1, abort_flag)) { ok = false; break; }
         if (!tc::mbar_wait(&bar[B_PFULL + s], ph, abort_flag)) { ok = false; break; }
         if (!tc::mbar_wait(&bar[B_OEMPTY + s], ph ^ 1, abort_flag)) { ok = false; break; }
         tc::fence_after_sync();
-        const uint32_t p_addr = tc::smem_u32(smem + OFF_P + s * TILE);
-        const uint32_t v_addr = tc::smem_u32(smem + OFF_V + s * TILE);
+        const uint32_t v_addr = tc::smem_u32(smem + OFF_V + vs * TILE);
 #pragma unroll
         for (int k = 0; k < BN / 16; ++k) {
-          const uint64_t da = tc::smem_desc_k_sw128(p_addr + (k >> 2) * SLAB + (k & 3) * 32);
+          // 16 keys of P = 8 packed 32-bit columns of the S/P buffer
           const uint64_t db = tc::smem_desc_mn_sw128(v_addr + k * 2048, SLAB);
-          tc::mma_f16(tmem_base + 2 * BN + s * HD, da, db, p.idesc_pv, k != 0);
+          tc::mma_f16_ts(tmem_base + 2 * BN + s * HD, tmem_base + s * BN + k * 8, db, p.idesc_pv, k != 0);
         }
         tc::mma_commit(&bar[B_OFULL + s]);
-        tc::mma_commit(&bar[B_VEMPTY + s]);
-        tc::mma_commit(&bar[B_PEMPTY + s]);
+        tc::mma_commit(&bar[B_VEMPTY + vs]);
       }
       if (!ok) { *abort_flag = 1; set_status(p.status, AKVS_ERR_TIMEOUT); }
     }
@@ -189,9 +192,6 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
       tc::tmem_ld32(lane_addr + s * BN + 64, *reinterpret_cast<float(*)[32]>(&t[64]));
       tc::tmem_ld32(lane_addr + s * BN + 96, *reinterpret_cast<float(*)[32]>(&t[96]));
       tc::tmem_ld_wait();
-      tc::fence_before_sync();
-      __syncwarp();
-      if (lane == 0) tc::mbar_arrive(&bar[B_SEMPTY + s]);      // S is in registers: the buffer is free
       const bool full_tile = lo <= j0 && j0 + BN - 1 <= hi;
       if (!full_tile) {
 #pragma unroll
@@ -215,19 +215,16 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
       }
       l_run = fmaf(l_run, corr, sum);
       if (j == n_tiles - 1) corr_ring[4 * 128 + m] = l_run;
-      // the P buffer is free once the PV product of tile j-2 has retired
-      if (!tc::mbar_wait(&bar[B_PEMPTY + s], ph ^ 1, abort_flag)) { ok = false; break; }
-      uint8_t* p_row = smem + OFF_P + s * TILE + m * 128;
+      // P overwrites the first 64 columns of this S buffer: two 16-bit probabilities per column
+      uint32_t pk[32];
 #pragma unroll
-      for (int c = 0; c < BN / 8; ++c) {                        // 16-byte chunks of the row
-        uint4 pk;
-        pk.x = pack2<T>(t[c * 8 + 0], t[c * 8 + 1]);
-        pk.y = pack2<T>(t[c * 8 + 2], t[c * 8 + 3]);
-        pk.z = pack2<T>(t[c * 8 + 4], t[c * 8 + 5]);
-        pk.w = pack2<T>(t[c * 8 + 6], t[c * 8 + 7]);
-        *reinterpret_cast<uint4*>(p_row + (c >> 3) * SLAB + (((c & 7) ^ (m & 7)) << 4)) = pk;
-      }
-      tc::fence_proxy_async();          // P writes visible to the tensor pipe
+      for (int i = 0; i < 32; ++i) pk[i] = pack2<T>(t[2 * i], t[2 * i + 1]);
+      tc::tmem_st32(lane_addr + s * BN, pk);
+#pragma unroll
+      for (int i = 0; i < 32; ++i) pk[i] = pack2<T>(t[64 + 2 * i], t[64 + 2 * i + 1]);
+      tc::tmem_st32(lane_addr + s * BN + 32, pk);
+      tc::tmem_st_wait();
+      tc::fence_before_sync();
       __syncwarp();
       if (lane == 0) tc::mbar_arrive(&bar[B_PFULL + s]);
     }
