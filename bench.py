@@ -30,6 +30,10 @@ SEED_W, SEED_IDS, SEED_LEN = 1234, 1235, 1236
 METRIC = "context tokens/s prefilled (corrected reuse, 15% refresh)"
 UNIT = "tokens/s"
 CHECK_LAYER = 2
+# dram__bytes_read.sum + dram__bytes_write.sum per gemm_tc_kernel launch (bytes), averaged over
+# the four linear-layer launches of one selective layer, from the ncu --set full capture
+# summarised in profiles/selective_layer_kernels_c3.md (algorithmic: 201 MB per launch)
+GEMM_TRAFFIC_PER_LAUNCH = {"c3": 199.9e6}
 
 
 def peaks():
@@ -264,7 +268,7 @@ def main():
     roofline = {"bound": "tensor", "kernel": "gemm_tc_kernel (all linear layers of the step)",
                 "achieved": achieved, "peak": pk["tensor"], "unit": "TFLOP/s", "frac": achieved / pk["tensor"],
                 "peak_source": pk["src"] + " bf16 cuBLAS sustained (f16 and bf16 MMAs run at the same rate)",
-                "traffic": None, "launches": len(gemm), "share_of_step": g_ms / (ms_step * args.steps),
+                "traffic": GEMM_TRAFFIC_PER_LAUNCH.get(args.workload), "launches": len(gemm), "share_of_step": g_ms / (ms_step * args.steps),
                 "by_epilogue": {{0: "qkv_store", 1: "residual", 2: "swiglu"}.get(k, str(k)):
                                 {"tflops": v[1] / (v[0] * 1e-3) / 1e12, "ms_per_step": v[0] / args.steps,
                                  "launches": v[2]} for k, v in sorted(by_epi.items())}}
