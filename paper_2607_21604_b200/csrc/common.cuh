@@ -117,12 +117,12 @@ __device__ __forceinline__ void ld16(const f16* p, float (&o)[8]) {
     o[2 * i + 1] = f.y;
   }
 }
-// float -> half with saturation to the largest finite value (no infinities are produced)
+// float -> half with saturation to the largest finite value (no infinities are produced):
+// one cvt for two values; the first operand of the instruction lands in the upper half
 __device__ __forceinline__ uint32_t pack_f16x2(float a, float b) {
-  a = fminf(fmaxf(a, -65504.f), 65504.f);
-  b = fminf(fmaxf(b, -65504.f), 65504.f);
-  __half2 h = __floats2half2_rn(a, b);
-  return *reinterpret_cast<uint32_t*>(&h);
+  uint32_t r;
+  asm("cvt.rn.satfinite.f16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(b), "f"(a));
+  return r;
 }
 __device__ __forceinline__ void st16(f16* p, const float (&o)[8]) {
   uint4 v;
@@ -144,7 +144,8 @@ template <typename T> __device__ __forceinline__ T from_f(float x);
 template <> __device__ __forceinline__ float from_f<float>(float x) { return x; }
 template <> __device__ __forceinline__ bf16 from_f<bf16>(float x) { return __float2bfloat16_rn(x); }
 template <> __device__ __forceinline__ f16 from_f<f16>(float x) {
-  return __float2half_rn(fminf(fmaxf(x, -65504.f), 65504.f));
+  const uint32_t r = pack_f16x2(x, 0.f);
+  return __ushort_as_half((unsigned short)(r & 0xFFFFu));
 }
 
 __device__ __forceinline__ float warp_sum(float v) {
