@@ -174,8 +174,11 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     const int r_local = m / p.g;
     const int r = r0 + r_local;
     const bool valid = r_local < p.BR && r < p.R;
-    const int lo = valid ? p.k_lo[r] : 1;
-    const int hi = valid ? p.k_hi[r] : 0;
+    const int hi = valid ? p.k_hi[r] : -1;
+    const int lo = valid && p.k_lo[r] <= hi ? p.k_lo[r] : 0x40000000;   // nothing visible: no key reaches lo
+    // key visible  <=>  lo <= key <= hi  <=>  (unsigned)(key - lo) <= hi - lo: one compare and a
+    // select per element (a per-element && / || compiles to divergent branches, measured 2x slower)
+    const unsigned span = hi >= lo ? (unsigned)(hi - lo) : 0u;
     const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16);
     float* corr_ring = reinterpret_cast<float*>(smem + OFF_CORR);
     float m_run = -1.0e30f, l_run = 0.f;
@@ -196,23 +199,26 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
       if (!full_tile) {
 #pragma unroll
         for (int i = 0; i < BN; ++i) {
-          const int key = j0 + i;
-          t[i] = (key >= lo && key <= hi) ? t[i] : -INFINITY;
+          t[i] = ((unsigned)(j0 + i - lo) <= span) ? t[i] : -INFINITY;
         }
       }
-      float mx = -INFINITY;
+      // four independent chains each for the maximum and the sum: a scheduler that runs one
+      // softmax warp cannot hide a 128-long dependent chain
+      float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-      for (int i = 0; i < BN; ++i) mx = fmaxf(mx, t[i]);
+      for (int i = 0; i < BN; ++i) mx4[i & 3] = fmaxf(mx4[i & 3], t[i]);
+      const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
       const float m_new = fmaxf(m_run, mx * p.scale_log2);
       const float corr = ex2(m_run - m_new);
       m_run = m_new;
       corr_ring[(j & 3) * 128 + m] = corr;
-      float sum = 0.f;
+      float sum4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
       for (int i = 0; i < BN; ++i) {
         t[i] = ex2(fmaf(t[i], p.scale_log2, -m_new));          // exp2(-inf) = 0 for masked keys
-        sum += t[i];
+        sum4[i & 3] += t[i];
       }
+      const float sum = (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
       l_run = fmaf(l_run, corr, sum);
       if (j == n_tiles - 1) corr_ring[4 * 128 + m] = l_run;
       // P overwrites the first 64 columns of this S buffer: two 16-bit probabilities per column
