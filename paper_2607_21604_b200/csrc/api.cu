@@ -155,13 +155,27 @@ struct Ctx {                   // host object that carries a request from select
 // ----------------------------------------------------------------------------- linear layers
 int g_bf16_linear_algo = 0;    // 16-bit models: 0 = tcgen05; 1 = CUDA cores (kept for cross-checking)
 
+// Projections that share the input x.  Segments whose bit is set in rope_mask are [M][heads][hd]
+// tensors that get RoPE at pos[row]: fused into the tensor-core epilogue when hd == 128,
+// otherwise done by the rotation kernel afterwards.
 int32_t linear_multi(const Dims& D, const void* x, int M, int K, int n_seg, const void* const* w, const int* n,
-                     void* const* out, const int* ldc, int32_t* status, cudaStream_t st) {
+                     void* const* out, const int* ldc, int32_t* status, cudaStream_t st,
+                     const float2* rope = nullptr, const int32_t* pos = nullptr, int rope_mask = 0,
+                     float rope_base = 0.f) {
   bool tc_ok = D.dtype != AKVS_F32 && g_bf16_linear_algo == 0 && K % 8 == 0;
   for (int i = 0; i < n_seg; ++i) tc_ok = tc_ok && n[i] % 128 == 0;
-  if (tc_ok) return launch_linear_tc(D.dtype, 0, x, M, K, n_seg, w, n, out, ldc, status, st);
-  for (int i = 0; i < n_seg; ++i)
-    AKVS_TRY(launch_linear_simt(D.dtype, x, w[i], nullptr, out[i], nullptr, M, n[i], K, ldc[i], st));
+  const bool fuse = tc_ok && D.hd == 128;
+  if (tc_ok) {
+    AKVS_TRY(launch_linear_tc(D.dtype, 0, x, M, K, n_seg, w, n, out, ldc, status, st, fuse ? rope : nullptr, pos,
+                              rope_mask));
+  } else {
+    for (int i = 0; i < n_seg; ++i)
+      AKVS_TRY(launch_linear_simt(D.dtype, x, w[i], nullptr, out[i], nullptr, M, n[i], K, ldc[i], st));
+  }
+  if (!fuse)
+    for (int i = 0; i < n_seg; ++i)
+      if ((rope_mask >> i) & 1)
+        AKVS_TRY(launch_rope(D.dtype, out[i], pos, M, n[i] / D.hd, D.hd, ldc[i], rope, rope_base, st));
   return AKVS_OK;
 }
 int32_t linear_resid(const Dims& D, const void* x, int M, int K, const void* w, int n, float* h, int32_t* status,
@@ -206,10 +220,8 @@ int32_t run_layer(const akvs_model_desc* m, const Dims& D, int l, const Workspac
     const void* w[3] = {m->wq[l], m->wk[l], m->wv[l]};
     const int ns[3] = {D.dq, D.dkv, D.dkv};
     void* out[3] = {ws.q, k_dst, v_dst};
-    AKVS_TRY(linear_multi(D, ws.x, n, D.d, 3, w, ns, out, ns, ws.status, st));
+    AKVS_TRY(linear_multi(D, ws.x, n, D.d, 3, w, ns, out, ns, ws.status, st, ws.rope, pos, 0b011, m->rope_base));
   }
-  AKVS_TRY(launch_rope(D.dtype, ws.q, pos, n, D.nq, D.hd, D.dq, ws.rope, m->rope_base, st));
-  AKVS_TRY(launch_rope(D.dtype, k_dst, pos, n, D.nkv, D.hd, D.dkv, ws.rope, m->rope_base, st));
   if (between) AKVS_TRY(between());
   AKVS_TRY(attention(D, ws.q, attn_k, attn_v, ws.ao, lo, hi, n, n_keys, ws.status, st));
   AKVS_TRY(linear_resid(D, ws.ao, n, D.dq, m->wo[l], D.d, ws.h, ws.status, st));
@@ -467,8 +479,7 @@ int32_t akvs_select_probes(const akvs_model_desc* model, const akvs_cache* cache
     const void* w[2] = {model->wk[lc], model->wv[lc]};
     const int ns[2] = {D.dkv, D.dkv};
     void* o[2] = {ws.k, ws.v};
-    AKVS_TRY(linear_multi(D, ws.x, N, D.d, 2, w, ns, o, ns, ws.status, st));
-    AKVS_TRY(launch_rope(D.dtype, ws.k, ws.pos, N, D.nkv, D.hd, D.dkv, ws.rope, model->rope_base, st));
+    AKVS_TRY(linear_multi(D, ws.x, N, D.d, 2, w, ns, o, ns, ws.status, st, ws.rope, ws.pos, 0b01, model->rope_base));
     AKVS_TRY(wait_layer(cache, lc, st));
     AKVS_TRY(launch_scores(D.dtype, cache_layer(cache, D, lc), req_maps(ws, N), ws.k, ws.v, N, D.nkv, D.hd, ws.rope,
                            out->d_k, out->d_v, st));

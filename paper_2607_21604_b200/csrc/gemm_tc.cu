@@ -32,6 +32,11 @@ struct GemmParams {
   int seg_ldc[3];
   int32_t* status;
   uint32_t idesc;         // tcgen05 instruction descriptor (operand formats, M, N)
+  // fused RoPE (EPI_STORE only): segments whose bit is set in rope_mask hold heads of 128
+  // columns; row r is rotated through rope[pos[r]] (rotate-half pairs (i, i + 64)) before the store
+  const float2* rope;     // [positions][64] (cos, sin)
+  const int32_t* pos;     // [M]
+  int rope_mask;
 };
 
 // Which weight matrix and which of its rows the 128-row block `block` of the concatenated
@@ -187,6 +192,35 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           locate(p, 2 * tn + hf, seg, brow);
           const bool valid = brow < p.seg_blocks[seg] * BNH;
           const int ldc = p.seg_ldc[seg];
+          if (EPI == EPI_STORE && ((p.rope_mask >> seg) & 1)) {
+            // this 128-column block is one head: rotate the pairs (i, i + 64) in registers
+            const float2* rt = p.rope + (size_t)(row < p.M ? p.pos[row] : 0) * 64;
+#pragma unroll 1
+            for (int c = 0; c < 2; ++c) {
+              float lo[32], hi[32];
+              tc::tmem_ld32(t_addr + hf * BNH + c * 32, lo);
+              tc::tmem_ld32(t_addr + hf * BNH + 64 + c * 32, hi);
+              tc::tmem_ld_wait();
+              if (row < p.M && valid) {
+                T* o = reinterpret_cast<T*>(p.seg_out[seg]) + (size_t)row * ldc + brow + c * 32;
+#pragma unroll
+                for (int v = 0; v < 4; ++v) {
+                  float rl[8], rh[8];
+#pragma unroll
+                  for (int i = 0; i < 8; i += 2) {
+                    const float4 cs = *reinterpret_cast<const float4*>(rt + c * 32 + v * 8 + i);   // two (cos, sin)
+                    rl[i] = lo[v * 8 + i] * cs.x - hi[v * 8 + i] * cs.y;
+                    rh[i] = hi[v * 8 + i] * cs.x + lo[v * 8 + i] * cs.y;
+                    rl[i + 1] = lo[v * 8 + i + 1] * cs.z - hi[v * 8 + i + 1] * cs.w;
+                    rh[i + 1] = hi[v * 8 + i + 1] * cs.z + lo[v * 8 + i + 1] * cs.w;
+                  }
+                  st16(o + v * 8, rl);
+                  st16(o + 64 + v * 8, rh);
+                }
+              }
+            }
+            continue;
+          }
 #pragma unroll 1
           for (int c = 0; c < BNH / 32; ++c) {
             float a[32];
@@ -299,7 +333,8 @@ int32_t encode_tmap_3d_16bit(CUtensorMap* map, const void* base, uint64_t d0, ui
 //   epi 0: out[i] = x w[i]^T (16-bit);   epi 1: out[0] (float) += x w[0]^T;
 //   epi 2: out[0] = silu(x w[0]^T) * (x w[1]^T) (16-bit), n[0] == n[1].
 int32_t launch_linear_tc(int dtype, int epi, const void* x, int M, int K, int n_seg, const void* const* w, const int* n,
-                         void* const* out, const int* ldc, int32_t* status, cudaStream_t st) {
+                         void* const* out, const int* ldc, int32_t* status, cudaStream_t st, const float2* rope,
+                         const int32_t* pos, int rope_mask) {
   if (M == 0) return AKVS_OK;
   if (K % 8 != 0 || n_seg < 1 || n_seg > 3) return AKVS_ERR_SHAPE;
   if (dtype != AKVS_BF16 && dtype != AKVS_F16) return AKVS_ERR_UNSUPPORTED;
@@ -318,6 +353,9 @@ int32_t launch_linear_tc(int dtype, int epi, const void* x, int M, int K, int n_
   p.K = K;
   p.n_seg = n_seg;
   p.status = status;
+  p.rope = rope;
+  p.pos = pos;
+  p.rope_mask = (epi == EPI_STORE && rope && pos) ? rope_mask : 0;
   const uint32_t fmt = dtype == AKVS_F16 ? tc::kF16 : tc::kBF16;
   p.idesc = tc::idesc_f16(fmt, fmt, BM, 2 * BNH, 0);
   CUtensorMap tmA, tmB[3];
