@@ -5,19 +5,26 @@
 // g heads of a row that share the kv head are stacked along M, so one K/V tile in shared
 // memory serves all of them.  Per key tile of 128 keys:
 //     S  = Q K^T          tcgen05.mma 128x128x16 x8, float in tensor memory
-//     P  = exp2(S*c - m)  4 softmax warps, one M row per thread (no shuffles); the 16-bit
-//                         probabilities go back into the first 64 columns of the S buffer
-//                         (tcgen05.st), two per 32-bit column
-//     O_j = P V           tcgen05.mma 128x128x16 x8 with P read from tensor memory as the A
-//                         operand and V from shared memory as an MN-major B operand
-//     O  = O*corr + O_j   accumulated in registers by 4 more warps (no TMEM read-modify-write)
-// S/P and O_j are double-buffered in tensor memory (4 x 128 columns): the tensor pipe computes
-// S(j+1) and O(j-1) while the softmax of tile j runs; the in-order tensor pipe itself keeps
-// S(j+2) from overwriting P(j) before P(j) V(j) has read it.  Keeping P out of shared memory
-// leaves room for three K and three V stages and halves the shared-memory traffic of P V.
-// Warp 0 feeds K and V tiles by TMA, warp 1 issues the MMAs, warps 2-5 do the softmax,
-// warps 6-9 fold the P V products into the output rows they keep in registers; the per-tile
-// rescale factors travel through shared memory.
+//     P  = exp2(S*c - m)  one M row per thread (no shuffles); the 16-bit probabilities go back
+//                         into the first 64 columns of the S buffer (tcgen05.st), two per
+//                         32-bit column
+//     O += P V            tcgen05.mma 128x128x16 x8 with P read from tensor memory as the A
+//                         operand and V from shared memory as an MN-major B operand; O stays
+//                         in tensor memory for the whole key loop
+// The exponentials bound the kernel (the special-function unit of a scheduler needs ~1030
+// cycles for the 32 x 128 values of its rows, as long as the 16 MMAs of the tile), so the
+// softmax of consecutive tiles overlaps: two warp groups take the even and the odd key tiles
+// and S is triple-buffered (tensor-memory columns: O 0..127, S0..S2 128..511); the tensor
+// pipe works two tiles ahead of the softmax.
+// Both groups scale their probabilities to one reference maximum m per row, kept in shared
+// memory and handed from tile to tile (the group of tile j takes it over from the group of
+// tile j-1 through an mbarrier per warp pair).  m is raised only when a tile's maximum
+// exceeds it by more than 8 (in log2 units): the probabilities then stay below 2^8, and the
+// rows of O in tensor memory are rescaled by that warp before its P V is issued - a rare
+// event after the first tiles.  Each group keeps the row sums of its own tiles; the two
+// halves are combined after the last tile and the groups write half of the columns each.
+// Warp 0 feeds Q and K tiles by TMA, warp 2 the V tiles, warp 1 issues the MMAs; the in-order
+// tensor pipe itself keeps S(j+3) from overwriting P(j) before P(j) V(j) has read it.
 // Row blocks are taken longest first across all kv heads (the last rows see the most keys).
 // Query row r sees keys k_lo[r] <= j <= k_hi[r]; both arrays are non-decreasing in r.
 #include "tc_common.cuh"
@@ -28,12 +35,14 @@ constexpr int HD = 128;              // head dimension
 constexpr int BN = 128;              // keys per tile
 constexpr int SLAB = 128 * 64 * 2;   // one 64-wide slab of a 128-row tile: 16 KB
 constexpr int TILE = 2 * SLAB;       // 32 KB
-constexpr int ATT_THREADS = 320;
+constexpr int ATT_THREADS = 384;     // warp group 0: TMA / MMA, warp groups 1 and 2: softmax
 constexpr int KV_STAGES = 3;
-// shared memory: Q | K[3] | V[3] | barriers | rescale factors
+constexpr int S_BUFS = 3;
+constexpr float RESCALE_STEP = 8.f;  // the reference maximum may lag a tile's maximum by this much
+// shared memory: Q | K[3] | V[3] | barriers | reference maxima and row sums
 constexpr int OFF_Q = 0, OFF_K = TILE, OFF_V = 4 * TILE, OFF_BAR = 7 * TILE;
-constexpr int OFF_CORR = OFF_BAR + 256;      // float corr[4][128], float l_final[128]
-constexpr int ATT_SMEM = OFF_CORR + 5 * 128 * 4;   // 232192 of the 232448 bytes a CTA may own: no slack for
+constexpr int OFF_ROW = OFF_BAR + 512;       // float m_ref[128], l_part[2][128], m_part[2][128]
+constexpr int ATT_SMEM = OFF_ROW + 5 * 128 * 4;    // 232448 bytes is all a CTA may own: no slack for
                                                    // re-aligning, the buffer itself is declared 1024-byte aligned
 
 struct AttnParams {
@@ -52,8 +61,12 @@ __device__ __forceinline__ float ex2(float x) {
   return y;
 }
 
-enum { B_QFULL = 0, B_KFULL = 1, B_KEMPTY = 4, B_VFULL = 7, B_VEMPTY = 10, B_SFULL = 13, B_PFULL = 15, B_OFULL = 17,
-       B_OEMPTY = 19, B_COUNT = 21 };
+enum { B_QFULL = 0, B_KFULL = 1, B_KEMPTY = 4, B_VFULL = 7, B_VEMPTY = 10, B_SFULL = 13, B_PFULL = 16,
+       B_ODONE = 19,    // [2] P V of an even / odd tile has completed
+       B_OFINAL = 21,   // the last P V has completed
+       B_DEC = 22,      // [2][4] the warp of this quad has settled the reference maximum of an even / odd tile
+       B_FIN = 30,      // [4] both warps of this quad have published their row sums
+       B_COUNT = 34 };
 
 template <typename T>
 __global__ void __launch_bounds__(ATT_THREADS, 1)
@@ -67,6 +80,9 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
   uint64_t* bar = reinterpret_cast<uint64_t*>(smem + OFF_BAR);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar + B_COUNT);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  float* m_ref = reinterpret_cast<float*>(smem + OFF_ROW);       // [128]
+  float* l_part = m_ref + 128;                                    // [2][128]
+  float* m_part = m_ref + 3 * 128;                                // [2][128]
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   // 1-D grid, kv head fastest: CTAs are handed out longest row block first across ALL heads
@@ -80,13 +96,16 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < B_COUNT; ++i) {
-      const bool four = (i >= B_PFULL && i < B_PFULL + 2) || (i >= B_OEMPTY && i < B_OEMPTY + 2);
-      tc::mbar_init(&bar[i], four ? 4 : 1);
+      int count = 1;
+      if (i >= B_PFULL && i < B_PFULL + S_BUFS) count = 4;     // the four warps of the tile's group
+      if (i >= B_FIN) count = 2;                                // one warp of each group
+      tc::mbar_init(&bar[i], count);
     }
     *abort_flag = 0;
     tc::fence_barrier_init();
     tc::fence_proxy_async();
   }
+  if (threadIdx.x < 128) m_ref[threadIdx.x] = -1.0e30f;
   if (warp == 1) {
     tc::tmem_alloc(tmem_slot, 512);
     tc::tmem_relinquish();
@@ -95,83 +114,102 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
   __syncthreads();
   tc::fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
-  // tensor-memory columns: S0 0..127, S1 128..255, O0 256..383, O1 384..511
+  constexpr uint32_t COL_S = HD;                  // O: columns 0..127, S buffer i: 128 + 128 i
 
-  if (warp == 0) {
-    // -------------------------------------------------------------------- TMA producer
-    if (lane == 0 && n_tiles > 0) {
-      tc::prefetch_tmap(&tmQ);
-      tc::prefetch_tmap(&tmK);
-      tc::prefetch_tmap(&tmV);
-      const uint32_t q_bytes = (uint32_t)(2 * p.BR * p.g * 128);
-      tc::mbar_expect_tx(&bar[B_QFULL], q_bytes);
-      tc::tma_load_3d(smem + OFF_Q, &tmQ, 0, hk * p.g, r0, &bar[B_QFULL]);
-      tc::tma_load_3d(smem + OFF_Q + SLAB, &tmQ, 64, hk * p.g, r0, &bar[B_QFULL]);
-      bool ok = true;
-      for (int j = 0; j < n_tiles && ok; ++j) {
-        const int s = j % KV_STAGES;
-        const uint32_t ph = ((j / KV_STAGES) & 1) ^ 1;
-        const int y = key_lo + j * BN;
-        if (!tc::mbar_wait(&bar[B_KEMPTY + s], ph, abort_flag)) { ok = false; break; }
-        tc::mbar_expect_tx(&bar[B_KFULL + s], TILE);
-        tc::tma_load_2d(smem + OFF_K + s * TILE, &tmK, hk * HD, y, &bar[B_KFULL + s]);
-        tc::tma_load_2d(smem + OFF_K + s * TILE + SLAB, &tmK, hk * HD + 64, y, &bar[B_KFULL + s]);
-        if (!tc::mbar_wait(&bar[B_VEMPTY + s], ph, abort_flag)) { ok = false; break; }
-        tc::mbar_expect_tx(&bar[B_VFULL + s], TILE);
-        tc::tma_load_2d(smem + OFF_V + s * TILE, &tmV, hk * HD, y, &bar[B_VFULL + s]);
-        tc::tma_load_2d(smem + OFF_V + s * TILE + SLAB, &tmV, hk * HD + 64, y, &bar[B_VFULL + s]);
-      }
-      if (!ok) { *abort_flag = 1; set_status(p.status, AKVS_ERR_TIMEOUT); }
-    }
-  } else if (warp == 1) {
-    // -------------------------------------------------------------------- MMA issuer
-    if (lane == 0 && n_tiles > 0) {
-      bool ok = tc::mbar_wait(&bar[B_QFULL], 0, abort_flag);
-      const uint32_t q_addr = tc::smem_u32(smem + OFF_Q);
-      // S(j) may overwrite the buffer that held S(j-2)/P(j-2): the tensor pipe runs the MMAs of
-      // this thread in order and P(j-2) V(j-2) was issued before, so no barrier is needed
-      auto issue_qk = [&](int j) -> bool {
-        const int s = j & 1, ks = j % KV_STAGES;
-        if (!tc::mbar_wait(&bar[B_KFULL + ks], (j / KV_STAGES) & 1, abort_flag)) return false;
-        tc::fence_after_sync();
-        const uint32_t k_addr = tc::smem_u32(smem + OFF_K + ks * TILE);
-#pragma unroll
-        for (int k = 0; k < HD / 16; ++k) {
-          const uint32_t off = (k >> 2) * SLAB + (k & 3) * 32;
-          tc::mma_f16(tmem_base + s * BN, tc::smem_desc_k_sw128(q_addr + off), tc::smem_desc_k_sw128(k_addr + off),
-                      p.idesc_qk, k != 0);
+  // Registers move from the TMA / MMA warp group to the two softmax groups (128 values of a
+  // row live in each thread): 40 + 2 x 232 = 504 of the 512 per thread column.  Every role
+  // branch starts with its own setmaxnreg so that the compiler budgets each region by itself.
+  if (warp < 4) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 40;");
+    if (warp == 0) {
+      // ------------------------------------------------------------------ TMA producer: Q, K
+      if (lane == 0 && n_tiles > 0) {
+        tc::prefetch_tmap(&tmQ);
+        tc::prefetch_tmap(&tmK);
+        const uint32_t q_bytes = (uint32_t)(2 * p.BR * p.g * 128);
+        tc::mbar_expect_tx(&bar[B_QFULL], q_bytes);
+        tc::tma_load_3d(smem + OFF_Q, &tmQ, 0, hk * p.g, r0, &bar[B_QFULL]);
+        tc::tma_load_3d(smem + OFF_Q + SLAB, &tmQ, 64, hk * p.g, r0, &bar[B_QFULL]);
+        bool ok = true;
+        for (int j = 0; j < n_tiles && ok; ++j) {
+          const int s = j % KV_STAGES;
+          const uint32_t ph = ((j / KV_STAGES) & 1) ^ 1;
+          const int y = key_lo + j * BN;
+          if (!tc::mbar_wait(&bar[B_KEMPTY + s], ph, abort_flag)) { ok = false; break; }
+          tc::mbar_expect_tx(&bar[B_KFULL + s], TILE);
+          tc::tma_load_2d(smem + OFF_K + s * TILE, &tmK, hk * HD, y, &bar[B_KFULL + s]);
+          tc::tma_load_2d(smem + OFF_K + s * TILE + SLAB, &tmK, hk * HD + 64, y, &bar[B_KFULL + s]);
         }
-        tc::mma_commit(&bar[B_SFULL + s]);
-        tc::mma_commit(&bar[B_KEMPTY + ks]);
-        return true;
-      };
-      if (ok) ok = issue_qk(0);
-      for (int j = 0; j < n_tiles && ok; ++j) {
-        const int s = j & 1;
-        const uint32_t ph = (j >> 1) & 1;
-        if (j + 1 < n_tiles && !issue_qk(j + 1)) { ok = false; break; }
-        const int vs = j % KV_STAGES;
-        if (!tc::mbar_wait(&bar[B_VFULL + vs], (j / KV_STAGES) & 1, abort_flag)) { ok = false; break; }
-        if (!tc::mbar_wait(&bar[B_PFULL + s], ph, abort_flag)) { ok = false; break; }
-        if (!tc::mbar_wait(&bar[B_OEMPTY + s], ph ^ 1, abort_flag)) { ok = false; break; }
-        tc::fence_after_sync();
-        const uint32_t v_addr = tc::smem_u32(smem + OFF_V + vs * TILE);
-#pragma unroll
-        for (int k = 0; k < BN / 16; ++k) {
-          // 16 keys of P = 8 packed 32-bit columns of the S/P buffer
-          const uint64_t db = tc::smem_desc_mn_sw128(v_addr + k * 2048, SLAB);
-          tc::mma_f16_ts(tmem_base + 2 * BN + s * HD, tmem_base + s * BN + k * 8, db, p.idesc_pv, k != 0);
-        }
-        tc::mma_commit(&bar[B_OFULL + s]);
-        tc::mma_commit(&bar[B_VEMPTY + vs]);
+        if (!ok) { *abort_flag = 1; set_status(p.status, AKVS_ERR_TIMEOUT); }
       }
-      if (!ok) { *abort_flag = 1; set_status(p.status, AKVS_ERR_TIMEOUT); }
+    } else if (warp == 2) {
+      // ------------------------------------------------------------------ TMA producer: V
+      if (lane == 0 && n_tiles > 0) {
+        tc::prefetch_tmap(&tmV);
+        bool ok = true;
+        for (int j = 0; j < n_tiles && ok; ++j) {
+          const int s = j % KV_STAGES;
+          const uint32_t ph = ((j / KV_STAGES) & 1) ^ 1;
+          const int y = key_lo + j * BN;
+          if (!tc::mbar_wait(&bar[B_VEMPTY + s], ph, abort_flag)) { ok = false; break; }
+          tc::mbar_expect_tx(&bar[B_VFULL + s], TILE);
+          tc::tma_load_2d(smem + OFF_V + s * TILE, &tmV, hk * HD, y, &bar[B_VFULL + s]);
+          tc::tma_load_2d(smem + OFF_V + s * TILE + SLAB, &tmV, hk * HD + 64, y, &bar[B_VFULL + s]);
+        }
+        if (!ok) { *abort_flag = 1; set_status(p.status, AKVS_ERR_TIMEOUT); }
+      }
+    } else if (warp == 1) {
+      // ------------------------------------------------------------------ MMA issuer
+      if (lane == 0 && n_tiles > 0) {
+        bool ok = tc::mbar_wait(&bar[B_QFULL], 0, abort_flag);
+        const uint32_t q_addr = tc::smem_u32(smem + OFF_Q);
+        // S(j) may overwrite the buffer that held S(j-3)/P(j-3): the tensor pipe runs the MMAs of
+        // this thread in order and P(j-3) V(j-3) was issued before, so no barrier is needed
+        auto issue_qk = [&](int j) -> bool {
+          const int s = j % S_BUFS, ks = j % KV_STAGES;
+          if (!tc::mbar_wait(&bar[B_KFULL + ks], (j / KV_STAGES) & 1, abort_flag)) return false;
+          tc::fence_after_sync();
+          const uint32_t k_addr = tc::smem_u32(smem + OFF_K + ks * TILE);
+#pragma unroll
+          for (int k = 0; k < HD / 16; ++k) {
+            const uint32_t off = (k >> 2) * SLAB + (k & 3) * 32;
+            tc::mma_f16(tmem_base + COL_S + s * BN, tc::smem_desc_k_sw128(q_addr + off),
+                        tc::smem_desc_k_sw128(k_addr + off), p.idesc_qk, k != 0);
+          }
+          tc::mma_commit(&bar[B_SFULL + s]);
+          tc::mma_commit(&bar[B_KEMPTY + ks]);
+          return true;
+        };
+        if (ok) ok = issue_qk(0);
+        if (ok && n_tiles > 1) ok = issue_qk(1);
+        for (int j = 0; j < n_tiles && ok; ++j) {
+          const int s = j % S_BUFS;
+          if (j + 2 < n_tiles && !issue_qk(j + 2)) { ok = false; break; }
+          const int vs = j % KV_STAGES;
+          if (!tc::mbar_wait(&bar[B_VFULL + vs], (j / KV_STAGES) & 1, abort_flag)) { ok = false; break; }
+          if (!tc::mbar_wait(&bar[B_PFULL + s], (j / S_BUFS) & 1, abort_flag)) { ok = false; break; }
+          tc::fence_after_sync();
+          const uint32_t v_addr = tc::smem_u32(smem + OFF_V + vs * TILE);
+#pragma unroll
+          for (int k = 0; k < BN / 16; ++k) {
+            // 16 keys of P = 8 packed 32-bit columns of the S/P buffer
+            const uint64_t db = tc::smem_desc_mn_sw128(v_addr + k * 2048, SLAB);
+            tc::mma_f16_ts(tmem_base, tmem_base + COL_S + s * BN + k * 8, db, p.idesc_pv, (j | k) != 0);
+          }
+          tc::mma_commit(&bar[B_ODONE + (j & 1)]);
+          tc::mma_commit(&bar[B_VEMPTY + vs]);
+          if (j == n_tiles - 1) tc::mma_commit(&bar[B_OFINAL]);
+        }
+        if (!ok) { *abort_flag = 1; set_status(p.status, AKVS_ERR_TIMEOUT); }
+      }
     }
-  } else if (warp < 6) {
-    // -------------------------------------------------------------------- softmax
+  } else {
+    // ---------------------------------------------------------------------- softmax groups
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 232;");
     const int quad = warp & 3;
+    const int grp = (warp >> 2) - 1;                // 0: tiles 0, 2, 4, ...   1: tiles 1, 3, 5, ...
     const int m = quad * 32 + lane;                 // row of the M tile owned by this thread
-    const int r_local = m / p.g;
+    const int r_local = m / p.g, head = m - r_local * p.g;
     const int r = r0 + r_local;
     const bool valid = r_local < p.BR && r < p.R;
     const int hi = valid ? p.k_hi[r] : -1;
@@ -180,20 +218,20 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     // select per element (a per-element && / || compiles to divergent branches, measured 2x slower)
     const unsigned span = hi >= lo ? (unsigned)(hi - lo) : 0u;
     const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16);
-    float* corr_ring = reinterpret_cast<float*>(smem + OFF_CORR);
-    float m_run = -1.0e30f, l_run = 0.f;
+    float m_mine = -1.0e30f;                        // reference maximum this thread's row sum is scaled to
+    float l_mine = 0.f;                             // row sum over this group's tiles
     bool ok = true;
-    for (int j = 0; j < n_tiles && ok; ++j) {
-      const int s = j & 1;
-      const uint32_t ph = (j >> 1) & 1;
+    for (int j = grp; j < n_tiles && ok; j += 2) {
+      const int s = j % S_BUFS;
       const int j0 = key_lo + j * BN;
-      if (!tc::mbar_wait(&bar[B_SFULL + s], ph, abort_flag)) { ok = false; break; }
+      const uint32_t s_addr = lane_addr + COL_S + s * BN;
+      if (!tc::mbar_wait(&bar[B_SFULL + s], (j / S_BUFS) & 1, abort_flag)) { ok = false; break; }
       tc::fence_after_sync();
       float t[BN];
-      tc::tmem_ld32(lane_addr + s * BN + 0, *reinterpret_cast<float(*)[32]>(&t[0]));
-      tc::tmem_ld32(lane_addr + s * BN + 32, *reinterpret_cast<float(*)[32]>(&t[32]));
-      tc::tmem_ld32(lane_addr + s * BN + 64, *reinterpret_cast<float(*)[32]>(&t[64]));
-      tc::tmem_ld32(lane_addr + s * BN + 96, *reinterpret_cast<float(*)[32]>(&t[96]));
+      tc::tmem_ld32(s_addr + 0, *reinterpret_cast<float(*)[32]>(&t[0]));
+      tc::tmem_ld32(s_addr + 32, *reinterpret_cast<float(*)[32]>(&t[32]));
+      tc::tmem_ld32(s_addr + 64, *reinterpret_cast<float(*)[32]>(&t[64]));
+      tc::tmem_ld32(s_addr + 96, *reinterpret_cast<float(*)[32]>(&t[96]));
       tc::tmem_ld_wait();
       const bool full_tile = lo <= j0 && j0 + BN - 1 <= hi;
       if (!full_tile) {
@@ -202,81 +240,93 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
           t[i] = ((unsigned)(j0 + i - lo) <= span) ? t[i] : -INFINITY;
         }
       }
-      // four independent chains each for the maximum and the sum: a scheduler that runs one
-      // softmax warp cannot hide a 128-long dependent chain
+      // four independent chains each for the maximum and the sum: a 128-long dependent chain
+      // would leave the scheduler waiting on latency
       float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
       for (int i = 0; i < BN; ++i) mx4[i & 3] = fmaxf(mx4[i & 3], t[i]);
-      const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
-      const float m_new = fmaxf(m_run, mx * p.scale_log2);
-      const float corr = ex2(m_run - m_new);
-      m_run = m_new;
-      corr_ring[(j & 3) * 128 + m] = corr;
+      const float cand = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * p.scale_log2;
+      // take the reference maximum over from tile j-1 (the other group's warp of this quad)
+      if (j > 0 && !tc::mbar_wait(&bar[B_DEC + ((j - 1) & 1) * 4 + quad], ((j - 1) >> 1) & 1, abort_flag)) {
+        ok = false;
+        break;
+      }
+      const float m_old = m_ref[m];
+      const bool raise = cand > m_old + RESCALE_STEP;
+      const float m_new = raise ? cand : m_old;
+      if (raise) m_ref[m] = m_new;
+      __syncwarp();
+      if (lane == 0 && j + 1 < n_tiles) tc::mbar_arrive(&bar[B_DEC + (j & 1) * 4 + quad]);
+      l_mine *= ex2(m_mine - m_new);
+      m_mine = m_new;
+      if (j > 0 && __any_sync(0xffffffffu, raise)) {
+        // rows of O accumulated so far move to the new maximum, once P(j-1) V(j-1) has landed
+        if (!tc::mbar_wait(&bar[B_ODONE + ((j - 1) & 1)], ((j - 1) >> 1) & 1, abort_flag)) { ok = false; break; }
+        tc::fence_after_sync();
+        const float f = ex2(m_old - m_new);         // exactly 1 for the rows that keep their maximum
+#pragma unroll 1
+        for (int c = 0; c < HD / 32; ++c) {
+          float o[32];
+          tc::tmem_ld32(lane_addr + c * 32, o);
+          tc::tmem_ld_wait();
+          uint32_t ob[32];
+#pragma unroll
+          for (int i = 0; i < 32; ++i) ob[i] = __float_as_uint(o[i] * f);
+          tc::tmem_st32(lane_addr + c * 32, ob);
+        }
+      }
       float sum4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
       for (int i = 0; i < BN; ++i) {
         t[i] = ex2(fmaf(t[i], p.scale_log2, -m_new));          // exp2(-inf) = 0 for masked keys
         sum4[i & 3] += t[i];
       }
-      const float sum = (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
-      l_run = fmaf(l_run, corr, sum);
-      if (j == n_tiles - 1) corr_ring[4 * 128 + m] = l_run;
+      l_mine += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
       // P overwrites the first 64 columns of this S buffer: two 16-bit probabilities per column
       uint32_t pk[32];
 #pragma unroll
       for (int i = 0; i < 32; ++i) pk[i] = pack2<T>(t[2 * i], t[2 * i + 1]);
-      tc::tmem_st32(lane_addr + s * BN, pk);
+      tc::tmem_st32(s_addr, pk);
 #pragma unroll
       for (int i = 0; i < 32; ++i) pk[i] = pack2<T>(t[64 + 2 * i], t[64 + 2 * i + 1]);
-      tc::tmem_st32(lane_addr + s * BN + 32, pk);
+      tc::tmem_st32(s_addr + 32, pk);
       tc::tmem_st_wait();
       tc::fence_before_sync();
       __syncwarp();
       if (lane == 0) tc::mbar_arrive(&bar[B_PFULL + s]);
     }
+    // ---- epilogue: combine the two groups' row sums, normalise, write half of the columns each
+    l_part[grp * 128 + m] = l_mine;
+    m_part[grp * 128 + m] = m_mine;
+    __syncwarp();
+    if (lane == 0) tc::mbar_arrive(&bar[B_FIN + quad]);
+    if (ok && !tc::mbar_wait(&bar[B_FIN + quad], 0, abort_flag)) ok = false;
+    if (ok && n_tiles > 0 && !tc::mbar_wait(&bar[B_OFINAL], 0, abort_flag)) ok = false;
     if (!ok && lane == 0) { *abort_flag = 1; set_status(p.status, AKVS_ERR_TIMEOUT); }
-  } else {
-    // -------------------------------------------------------------------- output accumulation
-    const int quad = warp & 3;
-    const int m = quad * 32 + lane;
-    const int r_local = m / p.g, head = m - r_local * p.g;
-    const int r = r0 + r_local;
-    const bool valid = r_local < p.BR && r < p.R;
-    const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16);
-    const float* corr_ring = reinterpret_cast<const float*>(smem + OFF_CORR);
-    float o[HD];
-#pragma unroll
-    for (int i = 0; i < HD; ++i) o[i] = 0.f;
-    bool ok = true;
-    for (int j = 0; j < n_tiles && ok; ++j) {
-      const int s = j & 1;
-      if (!tc::mbar_wait(&bar[B_OFULL + s], (j >> 1) & 1, abort_flag)) { ok = false; break; }
+    if (ok) {
       tc::fence_after_sync();
-      const float corr = corr_ring[(j & 3) * 128 + m];
-#pragma unroll
-      for (int c = 0; c < HD / 64; ++c) {
-        float t[64];
-        tc::tmem_ld32(lane_addr + 2 * BN + s * HD + c * 64, *reinterpret_cast<float(*)[32]>(&t[0]));
-        tc::tmem_ld32(lane_addr + 2 * BN + s * HD + c * 64 + 32, *reinterpret_cast<float(*)[32]>(&t[32]));
-        tc::tmem_ld_wait();
-#pragma unroll
-        for (int i = 0; i < 64; ++i) o[c * 64 + i] = fmaf(o[c * 64 + i], corr, t[i]);
-      }
-      tc::fence_before_sync();
-      __syncwarp();
-      if (lane == 0) tc::mbar_arrive(&bar[B_OEMPTY + s]);
-    }
-    if (!ok && lane == 0) { *abort_flag = 1; set_status(p.status, AKVS_ERR_TIMEOUT); }
-    if (valid) {
-      const float l = n_tiles > 0 ? corr_ring[4 * 128 + m] : 0.f;
+      const float ma = m_part[m], mb = m_part[128 + m];
+      const float m_fin = fmaxf(ma, mb);            // the maximum only grows: the later tile's is final
+      const float l = l_part[m] * ex2(ma - m_fin) + l_part[128 + m] * ex2(mb - m_fin);
       const float inv = l > 0.f ? 1.f / l : 0.f;
-      T* op = reinterpret_cast<T*>(p.out) + ((size_t)r * p.n_q + (size_t)hk * p.g + head) * HD;
+      float o[64];
+      if (n_tiles > 0) {
+        tc::tmem_ld32(lane_addr + grp * 64, *reinterpret_cast<float(*)[32]>(&o[0]));
+        tc::tmem_ld32(lane_addr + grp * 64 + 32, *reinterpret_cast<float(*)[32]>(&o[32]));
+        tc::tmem_ld_wait();
+      } else {
 #pragma unroll
-      for (int v = 0; v < HD / 8; ++v) {
-        float t[8];
+        for (int i = 0; i < 64; ++i) o[i] = 0.f;
+      }
+      if (valid) {
+        T* op = reinterpret_cast<T*>(p.out) + ((size_t)r * p.n_q + (size_t)hk * p.g + head) * HD + grp * 64;
 #pragma unroll
-        for (int i = 0; i < 8; ++i) t[i] = o[v * 8 + i] * inv;
-        st16(op + v * 8, t);
+        for (int v = 0; v < 8; ++v) {
+          float w[8];
+#pragma unroll
+          for (int i = 0; i < 8; ++i) w[i] = o[v * 8 + i] * inv;
+          st16(op + v * 8, w);
+        }
       }
     }
   }
