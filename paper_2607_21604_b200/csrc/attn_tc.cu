@@ -66,7 +66,8 @@ enum { B_QFULL = 0, B_KFULL = 1, B_KEMPTY = 4, B_VFULL = 7, B_VEMPTY = 10, B_SFU
        B_OFINAL = 21,   // the last P V has completed
        B_DEC = 22,      // [2][4] the warp of this quad has settled the reference maximum of an even / odd tile
        B_FIN = 30,      // [4] both warps of this quad have published their row sums
-       B_COUNT = 34 };
+       B_SEMPTY = 34,   // [3] the P V that read this S/P buffer has completed
+       B_COUNT = 37 };
 
 template <typename T>
 __global__ void __launch_bounds__(ATT_THREADS, 1)
@@ -98,7 +99,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     for (int i = 0; i < B_COUNT; ++i) {
       int count = 1;
       if (i >= B_PFULL && i < B_PFULL + S_BUFS) count = 4;     // the four warps of the tile's group
-      if (i >= B_FIN) count = 2;                                // one warp of each group
+      if (i >= B_FIN && i < B_FIN + 4) count = 2;                                // one warp of each group
       tc::mbar_init(&bar[i], count);
     }
     *abort_flag = 0;
@@ -159,15 +160,17 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         if (!ok) { *abort_flag = 1; set_status(p.status, AKVS_ERR_TIMEOUT); }
       }
     } else if (warp == 1) {
-      // ------------------------------------------------------------------ MMA issuer
+      // ------------------------------------------------------------------ MMA issuer: S = Q K^T
+      // Two threads feed the tensor pipe (this one and warp 3 for P V): each hides the other's
+      // barrier round trips.  MMAs of different threads are not ordered, so S(j) waits for the
+      // commit of P(j-3) V(j-3), the last reader of the buffer it overwrites.
       if (lane == 0 && n_tiles > 0) {
         bool ok = tc::mbar_wait(&bar[B_QFULL], 0, abort_flag);
         const uint32_t q_addr = tc::smem_u32(smem + OFF_Q);
-        // S(j) may overwrite the buffer that held S(j-3)/P(j-3): the tensor pipe runs the MMAs of
-        // this thread in order and P(j-3) V(j-3) was issued before, so no barrier is needed
-        auto issue_qk = [&](int j) -> bool {
+        for (int j = 0; j < n_tiles && ok; ++j) {
           const int s = j % S_BUFS, ks = j % KV_STAGES;
-          if (!tc::mbar_wait(&bar[B_KFULL + ks], (j / KV_STAGES) & 1, abort_flag)) return false;
+          if (j >= S_BUFS && !tc::mbar_wait(&bar[B_SEMPTY + s], (j / S_BUFS - 1) & 1, abort_flag)) { ok = false; break; }
+          if (!tc::mbar_wait(&bar[B_KFULL + ks], (j / KV_STAGES) & 1, abort_flag)) { ok = false; break; }
           tc::fence_after_sync();
           const uint32_t k_addr = tc::smem_u32(smem + OFF_K + ks * TILE);
 #pragma unroll
@@ -178,14 +181,15 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
           }
           tc::mma_commit(&bar[B_SFULL + s]);
           tc::mma_commit(&bar[B_KEMPTY + ks]);
-          return true;
-        };
-        if (ok) ok = issue_qk(0);
-        if (ok && n_tiles > 1) ok = issue_qk(1);
+        }
+        if (!ok) { *abort_flag = 1; set_status(p.status, AKVS_ERR_TIMEOUT); }
+      }
+    } else {
+      // ------------------------------------------------------------------ MMA issuer: O += P V
+      if (lane == 0 && n_tiles > 0) {
+        bool ok = true;
         for (int j = 0; j < n_tiles && ok; ++j) {
-          const int s = j % S_BUFS;
-          if (j + 2 < n_tiles && !issue_qk(j + 2)) { ok = false; break; }
-          const int vs = j % KV_STAGES;
+          const int s = j % S_BUFS, vs = j % KV_STAGES;
           if (!tc::mbar_wait(&bar[B_VFULL + vs], (j / KV_STAGES) & 1, abort_flag)) { ok = false; break; }
           if (!tc::mbar_wait(&bar[B_PFULL + s], (j / S_BUFS) & 1, abort_flag)) { ok = false; break; }
           tc::fence_after_sync();
@@ -197,6 +201,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             tc::mma_f16_ts(tmem_base, tmem_base + COL_S + s * BN + k * 8, db, p.idesc_pv, (j | k) != 0);
           }
           tc::mma_commit(&bar[B_ODONE + (j & 1)]);
+          tc::mma_commit(&bar[B_SEMPTY + s]);
           tc::mma_commit(&bar[B_VEMPTY + vs]);
           if (j == n_tiles - 1) tc::mma_commit(&bar[B_OFINAL]);
         }
