@@ -4,18 +4,22 @@
 // One CTA = one kv head x a block of BR = 128 / g query rows (g = q heads per kv head): the
 // g heads of a row that share the kv head are stacked along M, so one K/V tile in shared
 // memory serves all of them.  Per key tile of 128 keys:
-//     S  = Q K^T          tcgen05.mma 128x128x16 x8, float in tensor memory
-//     P  = exp2(S*c - m)  one M row per thread (no shuffles); the 16-bit probabilities go back
-//                         into the first 64 columns of the S buffer (tcgen05.st), two per
-//                         32-bit column
-//     O += P V            tcgen05.mma 128x128x16 x8 with P read from tensor memory as the A
-//                         operand and V from shared memory as an MN-major B operand; O stays
-//                         in tensor memory for the whole key loop
+//     S  = Q K^T          tcgen05.mma 128x128x16 x8, float in tensor memory; Q is the A operand
+//                         read from tensor memory (written there once per CTA), K comes from
+//                         shared memory
+//     P  = exp2(S*c - m)  one M row per thread (no shuffles); the 16-bit probabilities go to a
+//                         64-column buffer in tensor memory (tcgen05.st), two per column
+//     O += P V            tcgen05.mma 128x128x16 x8 with P as the A operand from tensor memory
+//                         and V from shared memory as an MN-major B operand; O stays in tensor
+//                         memory for the whole key loop
+// Tensor-memory columns: O 0..127 | Q 128..191 | P 192..255 | S0, S1 256..511.  With Q and P in
+// tensor memory the MMAs read only K and V from shared memory, and shared memory holds three
+// K and four V stages.
 // The exponentials bound the kernel (the special-function unit of a scheduler needs ~1030
 // cycles for the 32 x 128 values of its rows, as long as the 16 MMAs of the tile), so the
-// softmax of consecutive tiles overlaps: two warp groups take the even and the odd key tiles
-// and S is triple-buffered (tensor-memory columns: O 0..127, S0..S2 128..511); the tensor
-// pipe works two tiles ahead of the softmax.
+// softmax of consecutive tiles overlaps: two warp groups take the even and the odd key tiles,
+// each with its own S buffer, which it hands back as soon as the scores sit in registers; the
+// tensor pipe then works two tiles ahead of the softmax.
 // Both groups scale their probabilities to one reference maximum m per row, kept in shared
 // memory and handed from tile to tile (the group of tile j takes it over from the group of
 // tile j-1 through an mbarrier per warp pair).  m is raised only when a tile's maximum
@@ -23,8 +27,9 @@
 // rows of O in tensor memory are rescaled by that warp before its P V is issued - a rare
 // event after the first tiles.  Each group keeps the row sums of its own tiles; the two
 // halves are combined after the last tile and the groups write half of the columns each.
-// Warp 0 feeds Q and K tiles by TMA, warp 2 the V tiles, warp 1 issues the MMAs; the in-order
-// tensor pipe itself keeps S(j+3) from overwriting P(j) before P(j) V(j) has read it.
+// Warp 0 feeds K tiles by TMA, warp 2 the V tiles; warp 1 issues Q K^T and warp 3 P V, so
+// that each issuing thread hides the other's barrier round trips (MMAs of different threads
+// are not ordered: every reuse of a tensor-memory buffer goes through an mbarrier).
 // Row blocks are taken longest first across all kv heads (the last rows see the most keys).
 // Query row r sees keys k_lo[r] <= j <= k_hi[r]; both arrays are non-decreasing in r.
 #include "tc_common.cuh"
@@ -36,17 +41,19 @@ constexpr int BN = 128;              // keys per tile
 constexpr int SLAB = 128 * 64 * 2;   // one 64-wide slab of a 128-row tile: 16 KB
 constexpr int TILE = 2 * SLAB;       // 32 KB
 constexpr int ATT_THREADS = 384;     // warp group 0: TMA / MMA, warp groups 1 and 2: softmax
-constexpr int KV_STAGES = 3;
-constexpr int S_BUFS = 3;
+constexpr int K_STAGES = 3, V_STAGES = 4;
 constexpr float RESCALE_STEP = 8.f;  // the reference maximum may lag a tile's maximum by this much
-// shared memory: Q | K[3] | V[3] | barriers | reference maxima and row sums
-constexpr int OFF_Q = 0, OFF_K = TILE, OFF_V = 4 * TILE, OFF_BAR = 7 * TILE;
+// shared memory: K[3] | V[4] | barriers | reference maxima and row sums
+constexpr int OFF_K = 0, OFF_V = K_STAGES * TILE, OFF_BAR = (K_STAGES + V_STAGES) * TILE;
 constexpr int OFF_ROW = OFF_BAR + 512;       // float m_ref[128], l_part[2][128], m_part[2][128]
 constexpr int ATT_SMEM = OFF_ROW + 5 * 128 * 4;    // 232448 bytes is all a CTA may own: no slack for
                                                    // re-aligning, the buffer itself is declared 1024-byte aligned
+// tensor-memory columns
+constexpr uint32_t COL_O = 0, COL_Q = 128, COL_P = 192, COL_S = 256;
 
 struct AttnParams {
   int R, T, n_q, n_kv, g, BR, row_blocks;
+  const void* q;
   const int32_t* k_lo;
   const int32_t* k_hi;
   void* out;
@@ -61,18 +68,21 @@ __device__ __forceinline__ float ex2(float x) {
   return y;
 }
 
-enum { B_QFULL = 0, B_KFULL = 1, B_KEMPTY = 4, B_VFULL = 7, B_VEMPTY = 10, B_SFULL = 13, B_PFULL = 16,
-       B_ODONE = 19,    // [2] P V of an even / odd tile has completed
-       B_OFINAL = 21,   // the last P V has completed
-       B_DEC = 22,      // [2][4] the warp of this quad has settled the reference maximum of an even / odd tile
-       B_FIN = 30,      // [4] both warps of this quad have published their row sums
-       B_SEMPTY = 34,   // [3] the P V that read this S/P buffer has completed
+enum { B_QFULL = 0,     // Q sits in tensor memory (4 warps)
+       B_KFULL = 1, B_KEMPTY = 4, B_VFULL = 7, B_VEMPTY = 11,
+       B_SFULL = 15,    // [2] S of an even / odd tile is complete
+       B_SEMPTY = 17,   // [2] the group has taken S into registers (4 warps)
+       B_PFULL = 19,    // P of the next tile is in tensor memory (4 warps)
+       B_ODONE = 20,    // [4] P V of tile j (slot j mod 4) has completed
+       B_OFINAL = 24,   // the last P V has completed
+       B_DEC = 25,      // [2][4] the warp of this quad has settled the reference maximum of an even / odd tile
+       B_FIN = 33,      // [4] both warps of this quad have published their row sums
        B_COUNT = 37 };
 
 template <typename T>
 __global__ void __launch_bounds__(ATT_THREADS, 1)
-attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
-                    const __grid_constant__ CUtensorMap tmV, const AttnParams p) {
+attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
+                    const AttnParams p) {
   extern __shared__ __align__(1024) uint8_t smem[];
   if (tc::smem_u32(smem) & 1023u) {               // swizzled tiles need 1024-byte alignment
     if (threadIdx.x == 0) set_status(p.status, AKVS_ERR_UNSUPPORTED);
@@ -98,8 +108,8 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
   if (threadIdx.x == 0) {
     for (int i = 0; i < B_COUNT; ++i) {
       int count = 1;
-      if (i >= B_PFULL && i < B_PFULL + S_BUFS) count = 4;     // the four warps of the tile's group
-      if (i >= B_FIN && i < B_FIN + 4) count = 2;                                // one warp of each group
+      if (i == B_QFULL || i == B_PFULL || (i >= B_SEMPTY && i < B_SEMPTY + 2)) count = 4;   // the warps of a group
+      if (i >= B_FIN && i < B_FIN + 4) count = 2;                                           // one warp of each group
       tc::mbar_init(&bar[i], count);
     }
     *abort_flag = 0;
@@ -115,7 +125,6 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
   __syncthreads();
   tc::fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
-  constexpr uint32_t COL_S = HD;                  // O: columns 0..127, S buffer i: 128 + 128 i
 
   // Registers move from the TMA / MMA warp group to the two softmax groups (128 values of a
   // row live in each thread): 40 + 2 x 232 = 504 of the 512 per thread column.  Every role
@@ -123,18 +132,13 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
   if (warp < 4) {
     asm volatile("setmaxnreg.dec.sync.aligned.u32 40;");
     if (warp == 0) {
-      // ------------------------------------------------------------------ TMA producer: Q, K
+      // ------------------------------------------------------------------ TMA producer: K
       if (lane == 0 && n_tiles > 0) {
-        tc::prefetch_tmap(&tmQ);
         tc::prefetch_tmap(&tmK);
-        const uint32_t q_bytes = (uint32_t)(2 * p.BR * p.g * 128);
-        tc::mbar_expect_tx(&bar[B_QFULL], q_bytes);
-        tc::tma_load_3d(smem + OFF_Q, &tmQ, 0, hk * p.g, r0, &bar[B_QFULL]);
-        tc::tma_load_3d(smem + OFF_Q + SLAB, &tmQ, 64, hk * p.g, r0, &bar[B_QFULL]);
         bool ok = true;
         for (int j = 0; j < n_tiles && ok; ++j) {
-          const int s = j % KV_STAGES;
-          const uint32_t ph = ((j / KV_STAGES) & 1) ^ 1;
+          const int s = j % K_STAGES;
+          const uint32_t ph = ((j / K_STAGES) & 1) ^ 1;
           const int y = key_lo + j * BN;
           if (!tc::mbar_wait(&bar[B_KEMPTY + s], ph, abort_flag)) { ok = false; break; }
           tc::mbar_expect_tx(&bar[B_KFULL + s], TILE);
@@ -149,8 +153,8 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         tc::prefetch_tmap(&tmV);
         bool ok = true;
         for (int j = 0; j < n_tiles && ok; ++j) {
-          const int s = j % KV_STAGES;
-          const uint32_t ph = ((j / KV_STAGES) & 1) ^ 1;
+          const int s = j % V_STAGES;
+          const uint32_t ph = ((j / V_STAGES) & 1) ^ 1;
           const int y = key_lo + j * BN;
           if (!tc::mbar_wait(&bar[B_VEMPTY + s], ph, abort_flag)) { ok = false; break; }
           tc::mbar_expect_tx(&bar[B_VFULL + s], TILE);
@@ -162,24 +166,24 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     } else if (warp == 1) {
       // ------------------------------------------------------------------ MMA issuer: S = Q K^T
       // Two threads feed the tensor pipe (this one and warp 3 for P V): each hides the other's
-      // barrier round trips.  MMAs of different threads are not ordered, so S(j) waits for the
-      // commit of P(j-3) V(j-3), the last reader of the buffer it overwrites.
+      // barrier round trips.  MMAs of different threads are not ordered: every reuse of a
+      // tensor-memory buffer goes through an mbarrier.
       if (lane == 0 && n_tiles > 0) {
         bool ok = tc::mbar_wait(&bar[B_QFULL], 0, abort_flag);
-        const uint32_t q_addr = tc::smem_u32(smem + OFF_Q);
         for (int j = 0; j < n_tiles && ok; ++j) {
-          const int s = j % S_BUFS, ks = j % KV_STAGES;
-          if (j >= S_BUFS && !tc::mbar_wait(&bar[B_SEMPTY + s], (j / S_BUFS - 1) & 1, abort_flag)) { ok = false; break; }
-          if (!tc::mbar_wait(&bar[B_KFULL + ks], (j / KV_STAGES) & 1, abort_flag)) { ok = false; break; }
+          const int g = j & 1, ks = j % K_STAGES;
+          if (j >= 2 && !tc::mbar_wait(&bar[B_SEMPTY + g], ((j >> 1) - 1) & 1, abort_flag)) { ok = false; break; }
+          if (!tc::mbar_wait(&bar[B_KFULL + ks], (j / K_STAGES) & 1, abort_flag)) { ok = false; break; }
           tc::fence_after_sync();
           const uint32_t k_addr = tc::smem_u32(smem + OFF_K + ks * TILE);
 #pragma unroll
           for (int k = 0; k < HD / 16; ++k) {
+            // 16 elements of a Q row = 8 packed 32-bit columns
             const uint32_t off = (k >> 2) * SLAB + (k & 3) * 32;
-            tc::mma_f16(tmem_base + COL_S + s * BN, tc::smem_desc_k_sw128(q_addr + off),
-                        tc::smem_desc_k_sw128(k_addr + off), p.idesc_qk, k != 0);
+            tc::mma_f16_ts(tmem_base + COL_S + g * BN, tmem_base + COL_Q + k * 8, tc::smem_desc_k_sw128(k_addr + off),
+                           p.idesc_qk, k != 0);
           }
-          tc::mma_commit(&bar[B_SFULL + s]);
+          tc::mma_commit(&bar[B_SFULL + g]);
           tc::mma_commit(&bar[B_KEMPTY + ks]);
         }
         if (!ok) { *abort_flag = 1; set_status(p.status, AKVS_ERR_TIMEOUT); }
@@ -189,19 +193,18 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
       if (lane == 0 && n_tiles > 0) {
         bool ok = true;
         for (int j = 0; j < n_tiles && ok; ++j) {
-          const int s = j % S_BUFS, vs = j % KV_STAGES;
-          if (!tc::mbar_wait(&bar[B_VFULL + vs], (j / KV_STAGES) & 1, abort_flag)) { ok = false; break; }
-          if (!tc::mbar_wait(&bar[B_PFULL + s], (j / S_BUFS) & 1, abort_flag)) { ok = false; break; }
+          const int vs = j % V_STAGES;
+          if (!tc::mbar_wait(&bar[B_VFULL + vs], (j / V_STAGES) & 1, abort_flag)) { ok = false; break; }
+          if (!tc::mbar_wait(&bar[B_PFULL], j & 1, abort_flag)) { ok = false; break; }
           tc::fence_after_sync();
           const uint32_t v_addr = tc::smem_u32(smem + OFF_V + vs * TILE);
 #pragma unroll
           for (int k = 0; k < BN / 16; ++k) {
-            // 16 keys of P = 8 packed 32-bit columns of the S/P buffer
+            // 16 keys of P = 8 packed 32-bit columns
             const uint64_t db = tc::smem_desc_mn_sw128(v_addr + k * 2048, SLAB);
-            tc::mma_f16_ts(tmem_base, tmem_base + COL_S + s * BN + k * 8, db, p.idesc_pv, (j | k) != 0);
+            tc::mma_f16_ts(tmem_base + COL_O, tmem_base + COL_P + k * 8, db, p.idesc_pv, (j | k) != 0);
           }
-          tc::mma_commit(&bar[B_ODONE + (j & 1)]);
-          tc::mma_commit(&bar[B_SEMPTY + s]);
+          tc::mma_commit(&bar[B_ODONE + (j & 3)]);
           tc::mma_commit(&bar[B_VEMPTY + vs]);
           if (j == n_tiles - 1) tc::mma_commit(&bar[B_OFINAL]);
         }
@@ -223,14 +226,32 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     // select per element (a per-element && / || compiles to divergent branches, measured 2x slower)
     const unsigned span = hi >= lo ? (unsigned)(hi - lo) : 0u;
     const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16);
+    if (grp == 0 && n_tiles > 0) {
+      // Q row of this thread: global -> registers -> tensor memory, 16-bit pairs as they lie in memory
+      const uint4* qp = reinterpret_cast<const uint4*>(reinterpret_cast<const T*>(p.q) +
+                                                       ((size_t)r * p.n_q + (size_t)hk * p.g + head) * HD);
+#pragma unroll
+      for (int c = 0; c < 2; ++c) {
+        uint32_t w[32];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          const uint4 x = valid ? __ldg(qp + c * 8 + i) : make_uint4(0u, 0u, 0u, 0u);
+          w[4 * i] = x.x; w[4 * i + 1] = x.y; w[4 * i + 2] = x.z; w[4 * i + 3] = x.w;
+        }
+        tc::tmem_st32(lane_addr + COL_Q + c * 32, w);
+      }
+      tc::tmem_st_wait();
+      tc::fence_before_sync();
+      __syncwarp();
+      if (lane == 0) tc::mbar_arrive(&bar[B_QFULL]);
+    }
+    const uint32_t s_addr = lane_addr + COL_S + grp * BN;
     float m_mine = -1.0e30f;                        // reference maximum this thread's row sum is scaled to
     float l_mine = 0.f;                             // row sum over this group's tiles
     bool ok = true;
     for (int j = grp; j < n_tiles && ok; j += 2) {
-      const int s = j % S_BUFS;
       const int j0 = key_lo + j * BN;
-      const uint32_t s_addr = lane_addr + COL_S + s * BN;
-      if (!tc::mbar_wait(&bar[B_SFULL + s], (j / S_BUFS) & 1, abort_flag)) { ok = false; break; }
+      if (!tc::mbar_wait(&bar[B_SFULL + grp], (j >> 1) & 1, abort_flag)) { ok = false; break; }
       tc::fence_after_sync();
       float t[BN];
       tc::tmem_ld32(s_addr + 0, *reinterpret_cast<float(*)[32]>(&t[0]));
@@ -238,6 +259,10 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
       tc::tmem_ld32(s_addr + 64, *reinterpret_cast<float(*)[32]>(&t[64]));
       tc::tmem_ld32(s_addr + 96, *reinterpret_cast<float(*)[32]>(&t[96]));
       tc::tmem_ld_wait();
+      // S is in registers: the buffer may take the group's next tile already
+      tc::fence_before_sync();
+      __syncwarp();
+      if (lane == 0) tc::mbar_arrive(&bar[B_SEMPTY + grp]);
       const bool full_tile = lo <= j0 && j0 + BN - 1 <= hi;
       if (!full_tile) {
 #pragma unroll
@@ -266,18 +291,18 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
       m_mine = m_new;
       if (j > 0 && __any_sync(0xffffffffu, raise)) {
         // rows of O accumulated so far move to the new maximum, once P(j-1) V(j-1) has landed
-        if (!tc::mbar_wait(&bar[B_ODONE + ((j - 1) & 1)], ((j - 1) >> 1) & 1, abort_flag)) { ok = false; break; }
+        if (!tc::mbar_wait(&bar[B_ODONE + ((j - 1) & 3)], ((j - 1) >> 2) & 1, abort_flag)) { ok = false; break; }
         tc::fence_after_sync();
         const float f = ex2(m_old - m_new);         // exactly 1 for the rows that keep their maximum
 #pragma unroll 1
         for (int c = 0; c < HD / 32; ++c) {
           float o[32];
-          tc::tmem_ld32(lane_addr + c * 32, o);
+          tc::tmem_ld32(lane_addr + COL_O + c * 32, o);
           tc::tmem_ld_wait();
           uint32_t ob[32];
 #pragma unroll
           for (int i = 0; i < 32; ++i) ob[i] = __float_as_uint(o[i] * f);
-          tc::tmem_st32(lane_addr + c * 32, ob);
+          tc::tmem_st32(lane_addr + COL_O + c * 32, ob);
         }
       }
       float sum4[4] = {0.f, 0.f, 0.f, 0.f};
@@ -287,18 +312,22 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         sum4[i & 3] += t[i];
       }
       l_mine += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
-      // P overwrites the first 64 columns of this S buffer: two 16-bit probabilities per column
-      uint32_t pk[32];
+      // two 16-bit probabilities per 32-bit column, packed before the wait below: only the two
+      // stores stay on the chain P(j-1) ready -> P(j-1) V(j-1) -> P(j) stored
+      uint32_t pk[64];
 #pragma unroll
-      for (int i = 0; i < 32; ++i) pk[i] = pack2<T>(t[2 * i], t[2 * i + 1]);
-      tc::tmem_st32(s_addr, pk);
-#pragma unroll
-      for (int i = 0; i < 32; ++i) pk[i] = pack2<T>(t[64 + 2 * i], t[64 + 2 * i + 1]);
-      tc::tmem_st32(s_addr + 32, pk);
+      for (int i = 0; i < 64; ++i) pk[i] = pack2<T>(t[2 * i], t[2 * i + 1]);
+      // the P buffer is free once P(j-1) V(j-1) has read it
+      if (j > 0) {
+        if (!tc::mbar_wait(&bar[B_ODONE + ((j - 1) & 3)], ((j - 1) >> 2) & 1, abort_flag)) { ok = false; break; }
+        tc::fence_after_sync();
+      }
+      tc::tmem_st32(lane_addr + COL_P, *reinterpret_cast<uint32_t(*)[32]>(&pk[0]));
+      tc::tmem_st32(lane_addr + COL_P + 32, *reinterpret_cast<uint32_t(*)[32]>(&pk[32]));
       tc::tmem_st_wait();
       tc::fence_before_sync();
       __syncwarp();
-      if (lane == 0) tc::mbar_arrive(&bar[B_PFULL + s]);
+      if (lane == 0) tc::mbar_arrive(&bar[B_PFULL]);
     }
     // ---- epilogue: combine the two groups' row sums, normalise, write half of the columns each
     l_part[grp * 128 + m] = l_mine;
@@ -316,8 +345,8 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
       const float inv = l > 0.f ? 1.f / l : 0.f;
       float o[64];
       if (n_tiles > 0) {
-        tc::tmem_ld32(lane_addr + grp * 64, *reinterpret_cast<float(*)[32]>(&o[0]));
-        tc::tmem_ld32(lane_addr + grp * 64 + 32, *reinterpret_cast<float(*)[32]>(&o[32]));
+        tc::tmem_ld32(lane_addr + COL_O + grp * 64, *reinterpret_cast<float(*)[32]>(&o[0]));
+        tc::tmem_ld32(lane_addr + COL_O + grp * 64 + 32, *reinterpret_cast<float(*)[32]>(&o[32]));
         tc::tmem_ld_wait();
       } else {
 #pragma unroll
@@ -364,21 +393,20 @@ int32_t launch_attention_tc(int dtype, const void* q, const void* k, const void*
   p.R = R; p.T = T; p.n_q = n_q; p.n_kv = n_kv;
   p.g = n_q / n_kv;
   p.BR = 128 / p.g;
-  p.k_lo = k_lo; p.k_hi = k_hi; p.out = out; p.status = status;
+  p.q = q; p.k_lo = k_lo; p.k_hi = k_hi; p.out = out; p.status = status;
   p.scale_log2 = 1.4426950408889634f / sqrtf((float)HD);
   const uint32_t fmt = dtype == AKVS_F16 ? tc::kF16 : tc::kBF16;
   p.idesc_qk = tc::idesc_f16(fmt, fmt, 128, BN, 0);
   p.idesc_pv = tc::idesc_f16(fmt, fmt, 128, HD, 1);
-  CUtensorMap tmQ, tmK, tmV;
-  AKVS_TRY(encode_tmap_3d_16bit(&tmQ, q, HD, n_q, R, HD, (uint64_t)n_q * HD, p.g, p.BR));
+  CUtensorMap tmK, tmV;
   AKVS_TRY(encode_tmap_2d_16bit(&tmK, k, T, (uint64_t)n_kv * HD, (uint64_t)n_kv * HD, BN));
   AKVS_TRY(encode_tmap_2d_16bit(&tmV, v, T, (uint64_t)n_kv * HD, (uint64_t)n_kv * HD, BN));
   p.row_blocks = akvs_cdiv(R, p.BR);
   const dim3 grid((unsigned)p.row_blocks * n_kv);
   double flops = 0;   // filled by the caller's accounting when profiling attention
   ProfScope prof(3, 0, flops, st);
-  if (dtype == AKVS_BF16) attention_tc_kernel<bf16><<<grid, ATT_THREADS, ATT_SMEM, st>>>(tmQ, tmK, tmV, p);
-  else attention_tc_kernel<f16><<<grid, ATT_THREADS, ATT_SMEM, st>>>(tmQ, tmK, tmV, p);
+  if (dtype == AKVS_BF16) attention_tc_kernel<bf16><<<grid, ATT_THREADS, ATT_SMEM, st>>>(tmK, tmV, p);
+  else attention_tc_kernel<f16><<<grid, ATT_THREADS, ATT_SMEM, st>>>(tmK, tmV, p);
   AKVS_LAUNCHED();
   return AKVS_OK;
 }
