@@ -98,12 +98,25 @@ typedef struct akvs_cache {
                                 prefill.  Ignored by akvs_encode_units. */
 } akvs_cache;
 
-/* One request: which units, in which order (retrieval order differs per query), and the query. */
+/* One request: which units, in which order (retrieval order differs per query), and the query.
+ *
+ * A batch of requests that share the model (Section 4.4 measures batch sizes 4-16) is one
+ * akvs_request with n_requests > 1: unit_ids and query_ids hold the requests' lists one after
+ * the other and req_unit_off / req_query_off give the boundaries.  Every linear layer then
+ * runs once over the recomputed rows of all requests; attention, offsets and corrections stay
+ * per request (a row only sees its own request's context and query tokens, positions restart
+ * at 0 in every request, offsets are per unit as before).  Token order of every per-token
+ * argument and output (akvs_probes arrays, out_k / out_v rows, out_hidden rows): all context
+ * tokens, request after request, then all query tokens, request after request.  The results of
+ * a request do not depend on the other requests of its batch. */
 typedef struct akvs_request {
-  int32_t n_units;
+  int32_t n_units;           /* total over the batch                                          */
   const int32_t* unit_ids;   /* host   [n_units], indices into the unit store                 */
-  int32_t n_query;
+  int32_t n_query;           /* total over the batch                                          */
   const int32_t* query_ids;  /* device [n_query]                                              */
+  int32_t n_requests;        /* 0 or 1: a single request (the two arrays below are ignored)   */
+  const int32_t* req_unit_off;   /* host [n_requests + 1] boundaries in unit_ids, first 0, last n_units  */
+  const int32_t* req_query_off;  /* host [n_requests + 1] boundaries in query_ids, first 0, last n_query */
 } akvs_request;
 
 /* Probe sets and weights (Section 3.3).  Every array is device memory allocated by the

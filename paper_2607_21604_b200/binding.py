@@ -54,7 +54,8 @@ class CacheDesc(C.Structure):
 
 class RequestDesc(C.Structure):
     _fields_ = [("n_units", C.c_int32), ("unit_ids", C.POINTER(C.c_int32)), ("n_query", C.c_int32),
-                ("query_ids", C.c_void_p)]
+                ("query_ids", C.c_void_p), ("n_requests", C.c_int32), ("req_unit_off", C.POINTER(C.c_int32)),
+                ("req_query_off", C.POINTER(C.c_int32))]
 
 
 class ProbesDesc(C.Structure):
@@ -226,14 +227,35 @@ class Probes:
 
 
 class Request:
-    def __init__(self, unit_ids, query_ids, device="cuda"):
+    """One request (unit ids in retrieval order + query ids) or, with `batch`, several requests
+    that share the model: `Request.batch([(unit_ids, query_ids), ...])`."""
+
+    def __init__(self, unit_ids, query_ids, device="cuda", unit_off=None, query_off=None):
         self.unit_ids = (C.c_int32 * max(1, len(unit_ids)))(*[int(u) for u in unit_ids])
         self.query_ids = torch.as_tensor(query_ids, dtype=torch.int32).to(device).contiguous()
         d = RequestDesc()
         d.n_units, d.n_query = len(unit_ids), int(self.query_ids.numel())
         d.unit_ids = C.cast(self.unit_ids, C.POINTER(C.c_int32))
         d.query_ids = self.query_ids.data_ptr()
+        d.n_requests = 0
+        if unit_off is not None:
+            assert query_off is not None and len(unit_off) == len(query_off) >= 2
+            self.unit_off = (C.c_int32 * len(unit_off))(*[int(x) for x in unit_off])
+            self.query_off = (C.c_int32 * len(query_off))(*[int(x) for x in query_off])
+            d.n_requests = len(unit_off) - 1
+            d.req_unit_off = C.cast(self.unit_off, C.POINTER(C.c_int32))
+            d.req_query_off = C.cast(self.query_off, C.POINTER(C.c_int32))
         self.desc = d
+
+    @classmethod
+    def batch(cls, requests, device="cuda"):
+        units, queries, uo, qo = [], [], [0], [0]
+        for u, q in requests:
+            units += [int(x) for x in u]
+            queries += [int(x) for x in q]
+            uo.append(len(units))
+            qo.append(len(queries))
+        return cls(units, queries, device=device, unit_off=uo, query_off=qo)
 
 
 def workspace_bytes(model, n_ctx, n_query, n_units, check_layer):

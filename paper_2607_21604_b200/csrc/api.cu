@@ -89,6 +89,10 @@ struct Workspace {
   int32_t* pos;             // [T] 0..T-1 (or unit-local positions while encoding)
   int32_t* lo;              // [T] attention lower bounds
   int32_t* zeros;           // [T]
+  int32_t* unit_pos;        // [M+1] batched requests: position of a unit inside its own request
+  int32_t* tok_pos;         // [T]   batched requests: position of a token inside its own request
+  int32_t* tok_rng;         // [4][T] batched requests: visible key ranges (lo1, hi1, lo2, hi2) per token
+  int32_t* row_meta;        // [5][T] the same five arrays gathered for the recomputed rows
   float2* rope;             // [T][hd/2]
   float* mu_k;              // [M][dkv]
   float* mu_v;
@@ -122,6 +126,10 @@ Workspace carve(const Dims& D, int N, int nq, int M, int check_layer, void* base
   w.pos = c.take<int32_t>(T);
   w.lo = c.take<int32_t>(T);
   w.zeros = c.take<int32_t>(T);
+  w.unit_pos = c.take<int32_t>(M + 1);
+  w.tok_pos = c.take<int32_t>(T);
+  w.tok_rng = c.take<int32_t>(4 * T);
+  w.row_meta = c.take<int32_t>(5 * T);
   w.rope = c.take<float2>(T * (D.hd / 2));
   w.mu_k = c.take<float>((int64_t)M * D.dkv);
   w.mu_v = c.take<float>((int64_t)M * D.dkv);
@@ -148,7 +156,7 @@ int32_t check_workspace(const void* ws, int64_t have, int64_t need) {
 
 struct Ctx {                   // host object that carries a request from selection to prefill
   uint32_t magic;
-  int N, nq, M, check_layer, n_probe_total;
+  int N, nq, M, B, check_layer, n_probe_total;
   void* workspace;
 };
 
@@ -204,26 +212,36 @@ int32_t linear_swiglu(const Dims& D, const void* x, int M, int K, const void* wg
 // attn_k/attn_v with per-row key ranges [lo, hi].
 int g_attention_algo = 0;       // 16-bit models with head_dim 128: 0 = tcgen05; 1 = CUDA cores
 
-int32_t attention(const Dims& D, const void* q, const void* k, const void* v, void* out, const int32_t* lo,
-                  const int32_t* hi, int n, int n_keys, int32_t* status, cudaStream_t st) {
+// Per-row geometry of a set of rows: RoPE position and visible key ranges.  lo2/hi2 are null
+// for a single request (one contiguous causal range per row).
+struct RowGeom {
+  const int32_t* pos;
+  const int32_t* lo;
+  const int32_t* hi;
+  const int32_t* lo2;
+  const int32_t* hi2;
+};
+
+int32_t attention(const Dims& D, const void* q, const void* k, const void* v, void* out, const RowGeom& g, int n,
+                  int n_keys, int32_t* status, cudaStream_t st) {
   if (D.dtype != AKVS_F32 && D.hd == 128 && g_attention_algo == 0)
-    return launch_attention_tc(D.dtype, q, k, v, out, lo, hi, n, n_keys, D.nq, D.nkv, status, st);
-  return launch_attention_simt(D.dtype, q, k, v, out, lo, hi, n, D.nq, D.nkv, D.hd, st);
+    return launch_attention_tc(D.dtype, q, k, v, out, g.lo, g.hi, g.lo2, g.hi2, n, n_keys, D.nq, D.nkv, status, st);
+  return launch_attention_simt(D.dtype, q, k, v, out, g.lo, g.hi, g.lo2, g.hi2, n, D.nq, D.nkv, D.hd, st);
 }
 
-int32_t run_layer(const akvs_model_desc* m, const Dims& D, int l, const Workspace& ws, int n, const int32_t* pos,
-                  const int32_t* lo, const int32_t* hi, void* k_dst, void* v_dst, const void* attn_k,
-                  const void* attn_v, int n_keys, const std::function<int32_t()>& between, cudaStream_t st) {
+int32_t run_layer(const akvs_model_desc* m, const Dims& D, int l, const Workspace& ws, int n, const RowGeom& g,
+                  void* k_dst, void* v_dst, const void* attn_k, const void* attn_v, int n_keys,
+                  const std::function<int32_t()>& between, cudaStream_t st) {
   if (n == 0) return between ? between() : AKVS_OK;
   AKVS_TRY(launch_rmsnorm(D.dtype, ws.h, m->attn_norm[l], m->rms_eps, n, D.d, ws.x, st));
   {
     const void* w[3] = {m->wq[l], m->wk[l], m->wv[l]};
     const int ns[3] = {D.dq, D.dkv, D.dkv};
     void* out[3] = {ws.q, k_dst, v_dst};
-    AKVS_TRY(linear_multi(D, ws.x, n, D.d, 3, w, ns, out, ns, ws.status, st, ws.rope, pos, 0b011, m->rope_base));
+    AKVS_TRY(linear_multi(D, ws.x, n, D.d, 3, w, ns, out, ns, ws.status, st, ws.rope, g.pos, 0b011, m->rope_base));
   }
   if (between) AKVS_TRY(between());
-  AKVS_TRY(attention(D, ws.q, attn_k, attn_v, ws.ao, lo, hi, n, n_keys, ws.status, st));
+  AKVS_TRY(attention(D, ws.q, attn_k, attn_v, ws.ao, g, n, n_keys, ws.status, st));
   AKVS_TRY(linear_resid(D, ws.ao, n, D.dq, m->wo[l], D.d, ws.h, ws.status, st));
   AKVS_TRY(launch_rmsnorm(D.dtype, ws.h, m->mlp_norm[l], m->rms_eps, n, D.d, ws.x, st));
   AKVS_TRY(linear_swiglu(D, ws.x, n, D.d, m->w_gate[l], m->w_up[l], D.f, ws.act, ws.status, st));
@@ -274,6 +292,37 @@ int32_t check_cache(const akvs_cache* c, const Dims& D, bool need_kv) {
   return AKVS_OK;
 }
 
+// Boundaries of the requests of a batch in the merged token order (all context tokens, request
+// after request, then all query tokens, request after request).  B == 1: a single request.
+struct Batch {
+  int B = 1;
+  std::vector<int32_t> unit_off;    // [B+1] into the unit list
+  std::vector<int32_t> ctx_start;   // [B+1] into the context tokens
+  std::vector<int32_t> qry_start;   // [B+1] into the query tokens
+};
+
+int32_t check_batch(const akvs_request* r, const std::vector<int32_t>& ctx_off, Batch& b) {
+  b.B = r->n_requests > 1 ? r->n_requests : 1;
+  if (r->n_requests < 0) return AKVS_ERR_INVALID_ARG;
+  if (b.B == 1) {
+    b.unit_off = {0, r->n_units};
+    b.ctx_start = {0, ctx_off[r->n_units]};
+    b.qry_start = {0, r->n_query};
+    return AKVS_OK;
+  }
+  if (!r->req_unit_off || !r->req_query_off) return AKVS_ERR_INVALID_ARG;
+  if (r->req_unit_off[0] != 0 || r->req_unit_off[b.B] != r->n_units) return AKVS_ERR_SHAPE;
+  if (r->req_query_off[0] != 0 || r->req_query_off[b.B] != r->n_query) return AKVS_ERR_SHAPE;
+  b.unit_off.assign(r->req_unit_off, r->req_unit_off + b.B + 1);
+  b.qry_start.assign(r->req_query_off, r->req_query_off + b.B + 1);
+  b.ctx_start.assign(b.B + 1, 0);
+  for (int i = 0; i < b.B; ++i) {
+    if (b.unit_off[i + 1] < b.unit_off[i] || b.qry_start[i + 1] < b.qry_start[i]) return AKVS_ERR_SHAPE;
+    b.ctx_start[i + 1] = ctx_off[b.unit_off[i + 1]];
+  }
+  return AKVS_OK;
+}
+
 int32_t check_request(const akvs_request* r, const akvs_cache* c, std::vector<int32_t>& ctx_off,
                       std::vector<int32_t>& slot_src) {
   if (!r || r->n_units < 0 || r->n_query < 0) return AKVS_ERR_INVALID_ARG;
@@ -300,6 +349,66 @@ __global__ void local_pos_kernel(const int32_t* __restrict__ ctx_off, const int3
 }
 
 // Uploads the request's offsets and builds the maps every mode needs.
+__global__ void gather_i32_kernel(const int32_t* __restrict__ src, const int32_t* __restrict__ idx, int n, int stride_src,
+                                  int stride_dst, int n_arrays, int32_t* __restrict__ dst) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n) return;
+  const int j = idx[i];
+  for (int a = 0; a < n_arrays; ++a) dst[(size_t)a * stride_dst + i] = src[(size_t)a * stride_src + j];
+}
+
+// Batched requests: per-token position inside the token's own request and the key ranges it
+// sees in the merged order.  Context token j of request b sees [ctx_start_b, j]; query token
+// t = N + i of request b sees its whole context [ctx_start_b, ctx_start_{b+1}) and the query
+// tokens [N + qry_start_b, t].  tok_pos and the four range arrays are contiguous (5 x T).
+int32_t setup_batch(const Workspace& ws, const std::vector<int32_t>& ctx_off, const Batch& b, int M, int N, int nq,
+                    cudaStream_t st) {
+  const int T = N + nq;
+  std::vector<int32_t> unit_pos(M + 1, 0), arr((size_t)5 * T);
+  int32_t* pos = arr.data();
+  int32_t* lo1 = pos + T;
+  int32_t* hi1 = lo1 + T;
+  int32_t* lo2 = hi1 + T;
+  int32_t* hi2 = lo2 + T;
+  for (int r = 0; r < b.B; ++r) {
+    const int cs = b.ctx_start[r], ce = b.ctx_start[r + 1], qs = b.qry_start[r], qe = b.qry_start[r + 1];
+    for (int u = b.unit_off[r]; u < b.unit_off[r + 1]; ++u) unit_pos[u] = ctx_off[u] - cs;
+    for (int j = cs; j < ce; ++j) { pos[j] = j - cs; lo1[j] = cs; hi1[j] = j; lo2[j] = 1; hi2[j] = 0; }
+    for (int i = qs; i < qe; ++i) {
+      const int t = N + i;
+      pos[t] = (ce - cs) + (i - qs); lo1[t] = cs; hi1[t] = ce - 1; lo2[t] = N + qs; hi2[t] = t;
+    }
+  }
+  AKVS_CUDA(cudaMemcpyAsync(ws.unit_pos, unit_pos.data(), (M + 1) * sizeof(int32_t), cudaMemcpyHostToDevice, st));
+  if (T > 0) {
+    AKVS_CUDA(cudaMemcpyAsync(ws.tok_pos, pos, (size_t)T * sizeof(int32_t), cudaMemcpyHostToDevice, st));
+    AKVS_CUDA(cudaMemcpyAsync(ws.tok_rng, lo1, (size_t)4 * T * sizeof(int32_t), cudaMemcpyHostToDevice, st));
+    // the vectors die with this frame: pageable copies are staged before the call returns, but do not rely on it
+    AKVS_CUDA(cudaStreamSynchronize(st));
+  }
+  return AKVS_OK;
+}
+
+// Geometry of all T tokens taken as rows (dense layers, full recompute).
+RowGeom token_geom(const Workspace& ws, const Batch& b, int T) {
+  if (b.B == 1) return RowGeom{ws.pos, ws.zeros, ws.pos, nullptr, nullptr};
+  return RowGeom{ws.tok_pos, ws.tok_rng, ws.tok_rng + T, ws.tok_rng + 2 * (size_t)T, ws.tok_rng + 3 * (size_t)T};
+}
+
+// Geometry of the recomputed rows `rows[0..R)` (merged token indices, device).
+int32_t row_geom(const Workspace& ws, const Batch& b, const int32_t* rows, int R, int T, RowGeom& g, cudaStream_t st) {
+  if (b.B == 1) { g = RowGeom{rows, ws.zeros, rows, nullptr, nullptr}; return AKVS_OK; }
+  if (R > 0) {
+    gather_i32_kernel<<<akvs_cdiv(R, 256), 256, 0, st>>>(ws.tok_pos, rows, R, 0, 0, 1, ws.row_meta);
+    AKVS_LAUNCHED();
+    gather_i32_kernel<<<akvs_cdiv(R, 256), 256, 0, st>>>(ws.tok_rng, rows, R, T, T, 4, ws.row_meta + T);
+    AKVS_LAUNCHED();
+  }
+  g = RowGeom{ws.row_meta, ws.row_meta + T, ws.row_meta + 2 * (size_t)T, ws.row_meta + 3 * (size_t)T,
+              ws.row_meta + 4 * (size_t)T};
+  return AKVS_OK;
+}
+
 int32_t setup_request(const Dims& D, const Workspace& ws, const std::vector<int32_t>& ctx_off,
                       const std::vector<int32_t>& slot_src, int M, int N, int nq, cudaStream_t st) {
   const int T = N + nq;
@@ -312,9 +421,10 @@ int32_t setup_request(const Dims& D, const Workspace& ws, const std::vector<int3
   return AKVS_OK;
 }
 
-ReqMaps req_maps(const Workspace& ws, int N) {
+ReqMaps req_maps(const Workspace& ws, int N, bool batched = false) {
   ReqMaps mp;
   mp.ctx_off = ws.ctx_off;
+  mp.unit_pos = batched ? ws.unit_pos : ws.ctx_off;
   mp.tok_unit = ws.tok_unit;
   mp.tok_src = ws.tok_src;
   mp.row_of_pos = ws.row_of_pos;
@@ -424,7 +534,8 @@ int32_t akvs_encode_units(const akvs_model_desc* model, akvs_cache* cache, void*
                                reinterpret_cast<char*>(cache->v) + l * lstride,
                                reinterpret_cast<char*>(cache->v_meta) + l * mstride, st);
       };
-    AKVS_TRY(run_layer(model, D, l, ws, N, local_pos, ws.lo, ws.pos, k_dst, v_dst, k_dst, v_dst, N, store, st));
+    AKVS_TRY(run_layer(model, D, l, ws, N, RowGeom{local_pos, ws.lo, ws.pos, nullptr, nullptr}, k_dst, v_dst, k_dst,
+                       v_dst, N, store, st));
   }
   return AKVS_OK;
 }
@@ -442,6 +553,8 @@ int32_t akvs_select_probes(const akvs_model_desc* model, const akvs_cache* cache
     return AKVS_ERR_INVALID_ARG;
   std::vector<int32_t> ctx_off, slot_src;
   AKVS_TRY(check_request(req, cache, ctx_off, slot_src));
+  Batch batch;
+  AKVS_TRY(check_batch(req, ctx_off, batch));
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
   const int M = req->n_units, N = ctx_off[M], nq = req->n_query, T = N + nq;
   Workspace ws = carve(D, N, nq, M, check_layer, workspace);
@@ -456,6 +569,8 @@ int32_t akvs_select_probes(const akvs_model_desc* model, const akvs_cache* cache
     probe_off[u + 1] = probe_off[u] + (int32_t)b;
   }
   AKVS_TRY(setup_request(D, ws, ctx_off, slot_src, M, N, nq, st));
+  if (batch.B > 1) AKVS_TRY(setup_batch(ws, ctx_off, batch, M, N, nq, st));
+  const RowGeom all_tokens = token_geom(ws, batch, T);
   AKVS_CUDA(cudaMemcpyAsync(ws.probe_off, probe_off.data(), (M + 1) * sizeof(int32_t), cudaMemcpyHostToDevice, st));
   AKVS_CUDA(cudaMemcpyAsync(out->ctx_off, ctx_off.data(), (M + 1) * sizeof(int32_t), cudaMemcpyHostToDevice, st));
   AKVS_CUDA(cudaMemcpyAsync(out->probe_off, probe_off.data(), (M + 1) * sizeof(int32_t), cudaMemcpyHostToDevice, st));
@@ -467,7 +582,7 @@ int32_t akvs_select_probes(const akvs_model_desc* model, const akvs_cache* cache
   for (int l = 0; l < check_layer - 1; ++l) {
     void* kd = reinterpret_cast<char*>(ws.stash_k) + l * kv_l;
     void* vd = reinterpret_cast<char*>(ws.stash_v) + l * kv_l;
-    AKVS_TRY(run_layer(model, D, l, ws, T, ws.pos, ws.zeros, ws.pos, kd, vd, kd, vd, T, nullptr, st));
+    AKVS_TRY(run_layer(model, D, l, ws, T, all_tokens, kd, vd, kd, vd, T, nullptr, st));
   }
   if (T > 0)
     AKVS_CUDA(cudaMemcpyAsync(ws.stash_h, ws.h, (size_t)T * D.d * sizeof(float), cudaMemcpyDeviceToDevice, st));
@@ -479,9 +594,10 @@ int32_t akvs_select_probes(const akvs_model_desc* model, const akvs_cache* cache
     const void* w[2] = {model->wk[lc], model->wv[lc]};
     const int ns[2] = {D.dkv, D.dkv};
     void* o[2] = {ws.k, ws.v};
-    AKVS_TRY(linear_multi(D, ws.x, N, D.d, 2, w, ns, o, ns, ws.status, st, ws.rope, ws.pos, 0b01, model->rope_base));
+    AKVS_TRY(linear_multi(D, ws.x, N, D.d, 2, w, ns, o, ns, ws.status, st, ws.rope, all_tokens.pos, 0b01,
+                          model->rope_base));
     AKVS_TRY(wait_layer(cache, lc, st));
-    AKVS_TRY(launch_scores(D.dtype, cache_layer(cache, D, lc), req_maps(ws, N), ws.k, ws.v, N, D.nkv, D.hd, ws.rope,
+    AKVS_TRY(launch_scores(D.dtype, cache_layer(cache, D, lc), req_maps(ws, N, batch.B > 1), ws.k, ws.v, N, D.nkv, D.hd, ws.rope,
                            out->d_k, out->d_v, st));
   }
   AKVS_TRY(launch_select(out->d_k, out->d_v, ws.ctx_off, ws.probe_off, M, N, nq, out->sk_idx, out->sv_idx, out->w_k,
@@ -501,7 +617,7 @@ int32_t akvs_select_probes(const akvs_model_desc* model, const akvs_cache* cache
     *ctx_inout = ctx;
   }
   ctx->magic = kCtxMagic;
-  ctx->N = N; ctx->nq = nq; ctx->M = M; ctx->check_layer = check_layer;
+  ctx->N = N; ctx->nq = nq; ctx->M = M; ctx->B = batch.B; ctx->check_layer = check_layer;
   ctx->n_probe_total = probe_off[M];
   ctx->workspace = workspace;
   return AKVS_OK;
@@ -517,6 +633,8 @@ int32_t akvs_prefill_corrected(const akvs_model_desc* model, const akvs_cache* c
   if (!out_hidden || !out_k || !out_v) return AKVS_ERR_INVALID_ARG;
   std::vector<int32_t> ctx_off, slot_src;
   AKVS_TRY(check_request(req, cache, ctx_off, slot_src));
+  Batch batch;
+  AKVS_TRY(check_batch(req, ctx_off, batch));
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
   const int M = req->n_units, N = ctx_off[M], nq = req->n_query, T = N + nq;
   const size_t kv_l = (size_t)T * D.dkv * D.es;
@@ -527,11 +645,13 @@ int32_t akvs_prefill_corrected(const akvs_model_desc* model, const akvs_cache* c
     Workspace ws = carve(D, N, nq, M, 1, workspace);
     AKVS_TRY(check_workspace(workspace, ws_bytes, ws.bytes));
     AKVS_TRY(setup_request(D, ws, ctx_off, slot_src, M, N, nq, st));
+    if (batch.B > 1) AKVS_TRY(setup_batch(ws, ctx_off, batch, M, N, nq, st));
     AKVS_TRY(launch_rope_table(model->rope_base, D.hd, T, ws.rope, st));
     AKVS_TRY(embed_all(model, D, cache, req, ws, N, st));
+    const RowGeom all_tokens = token_geom(ws, batch, T);
     for (int l = 0; l < D.L; ++l)
-      AKVS_TRY(run_layer(model, D, l, ws, T, ws.pos, ws.zeros, ws.pos, ok + l * kv_l, ov + l * kv_l, ok + l * kv_l,
-                         ov + l * kv_l, T, nullptr, st));
+      AKVS_TRY(run_layer(model, D, l, ws, T, all_tokens, ok + l * kv_l, ov + l * kv_l, ok + l * kv_l, ov + l * kv_l, T,
+                         nullptr, st));
     return launch_rmsnorm(AKVS_F32, ws.h + (size_t)N * D.d, model->final_norm, model->rms_eps, nq, D.d, out_hidden, st);
   }
 
@@ -542,6 +662,7 @@ int32_t akvs_prefill_corrected(const akvs_model_desc* model, const akvs_cache* c
     ws = carve(D, N, nq, M, 1, workspace);
     AKVS_TRY(check_workspace(workspace, ws_bytes, ws.bytes));
     AKVS_TRY(setup_request(D, ws, ctx_off, slot_src, M, N, nq, st));
+    if (batch.B > 1) AKVS_TRY(setup_batch(ws, ctx_off, batch, M, N, nq, st));
     AKVS_TRY(launch_rope_table(model->rope_base, D.hd, T, ws.rope, st));
     rows = ws.pos + N;                                   // the query positions N..T-1
     AKVS_TRY(launch_row_maps(rows, nq, nullptr, nullptr, 0, N, T, ws.row_of_pos, ws.flags, ws.flags + N, st));
@@ -550,7 +671,8 @@ int32_t akvs_prefill_corrected(const akvs_model_desc* model, const akvs_cache* c
   } else {
     const Ctx* ctx = reinterpret_cast<const Ctx*>(ctx_v);
     if (!ctx || ctx->magic != kCtxMagic || !probes) return AKVS_ERR_INVALID_ARG;
-    if (ctx->N != N || ctx->nq != nq || ctx->M != M || ctx->workspace != workspace) return AKVS_ERR_SHAPE;
+    if (ctx->N != N || ctx->nq != nq || ctx->M != M || ctx->B != batch.B || ctx->workspace != workspace)
+      return AKVS_ERR_SHAPE;
     if (probes->n_ctx != N || probes->n_probe_rows < 0 || probes->n_probe_rows > N ||
         probes->n_rows != probes->n_probe_rows + nq)
       return AKVS_ERR_SHAPE;
@@ -574,7 +696,9 @@ int32_t akvs_prefill_corrected(const akvs_model_desc* model, const akvs_cache* c
     AKVS_TRY(launch_gather_rows(ws.stash_h, rows, R, D.d, ws.h, st));
   }
 
-  const ReqMaps maps = req_maps(ws, N);
+  const ReqMaps maps = req_maps(ws, N, batch.B > 1);
+  RowGeom geom;
+  AKVS_TRY(row_geom(ws, batch, rows, R, T, geom, st));
   const bool corrected = mode == AKVS_MODE_CORRECTED;
   for (int l = first_layer; l < D.L; ++l) {
     const KvLayer kv = cache_layer(cache, D, l);
@@ -587,8 +711,7 @@ int32_t akvs_prefill_corrected(const akvs_model_desc* model, const akvs_cache* c
                             corrected ? probes->w_v : nullptr, ws.mu_k, ws.mu_v, N, nq, P, D.nkv, D.hd, ws.rope,
                             ok + l * kv_l, ov + l * kv_l, st);
     };
-    AKVS_TRY(run_layer(model, D, l, ws, R, rows, ws.zeros, rows, ws.k, ws.v, ok + l * kv_l, ov + l * kv_l, T,
-                       assemble, st));
+    AKVS_TRY(run_layer(model, D, l, ws, R, geom, ws.k, ws.v, ok + l * kv_l, ov + l * kv_l, T, assemble, st));
   }
   return launch_rmsnorm(AKVS_F32, ws.h + (size_t)P * D.d, model->final_norm, model->rms_eps, nq, D.d, out_hidden, st);
 }
@@ -641,8 +764,8 @@ int32_t akvs_op_attention(int32_t dtype, const void* q, const void* k, const voi
   if (dtype != AKVS_F32 && dtype != AKVS_BF16 && dtype != AKVS_F16) return AKVS_ERR_UNSUPPORTED;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
   if (dtype != AKVS_F32 && head_dim == 128 && algo == 0)
-    return launch_attention_tc(dtype, q, k, v, out, k_lo, k_hi, R, T, n_q_heads, n_kv_heads, nullptr, st);
-  return launch_attention_simt(dtype, q, k, v, out, k_lo, k_hi, R, n_q_heads, n_kv_heads, head_dim, st);
+    return launch_attention_tc(dtype, q, k, v, out, k_lo, k_hi, nullptr, nullptr, R, T, n_q_heads, n_kv_heads, nullptr, st);
+  return launch_attention_simt(dtype, q, k, v, out, k_lo, k_hi, nullptr, nullptr, R, n_q_heads, n_kv_heads, head_dim, st);
 }
 
 int64_t akvs_op_scratch_bytes(int32_t n_ctx, int32_t n_query, int32_t n_units, int32_t head_dim) {
@@ -721,7 +844,7 @@ int32_t akvs_op_correct_layer(int32_t dtype, int32_t kv_format, const void* cach
   AKVS_TRY(launch_rope_table(rope_base, head_dim, T, table, st));
   AKVS_TRY(launch_tok_meta(tok_unit, src_tok, row_of_pos, flags, flags + N, N, T, probes->n_probe_rows, tok_meta, st));
   KvLayer kv{cache_k, cache_v, k_meta, v_meta, kv_format};
-  ReqMaps maps{probes->ctx_off, tok_unit, src_tok, row_of_pos, flags, flags + N, tok_meta};
+  ReqMaps maps{probes->ctx_off, probes->ctx_off, tok_unit, src_tok, row_of_pos, flags, flags + N, tok_meta};
   AKVS_TRY(launch_offsets(dtype, kv, maps, probes->probe_off, probes->sk_idx, probes->sv_idx, fresh_k, fresh_v, M,
                           n_kv_heads, head_dim, table, mu_k, mu_v, st));
   return launch_correct(dtype, kv, maps, fresh_k, fresh_v, probes->w_k, probes->w_v, mu_k, mu_v, N, n_query,

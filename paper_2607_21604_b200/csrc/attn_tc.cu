@@ -32,6 +32,10 @@
 // are not ordered: every reuse of a tensor-memory buffer goes through an mbarrier).
 // Row blocks are taken longest first across all kv heads (the last rows see the most keys).
 // Query row r sees keys k_lo[r] <= j <= k_hi[r]; both arrays are non-decreasing in r.
+// With second-range arrays (batched requests: a query row sees its own context and, not
+// adjacent to it, its own query tokens) a row also sees k_lo2[r] <= j <= k_hi2[r]; the key
+// tiles of a CTA then walk the hull of its rows' first ranges and after it the hull of the
+// second ranges, each tile masked with the range of its segment.
 #include "tc_common.cuh"
 
 namespace {
@@ -56,6 +60,8 @@ struct AttnParams {
   const void* q;
   const int32_t* k_lo;
   const int32_t* k_hi;
+  const int32_t* k_lo2;        // second visible range per row, or null
+  const int32_t* k_hi2;
   void* out;
   float scale_log2;            // log2(e) / sqrt(head_dim)
   uint32_t idesc_qk, idesc_pv;
@@ -101,9 +107,26 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
   const int hk = blockIdx.x % p.n_kv;
   const int r0 = (p.row_blocks - 1 - blockIdx.x / p.n_kv) * p.BR;
   const int n_rows = min(p.BR, p.R - r0);
-  const int key_lo = p.k_lo[r0];
-  const int key_hi = p.k_hi[r0 + n_rows - 1];
-  const int n_tiles = key_hi >= key_lo ? (key_hi - key_lo) / BN + 1 : 0;
+  int key_lo = p.k_lo[r0];
+  int key_hi = p.k_hi[r0 + n_rows - 1];
+  int key_lo2 = 1, key_hi2 = 0;
+  if (p.k_lo2) {
+    // two ranges per row: neither is monotone across the rows of a block, take the hulls
+    int a = 0x7fffffff, b = -1, c = 0x7fffffff, d = -1;
+    for (int i = lane; i < n_rows; i += 32) {
+      const int l1 = p.k_lo[r0 + i], h1 = p.k_hi[r0 + i], l2 = p.k_lo2[r0 + i], h2 = p.k_hi2[r0 + i];
+      if (l1 <= h1) { a = min(a, l1); b = max(b, h1); }
+      if (l2 <= h2) { c = min(c, l2); d = max(d, h2); }
+    }
+    key_lo = __reduce_min_sync(0xffffffffu, a);
+    key_hi = __reduce_max_sync(0xffffffffu, b);
+    key_lo2 = __reduce_min_sync(0xffffffffu, c);
+    key_hi2 = __reduce_max_sync(0xffffffffu, d);
+  }
+  const int n_tiles1 = key_hi >= key_lo ? (key_hi - key_lo) / BN + 1 : 0;
+  const int n_tiles = n_tiles1 + (key_hi2 >= key_lo2 ? (key_hi2 - key_lo2) / BN + 1 : 0);
+  // first key of tile j
+  auto tile_key = [&](int j) { return j < n_tiles1 ? key_lo + j * BN : key_lo2 + (j - n_tiles1) * BN; };
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < B_COUNT; ++i) {
@@ -139,7 +162,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         for (int j = 0; j < n_tiles && ok; ++j) {
           const int s = j % K_STAGES;
           const uint32_t ph = ((j / K_STAGES) & 1) ^ 1;
-          const int y = key_lo + j * BN;
+          const int y = tile_key(j);
           if (!tc::mbar_wait(&bar[B_KEMPTY + s], ph, abort_flag)) { ok = false; break; }
           tc::mbar_expect_tx(&bar[B_KFULL + s], TILE);
           tc::tma_load_2d(smem + OFF_K + s * TILE, &tmK, hk * HD, y, &bar[B_KFULL + s]);
@@ -155,7 +178,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         for (int j = 0; j < n_tiles && ok; ++j) {
           const int s = j % V_STAGES;
           const uint32_t ph = ((j / V_STAGES) & 1) ^ 1;
-          const int y = key_lo + j * BN;
+          const int y = tile_key(j);
           if (!tc::mbar_wait(&bar[B_VEMPTY + s], ph, abort_flag)) { ok = false; break; }
           tc::mbar_expect_tx(&bar[B_VFULL + s], TILE);
           tc::tma_load_2d(smem + OFF_V + s * TILE, &tmV, hk * HD, y, &bar[B_VFULL + s]);
@@ -220,11 +243,14 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
     const int r_local = m / p.g, head = m - r_local * p.g;
     const int r = r0 + r_local;
     const bool valid = r_local < p.BR && r < p.R;
-    const int hi = valid ? p.k_hi[r] : -1;
-    const int lo = valid && p.k_lo[r] <= hi ? p.k_lo[r] : 0x40000000;   // nothing visible: no key reaches lo
+    const int hi1 = valid ? p.k_hi[r] : -1;
+    const int lo1 = valid && p.k_lo[r] <= hi1 ? p.k_lo[r] : 0x40000000;   // nothing visible: no key reaches lo
+    const int hi2 = valid && p.k_lo2 ? p.k_hi2[r] : -1;
+    const int lo2 = valid && p.k_lo2 && p.k_lo2[r] <= hi2 ? p.k_lo2[r] : 0x40000000;
     // key visible  <=>  lo <= key <= hi  <=>  (unsigned)(key - lo) <= hi - lo: one compare and a
     // select per element (a per-element && / || compiles to divergent branches, measured 2x slower)
-    const unsigned span = hi >= lo ? (unsigned)(hi - lo) : 0u;
+    const unsigned span1 = hi1 >= lo1 ? (unsigned)(hi1 - lo1) : 0u;
+    const unsigned span2 = hi2 >= lo2 ? (unsigned)(hi2 - lo2) : 0u;
     const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16);
     if (grp == 0 && n_tiles > 0) {
       // Q row of this thread: global -> registers -> tensor memory, 16-bit pairs as they lie in memory
@@ -250,7 +276,10 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
     float l_mine = 0.f;                             // row sum over this group's tiles
     bool ok = true;
     for (int j = grp; j < n_tiles && ok; j += 2) {
-      const int j0 = key_lo + j * BN;
+      const int j0 = tile_key(j);
+      const bool seg2 = j >= n_tiles1;              // the tile belongs to the second ranges
+      const int lo = seg2 ? lo2 : lo1, hi = seg2 ? hi2 : hi1;
+      const unsigned span = seg2 ? span2 : span1;
       if (!tc::mbar_wait(&bar[B_SFULL + grp], (j >> 1) & 1, abort_flag)) { ok = false; break; }
       tc::fence_after_sync();
       float t[BN];
@@ -379,7 +408,8 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
 
 // q [R][n_q][128], k/v [T][n_kv][128], out [R][n_q][128], all of the 16-bit type `dtype`.
 int32_t launch_attention_tc(int dtype, const void* q, const void* k, const void* v, void* out, const int32_t* k_lo,
-                            const int32_t* k_hi, int R, int T, int n_q, int n_kv, int32_t* status, cudaStream_t st) {
+                            const int32_t* k_hi, const int32_t* k_lo2, const int32_t* k_hi2, int R, int T, int n_q,
+                            int n_kv, int32_t* status, cudaStream_t st) {
   if (R == 0) return AKVS_OK;
   if (dtype != AKVS_BF16 && dtype != AKVS_F16) return AKVS_ERR_UNSUPPORTED;
   if (n_kv <= 0 || n_q % n_kv != 0 || n_q / n_kv > 128 || T <= 0) return AKVS_ERR_SHAPE;
@@ -393,7 +423,7 @@ int32_t launch_attention_tc(int dtype, const void* q, const void* k, const void*
   p.R = R; p.T = T; p.n_q = n_q; p.n_kv = n_kv;
   p.g = n_q / n_kv;
   p.BR = 128 / p.g;
-  p.q = q; p.k_lo = k_lo; p.k_hi = k_hi; p.out = out; p.status = status;
+  p.q = q; p.k_lo = k_lo; p.k_hi = k_hi; p.k_lo2 = k_lo2; p.k_hi2 = k_lo2 ? k_hi2 : nullptr; p.out = out; p.status = status;
   p.scale_log2 = 1.4426950408889634f / sqrtf((float)HD);
   const uint32_t fmt = dtype == AKVS_F16 ? tc::kF16 : tc::kBF16;
   p.idesc_qk = tc::idesc_f16(fmt, fmt, 128, BN, 0);

@@ -182,6 +182,7 @@ struct KvLayer {            // one layer of a unit store, as the correction kern
 
 struct ReqMaps {            // per-request index maps (device)
   const int32_t* ctx_off;   // [M+1]
+  const int32_t* unit_pos;  // [M] position of a unit's first token within its own request (= ctx_off for one request)
   const int32_t* tok_unit;  // [N] unit slot of context token j
   const int32_t* tok_src;   // [N] row of token j in the unit store
   const int32_t* row_of_pos;// [T] index into the recomputed rows, or -1
@@ -215,11 +216,11 @@ int32_t launch_linear_tc(int dtype, int epi, const void* x, int M, int K, int n_
 
 // tcgen05 attention (attn_tc.cu): 16-bit types, head_dim 128.
 int32_t launch_attention_tc(int dtype, const void* q, const void* k, const void* v, void* out, const int32_t* k_lo,
-                            const int32_t* k_hi, int R, int T, int n_q, int n_kv, int32_t* status, cudaStream_t st);
-
+                            const int32_t* k_hi, const int32_t* k_lo2, const int32_t* k_hi2, int R, int T, int n_q,
+                            int n_kv, int32_t* status, cudaStream_t st);
 int32_t launch_attention_simt(int dtype, const void* q, const void* k, const void* v, void* out,
-                              const int32_t* k_lo, const int32_t* k_hi, int R, int n_q, int n_kv, int hd,
-                              cudaStream_t st);
+                              const int32_t* k_lo, const int32_t* k_hi, const int32_t* k_lo2, const int32_t* k_hi2,
+                              int R, int n_q, int n_kv, int hd, cudaStream_t st);
 
 int32_t launch_tok_maps(const int32_t* ctx_off, const int32_t* slot_src_off, int M, int N, int32_t* tok_unit,
                         int32_t* tok_src, cudaStream_t st);

@@ -137,7 +137,7 @@ __global__ void scores_kernel(KvLayer kv, ReqMaps maps, const T* __restrict__ k_
   const int half = hd / 2, ch = half / V;
   const int u = maps.tok_unit[j];
   const int64_t src = maps.tok_src[j];
-  const float2* rot = table + (size_t)maps.ctx_off[u] * half;
+  const float2* rot = table + (size_t)maps.unit_pos[u] * half;
   float sk = 0.f, sv = 0.f;
   for (int pc = lane; pc < n_kv * ch; pc += 32) {
     const int h = pc / ch, c = pc % ch;
@@ -341,7 +341,7 @@ offsets_kernel(KvLayer kv, ReqMaps maps, const int32_t* __restrict__ probe_off, 
   const int half = hd / 2;
   const int p0 = probe_off[u], b = probe_off[u + 1] - p0;
   const int32_t* S = (is_v ? sv_idx : sk_idx) + p0;
-  const float2* rot = table + (size_t)maps.ctx_off[u] * half;
+  const float2* rot = table + (size_t)maps.unit_pos[u] * half;
   const T* fresh = is_v ? v_fresh : k_fresh;
   const void* cbase = is_v ? kv.v : kv.k;
   const void* cmeta = is_v ? kv.v_meta : kv.k_meta;
@@ -549,7 +549,7 @@ correct_kernel(KvLayer kv, ReqMaps maps, const T* __restrict__ k_fresh, const T*
       const int u = meta[t].w;
       if ((!kf || !vf) && u != cur_unit) {
         cur_unit = u;
-        ld_f2<V>(table + (size_t)maps.ctx_off[u] * half + c * V, rot);
+        ld_f2<V>(table + (size_t)maps.unit_pos[u] * half + c * V, rot);
         if (weighted) {
           const float* mk = mu_k + ((size_t)u * n_kv + h) * hd + c * V;
           const float* mv = mu_v + ((size_t)u * n_kv + h) * hd + c * V;

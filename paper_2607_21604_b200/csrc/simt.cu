@@ -87,7 +87,8 @@ constexpr int SA_ROWS = 16, SA_KEYS = 32, SA_RPW = 4;   // rows per CTA, keys pe
 template <typename T, int HD>
 __global__ void __launch_bounds__(128)
 attention_simt_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __restrict__ v, T* __restrict__ out,
-                      const int32_t* __restrict__ k_lo, const int32_t* __restrict__ k_hi, int R, int n_q, int n_kv) {
+                      const int32_t* __restrict__ k_lo, const int32_t* __restrict__ k_hi,
+                      const int32_t* __restrict__ k_lo2, const int32_t* __restrict__ k_hi2, int R, int n_q, int n_kv) {
   extern __shared__ float smem[];
   float* qs = smem;                               // [SA_ROWS][HD]
   float* ks = qs + SA_ROWS * HD;                  // [SA_KEYS][HD + 1]
@@ -107,15 +108,28 @@ attention_simt_kernel(const T* __restrict__ q, const T* __restrict__ k, const T*
   float m_r[SA_RPW], l_r[SA_RPW], o_r[SA_RPW][DPL];
 #pragma unroll
   for (int i = 0; i < SA_RPW; ++i) {
-    const int r = wid * SA_RPW + i;
-    lo_r[i] = r < nrows ? k_lo[r0 + r] : 1;
-    hi_r[i] = r < nrows ? k_hi[r0 + r] : 0;
     m_r[i] = -INFINITY;
     l_r[i] = 0.f;
 #pragma unroll
     for (int d = 0; d < DPL; ++d) o_r[i][d] = 0.f;
   }
-  const int key_lo = k_lo[r0], key_hi = k_hi[r0 + nrows - 1];   // both arrays are non-decreasing
+  // A row sees the keys of its first range and, when second-range arrays are given (batched
+  // requests: a query row's own context and its own query tokens are not adjacent), of its
+  // second range.  Each range is walked over the hull of the block's rows.
+  for (int seg = 0; seg < (k_lo2 ? 2 : 1); ++seg) {
+  const int32_t* klo = seg ? k_lo2 : k_lo;
+  const int32_t* khi = seg ? k_hi2 : k_hi;
+  int key_lo = 0x7fffffff, key_hi = -1;
+  for (int r = 0; r < nrows; ++r) {
+    const int a = klo[r0 + r], b = khi[r0 + r];
+    if (a <= b) { key_lo = min(key_lo, a); key_hi = max(key_hi, b); }
+  }
+#pragma unroll
+  for (int i = 0; i < SA_RPW; ++i) {
+    const int r = wid * SA_RPW + i;
+    lo_r[i] = r < nrows ? klo[r0 + r] : 1;
+    hi_r[i] = r < nrows ? khi[r0 + r] : 0;
+  }
   for (int t0 = key_lo; t0 <= key_hi; t0 += SA_KEYS) {
     __syncthreads();
     for (int i = threadIdx.x; i < SA_KEYS * HD; i += 128) {
@@ -160,6 +174,7 @@ attention_simt_kernel(const T* __restrict__ q, const T* __restrict__ k, const T*
       }
     }
   }
+  }
 #pragma unroll
   for (int i = 0; i < SA_RPW; ++i) {
     const int r = wid * SA_RPW + i;
@@ -173,24 +188,25 @@ attention_simt_kernel(const T* __restrict__ q, const T* __restrict__ k, const T*
 
 template <typename T, int HD>
 static int32_t launch_attention_simt_t(const void* q, const void* k, const void* v, void* out, const int32_t* k_lo,
-                                       const int32_t* k_hi, int R, int n_q, int n_kv, cudaStream_t st) {
+                                       const int32_t* k_hi, const int32_t* k_lo2, const int32_t* k_hi2, int R, int n_q,
+                                       int n_kv, cudaStream_t st) {
   const size_t smem = sizeof(float) * (SA_ROWS * HD + SA_KEYS * (HD + 1) + SA_KEYS * HD + SA_ROWS * SA_KEYS);
   const dim3 grid(akvs_cdiv(R, SA_ROWS), n_q);
-  attention_simt_kernel<T, HD><<<grid, 128, smem, st>>>((const T*)q, (const T*)k, (const T*)v, (T*)out, k_lo, k_hi, R,
-                                                       n_q, n_kv);
+  attention_simt_kernel<T, HD><<<grid, 128, smem, st>>>((const T*)q, (const T*)k, (const T*)v, (T*)out, k_lo, k_hi, k_lo2,
+                                                       k_hi2, R, n_q, n_kv);
   AKVS_LAUNCHED();
   return AKVS_OK;
 }
 
 int32_t launch_attention_simt(int dtype, const void* q, const void* k, const void* v, void* out,
-                              const int32_t* k_lo, const int32_t* k_hi, int R, int n_q, int n_kv, int hd,
-                              cudaStream_t st) {
+                              const int32_t* k_lo, const int32_t* k_hi, const int32_t* k_lo2, const int32_t* k_hi2,
+                              int R, int n_q, int n_kv, int hd, cudaStream_t st) {
   if (R == 0) return AKVS_OK;
   if (n_kv <= 0 || n_q % n_kv != 0) return AKVS_ERR_SHAPE;
   return dispatch_dtype(dtype, [&](auto tag) -> int32_t {
     using T = decltype(tag);
-    if (hd == 64) return launch_attention_simt_t<T, 64>(q, k, v, out, k_lo, k_hi, R, n_q, n_kv, st);
-    if (hd == 128) return launch_attention_simt_t<T, 128>(q, k, v, out, k_lo, k_hi, R, n_q, n_kv, st);
+    if (hd == 64) return launch_attention_simt_t<T, 64>(q, k, v, out, k_lo, k_hi, k_lo2, k_hi2, R, n_q, n_kv, st);
+    if (hd == 128) return launch_attention_simt_t<T, 128>(q, k, v, out, k_lo, k_hi, k_lo2, k_hi2, R, n_q, n_kv, st);
     return AKVS_ERR_UNSUPPORTED;
   });
 }
