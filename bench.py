@@ -140,6 +140,9 @@ def main():
     ap.add_argument("--dtype", default="f16", choices=["f16", "bf16"],
                     help="16-bit storage type of weights, cache and activations (weight VALUES are bf16 either way)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--batch", type=int, default=1,
+                    help="requests per call that share the model (each retrieves all units in its own order); "
+                         "the metric's configuration is 1")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -184,8 +187,16 @@ def main():
     kvf = {"native": akvs.KV_NATIVE, "q4": akvs.KV_Q4, "q2": akvs.KV_Q2}[w.kv_format]
     store = akvs.UnitStore(gmodel, lens, ctx_ids, kvf)
     order = list(range(w.n_units))
-    req = akvs.Request(order, qry_ids)
     N, nq, M = int(lens.sum()), w.n_query, w.n_units
+    B = max(1, args.batch)
+    if B == 1:
+        req = akvs.Request(order, qry_ids)
+        pos_local = np.arange(N + nq, dtype=np.float64)
+    else:
+        # every request retrieves the same units in its own order and asks its own question
+        req = akvs.Request.batch([([(u + 5 * b) % M for u in order], np.roll(qry_ids, 7 * b)) for b in range(B)])
+        pos_local = np.concatenate([np.tile(np.arange(N), B), np.tile(N + np.arange(nq), B)]).astype(np.float64)
+        N, nq, M = N * B, nq * B, M * B
     T = N + nq
     ws = akvs.alloc_workspace(akvs.workspace_bytes(gmodel, N, nq, M, CHECK_LAYER))
     ev = lambda: torch.cuda.Event(enable_timing=True)
@@ -251,8 +262,9 @@ def main():
         a[0] += ms_; a[1] += fl; a[2] += 1
     # attention flops of one step from the recomputed rows: 4 * dq * sum_r (keys visible to r);
     # the dense first layer sees every row, the selective layers the probe and query rows
-    rows = probes.rows[:probes.n_rows].cpu().numpy().astype(np.float64)
-    a_fl = 4.0 * m.dq * ((CHECK_LAYER - 1) * (T * (T + 1) / 2.0) + (m.n_layers - CHECK_LAYER + 1) * float((rows + 1).sum()))
+    rows = probes.rows[:probes.n_rows].cpu().numpy()
+    a_fl = 4.0 * m.dq * ((CHECK_LAYER - 1) * float((pos_local + 1).sum()) +
+                         (m.n_layers - CHECK_LAYER + 1) * float((pos_local[rows] + 1).sum()))
     a_ms = sum(r[0] for r in attn) / args.steps
     c_ms = sum(r[0] for r in corr)
     c_by = sum(r[1] for r in corr)
@@ -268,7 +280,7 @@ def main():
     roofline = {"bound": "tensor", "kernel": "gemm_tc_kernel (all linear layers of the step)",
                 "achieved": achieved, "peak": pk["tensor"], "unit": "TFLOP/s", "frac": achieved / pk["tensor"],
                 "peak_source": pk["src"] + " bf16 cuBLAS sustained (f16 and bf16 MMAs run at the same rate)",
-                "traffic": GEMM_TRAFFIC_PER_LAUNCH.get(args.workload), "launches": len(gemm), "share_of_step": g_ms / (ms_step * args.steps),
+                "traffic": GEMM_TRAFFIC_PER_LAUNCH.get(args.workload) if B == 1 else None, "launches": len(gemm), "share_of_step": g_ms / (ms_step * args.steps),
                 "by_epilogue": {{0: "qkv_store", 1: "residual", 2: "swiglu"}.get(k, str(k)):
                                 {"tflops": v[1] / (v[0] * 1e-3) / 1e12, "ms_per_step": v[0] / args.steps,
                                  "launches": v[2]} for k, v in sorted(by_epi.items())}}
@@ -330,7 +342,9 @@ def main():
                   "bf16": "bf16 storage, f32 accumulate", "f32": "f32"}[m.dtype],
         "data": "synthetic",
         "config": {"workload": f"{w.name}: {m.name}-class decoder L{m.n_layers} d{m.d_model} {m.n_q_heads}q/{m.n_kv_heads}kv "
-                               f"hd{m.head_dim} ff{m.d_ff}; {M} units {w.len_lo}-{w.len_hi} tok (N={N}) + {nq} query",
+                               f"hd{m.head_dim} ff{m.d_ff}; {M // B} units {w.len_lo}-{w.len_hi} tok (N={N // B}) + {nq // B} query"
+                               + (f", batch of {B} requests per call" if B > 1 else ""),
+                   "batch": B,
                    "refresh_bp": bp, "check_layer": CHECK_LAYER, "probe_rows": P, "rows_recomputed": P + nq,
                    "effective_refresh": P / max(1, N), "kv_format": w.kv_format, "parallelism": f"replicas x{world}",
                    "l2": "inputs larger than L2: each step streams all layer weights "
