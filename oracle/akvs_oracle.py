@@ -209,13 +209,51 @@ def pack_codes(codes, bits):
     return out.astype(np.uint8)
 
 
+# --------------------------------------------------------------------------- FP8 cache
+
+E4M3_MAX = 448.0
+
+
+def e4m3_encode(x):
+    """Element-wise cast to FP8 E4M3 (the format the quantisation study of Section 4.5 names:
+    1 sign, 4 exponent bits with bias 7, 3 mantissa bits, no infinities, largest finite value
+    448, subnormals in steps of 2^-9).  The paper gives no scaling, so the reading is a plain
+    cast of the value (first rounded to float32): round to nearest, ties to the even mantissa,
+    magnitudes above 448 saturate to 448.  Returns the uint8 bit patterns."""
+    x = np.asarray(x, np.float32).astype(np.float64)
+    if not np.all(np.isfinite(x)):
+        raise ValueError("e4m3_encode: non-finite input")
+    sign = np.signbit(x)
+    a = np.minimum(np.abs(x), E4M3_MAX)
+    _, ex = np.frexp(a)                              # a = m 2^ex, m in [0.5, 1)
+    e = np.clip(ex - 1, -6, 8)                       # binade; everything below 2^-6 is subnormal
+    q = np.exp2(e - 3.0)                             # spacing of the grid in that binade
+    v = np.rint(a / q) * q                           # half to even; may land on the next binade's first value
+    _, ex2 = np.frexp(v)
+    e2 = ex2 - 1
+    normal = v >= 2.0 ** -6
+    ebits = np.where(normal, e2 + 7, 0).astype(np.int64)
+    mant = np.where(normal, np.rint((v / np.exp2(np.where(normal, e2, 0).astype(np.float64)) - 1.0) * 8.0),
+                    np.rint(v / 2.0 ** -9)).astype(np.int64)
+    return ((sign.astype(np.int64) << 7) | (ebits << 3) | mant).astype(np.uint8)
+
+
+def e4m3_decode(code):
+    """Value of an E4M3 bit pattern (the two NaN patterns 0x7f / 0xff never occur here)."""
+    c = np.asarray(code, np.uint8).astype(np.int64)
+    s = np.where(c & 0x80, -1.0, 1.0)
+    ebits, m = (c >> 3) & 15, c & 7
+    return s * np.where(ebits == 0, m * 2.0 ** -9, (1.0 + m / 8.0) * np.exp2(ebits - 7.0))
+
+
 # --------------------------------------------------------------------------- the four modes
 
 def encode_units(model, unit_ids_list, kv_bits=0, dtype=np.float64):
     """Section 3.1: each unit alone, positions 0..n-1, causal.  Returns a list (one entry
     per unit) of dicts with K [L][n][n_kv][hd] (post-RoPE at LOCAL positions) and V.
     With kv_bits in (2, 4) the cached values are the dequantised reconstructions and the
-    codes/scale/minimum are kept beside them."""
+    codes/scale/minimum are kept beside them; kv_bits = 8 is the FP8 (E4M3) cache: the cached
+    values are the decoded bytes, kept beside them as codes."""
     c = model.cfg
     out = []
     for ids in unit_ids_list:
@@ -228,7 +266,11 @@ def encode_units(model, unit_ids_list, kv_bits=0, dtype=np.float64):
             Ks.append(k)
             Vs.append(v)
         unit = {"K": np.stack(Ks), "V": np.stack(Vs), "hidden": h}
-        if kv_bits:
+        if kv_bits == 8:
+            for name in ("K", "V"):
+                unit[name + "_codes"] = e4m3_encode(unit[name])
+                unit[name] = e4m3_decode(unit[name + "_codes"]).astype(dtype)
+        elif kv_bits:
             for name in ("K", "V"):
                 codes, s16, m16 = quantize_groups(unit[name], kv_bits)
                 unit[name + "_codes"], unit[name + "_scale"], unit[name + "_min"] = codes, s16, m16

@@ -288,3 +288,46 @@ def test_quantiser_round_half_even_and_packing():
     c4 = (np.arange(64) % 16).astype(np.uint8).reshape(1, 64)
     p4 = orc.pack_codes(c4, 4)
     assert p4.shape == (1, 32) and p4[0, 0] == (0 | 1 << 4) and p4[0, 7] == (14 | 15 << 4)
+
+
+# ----------------------------------------------------------------------------- FP8 (E4M3) cache
+
+def test_e4m3_every_code_round_trips():
+    """All 254 finite bit patterns decode to a value that encodes back to the same pattern
+    (brute force over the whole format); the decoded table has the format's landmarks."""
+    codes = np.array([c for c in range(256) if c & 0x7f != 0x7f], np.uint8)
+    vals = orc.e4m3_decode(codes)
+    assert np.array_equal(orc.e4m3_encode(vals), codes)
+    assert vals.max() == 448.0 and vals.min() == -448.0
+    pos = np.sort(vals[vals > 0])
+    assert pos[0] == 2.0 ** -9 and pos[7] == 2.0 ** -6          # smallest subnormal, smallest normal
+    assert orc.e4m3_decode(np.uint8(0x38)) == 1.0 and orc.e4m3_decode(np.uint8(0x40)) == 2.0
+
+
+def test_e4m3_rounding_rules():
+    """Ties go to the even mantissa, everything else to the nearest value, magnitudes above
+    448 saturate (hand-computed cases: between 1 and 2 the grid step is 1/8)."""
+    enc = lambda x: float(orc.e4m3_decode(orc.e4m3_encode(np.float32(x))))
+    assert enc(1.0625) == 1.0            # tie between 1.0 (mantissa 0) and 1.125 (mantissa 1)
+    assert enc(1.1875) == 1.25           # tie between 1.125 (1) and 1.25 (2)
+    assert enc(1.07) == 1.125 and enc(1.05) == 1.0
+    assert enc(1.96) == 2.0              # rounds up into the next binade
+    assert enc(447.0) == 448.0 and enc(1.0e6) == 448.0 and enc(-3.0e4) == -448.0
+    assert enc(2.0 ** -10) == 0.0        # tie between 0 and the smallest subnormal 2^-9: even is 0
+    assert enc(3 * 2.0 ** -10) == 2.0 ** -8   # tie between 1 and 2 subnormal steps: even is 2
+    assert enc(0.0) == 0.0 and orc.e4m3_encode(np.float32(-0.0)) == 0x80
+
+
+def test_e4m3_matches_the_library_cast_and_is_monotone():
+    """Against torch's CPU float8_e4m3fn conversion (an independent implementation) on random
+    values inside the finite range, plus monotonicity and idempotence."""
+    import torch
+    g = np.random.default_rng(5)
+    x = np.concatenate([g.normal(0, 3, 20000), g.normal(0, 0.01, 5000), g.uniform(-448, 448, 5000)]).astype(np.float32)
+    ours = orc.e4m3_decode(orc.e4m3_encode(x))
+    lib = torch.from_numpy(x).to(torch.float8_e4m3fn).to(torch.float64).numpy()
+    assert np.array_equal(ours, lib)
+    xs = np.sort(x)
+    assert np.all(np.diff(orc.e4m3_decode(orc.e4m3_encode(xs))) >= 0)
+    assert np.array_equal(orc.e4m3_encode(ours), orc.e4m3_encode(x))
+    assert np.all(np.abs(ours - x) <= np.maximum(np.abs(x) / 16, 2.0 ** -10))   # half a step of 3 mantissa bits
