@@ -184,7 +184,7 @@ def main():
                                       n_threads=max(1, min(12, cores // max(1, world))))
     lens = testgen.unit_lengths(w, SEED_LEN)
     ctx_ids, qry_ids = testgen.token_ids(w, SEED_IDS, lens)
-    kvf = {"native": akvs.KV_NATIVE, "q4": akvs.KV_Q4, "q2": akvs.KV_Q2}[w.kv_format]
+    kvf = {"native": akvs.KV_NATIVE, "q4": akvs.KV_Q4, "q2": akvs.KV_Q2, "fp8": akvs.KV_FP8}[w.kv_format]
     store = akvs.UnitStore(gmodel, lens, ctx_ids, kvf)
     order = list(range(w.n_units))
     N, nq, M = int(lens.sum()), w.n_query, w.n_units

@@ -55,6 +55,8 @@ extern "C" {
 #define AKVS_KV_NATIVE 0           /* cache holds the model dtype                            */
 #define AKVS_KV_Q2     2           /* 2-bit codes, asymmetric min-max, groups of 64 along head_dim */
 #define AKVS_KV_Q4     4           /* 4-bit codes, same scheme                               */
+#define AKVS_KV_FP8    8           /* FP8 E4M3 bytes (Section 4.5 names the format; no scale: a saturating
+                                      round-to-nearest-even cast of each value), no k_meta / v_meta */
 
 #define AKVS_MODE_CORRECTED 0      /* Algorithm 1                                            */
 #define AKVS_MODE_NAIVE     1      /* direct reuse (Section 3.1): only the query is computed */
@@ -278,7 +280,8 @@ int32_t akvs_op_correct_layer(int32_t dtype, int32_t kv_format,
                               void* scratch, void* stream);
 
 /* Group quantiser of the cache (asymmetric min-max, groups of 64 along head_dim, float16
- * scale and minimum): x [n][n_kv][hd] -> codes [n][n_kv][hd*bits/8], meta half2 [n][n_kv][hd/64]. */
+ * scale and minimum): x [n][n_kv][hd] -> codes [n][n_kv][hd*bits/8], meta half2 [n][n_kv][hd/64].
+ * bits = 8 is the FP8 (E4M3) cast: one byte per value, meta unused (may be NULL). */
 int32_t akvs_op_quantize(int32_t dtype, const void* x, int32_t n, int32_t n_kv_heads, int32_t head_dim,
                          int32_t bits, void* codes, void* meta, void* stream);
 

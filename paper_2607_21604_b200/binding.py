@@ -19,7 +19,7 @@ ERR = {0: "AKVS_OK", -1: "AKVS_ERR_INVALID_ARG", -2: "AKVS_ERR_SHAPE", -3: "AKVS
        -4: "AKVS_ERR_UNSUPPORTED", -5: "AKVS_ERR_CUDA", -6: "AKVS_ERR_TIMEOUT", -7: "AKVS_ERR_NAN_SCORE",
        -8: "AKVS_ERR_TOO_LARGE"}
 F32, BF16, F16 = 0, 1, 2
-KV_NATIVE, KV_Q2, KV_Q4 = 0, 2, 4
+KV_NATIVE, KV_Q2, KV_Q4, KV_FP8 = 0, 2, 4, 8
 MODE_CORRECTED, MODE_NAIVE, MODE_FULL = 0, 1, 2
 
 EXPORTS = ["akvs_workspace_bytes", "akvs_debug_set_linear_algo", "akvs_launch_count", "akvs_prof_enable",
@@ -176,6 +176,10 @@ class UnitStore:
         if kv_format == KV_NATIVE:
             td = _tdtype(model.dtype)
             self.k = torch.zeros((L, N, cfg.n_kv_heads, cfg.head_dim), dtype=td, device=device)
+            self.v = torch.zeros_like(self.k)
+            self.k_meta = self.v_meta = None
+        elif kv_format == KV_FP8:
+            self.k = torch.zeros((L, N, cfg.n_kv_heads, cfg.head_dim), dtype=torch.uint8, device=device)
             self.v = torch.zeros_like(self.k)
             self.k_meta = self.v_meta = None
         else:
@@ -411,7 +415,7 @@ def op_quantize(x, bits):
     dtype = _dt(x)
     n, nkv, hd = x.shape
     codes = torch.empty((n, nkv, hd * bits // 8), dtype=torch.uint8, device=x.device)
-    meta = torch.empty((n, nkv, hd // 64, 2), dtype=torch.float16, device=x.device)
+    meta = None if bits == KV_FP8 else torch.empty((n, nkv, hd // 64, 2), dtype=torch.float16, device=x.device)
     _chk(lib.akvs_op_quantize(dtype, _ptr(x), n, nkv, hd, bits, _ptr(codes), _ptr(meta), _stream()),
          "akvs_op_quantize")
     return codes, meta

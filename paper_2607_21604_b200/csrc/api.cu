@@ -259,7 +259,7 @@ KvLayer cache_layer(const akvs_cache* c, const Dims& D, int l) {
   kv.k = reinterpret_cast<const char*>(c->k) + l * stride;
   kv.v = reinterpret_cast<const char*>(c->v) + l * stride;
   kv.fmt = c->kv_format;
-  if (c->kv_format == AKVS_KV_NATIVE) {
+  if (c->kv_format == AKVS_KV_NATIVE || c->kv_format == AKVS_KV_FP8) {
     kv.k_meta = kv.v_meta = nullptr;
   } else {
     const size_t ms = (size_t)c->n_tokens * D.nkv * (D.hd / 64) * 4;
@@ -279,15 +279,15 @@ int32_t wait_layer(const akvs_cache* c, int l, cudaStream_t st) {
 int32_t check_cache(const akvs_cache* c, const Dims& D, bool need_kv) {
   if (!c || !c->unit_off || !c->token_ids) return AKVS_ERR_INVALID_ARG;
   if (c->n_units < 0 || c->n_tokens < 0) return AKVS_ERR_INVALID_ARG;
-  if (c->kv_format != AKVS_KV_NATIVE && c->kv_format != AKVS_KV_Q4 && c->kv_format != AKVS_KV_Q2)
-    return AKVS_ERR_UNSUPPORTED;
-  if (c->kv_format != AKVS_KV_NATIVE && D.hd % 64 != 0) return AKVS_ERR_UNSUPPORTED;
+  const bool grouped = c->kv_format == AKVS_KV_Q4 || c->kv_format == AKVS_KV_Q2;
+  if (c->kv_format != AKVS_KV_NATIVE && c->kv_format != AKVS_KV_FP8 && !grouped) return AKVS_ERR_UNSUPPORTED;
+  if (grouped && D.hd % 64 != 0) return AKVS_ERR_UNSUPPORTED;
   if (c->unit_off[0] != 0 || c->unit_off[c->n_units] != c->n_tokens) return AKVS_ERR_SHAPE;
   for (int u = 0; u < c->n_units; ++u)
     if (c->unit_off[u + 1] < c->unit_off[u]) return AKVS_ERR_SHAPE;
   if (need_kv) {
     if (!c->k || !c->v) return AKVS_ERR_INVALID_ARG;
-    if (c->kv_format != AKVS_KV_NATIVE && (!c->k_meta || !c->v_meta)) return AKVS_ERR_INVALID_ARG;
+    if (grouped && (!c->k_meta || !c->v_meta)) return AKVS_ERR_INVALID_ARG;
   }
   return AKVS_OK;
 }
@@ -527,12 +527,13 @@ int32_t akvs_encode_units(const akvs_model_desc* model, akvs_cache* cache, void*
     std::function<int32_t()> store;
     if (!native)
       store = [&, l]() -> int32_t {
+        const bool has_meta = cache->kv_format != AKVS_KV_FP8;
         AKVS_TRY(launch_quantize(D.dtype, ws.k, N, D.nkv, D.hd, cache->kv_format,
                                  reinterpret_cast<char*>(cache->k) + l * lstride,
-                                 reinterpret_cast<char*>(cache->k_meta) + l * mstride, st));
+                                 has_meta ? reinterpret_cast<char*>(cache->k_meta) + l * mstride : nullptr, st));
         return launch_quantize(D.dtype, ws.v, N, D.nkv, D.hd, cache->kv_format,
                                reinterpret_cast<char*>(cache->v) + l * lstride,
-                               reinterpret_cast<char*>(cache->v_meta) + l * mstride, st);
+                               has_meta ? reinterpret_cast<char*>(cache->v_meta) + l * mstride : nullptr, st);
       };
     AKVS_TRY(run_layer(model, D, l, ws, N, RowGeom{local_pos, ws.lo, ws.pos, nullptr, nullptr}, k_dst, v_dst, k_dst,
                        v_dst, N, store, st));
@@ -853,7 +854,7 @@ int32_t akvs_op_correct_layer(int32_t dtype, int32_t kv_format, const void* cach
 
 int32_t akvs_op_quantize(int32_t dtype, const void* x, int32_t n, int32_t n_kv_heads, int32_t head_dim, int32_t bits,
                          void* codes, void* meta, void* stream) {
-  if (!x || !codes || !meta || n < 0) return AKVS_ERR_INVALID_ARG;
+  if (!x || !codes || (!meta && bits != AKVS_KV_FP8) || n < 0) return AKVS_ERR_INVALID_ARG;
   if (dtype != AKVS_F32 && dtype != AKVS_BF16 && dtype != AKVS_F16) return AKVS_ERR_UNSUPPORTED;
   return launch_quantize(dtype, x, n, n_kv_heads, head_dim, bits, codes, meta, reinterpret_cast<cudaStream_t>(stream));
 }

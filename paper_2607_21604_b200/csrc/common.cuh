@@ -62,6 +62,7 @@ static inline int32_t dispatch_fmt(int fmt, F&& f) {
     case AKVS_KV_NATIVE: return f(std::integral_constant<int, AKVS_KV_NATIVE>{});
     case AKVS_KV_Q4: return f(std::integral_constant<int, AKVS_KV_Q4>{});
     case AKVS_KV_Q2: return f(std::integral_constant<int, AKVS_KV_Q2>{});
+    case AKVS_KV_FP8: return f(std::integral_constant<int, AKVS_KV_FP8>{});
     default: return AKVS_ERR_UNSUPPORTED;
   }
 }

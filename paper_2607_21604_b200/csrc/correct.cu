@@ -8,10 +8,29 @@
 // so that the re-alignment rotation needs no exchange between threads and every global
 // access is a full 16-byte vector.
 #include "common.cuh"
+#include <cuda_fp8.h>
 
 // ---------------------------------------------------------------------------------------
 // Reading one pair chunk of the reused K or V of store row `src`, head `h`, chunk `c`.
 // ---------------------------------------------------------------------------------------
+// Eight (or four) FP8 E4M3 bytes -> floats (E4M3 values are exact in float16).
+template <int V>
+__device__ __forceinline__ void ld_fp8(const uint8_t* p, float (&out)[V]) {
+  uint32_t w[V / 4];
+  if constexpr (V == 8) {
+    const uint2 t = *reinterpret_cast<const uint2*>(p);
+    w[0] = t.x; w[1] = t.y;
+  } else {
+    w[0] = *reinterpret_cast<const uint32_t*>(p);
+  }
+#pragma unroll
+  for (int i = 0; i < V / 2; ++i) {
+    const __half2_raw h = __nv_cvt_fp8x2_to_halfraw2((__nv_fp8x2_storage_t)((w[i >> 1] >> (16 * (i & 1))) & 0xFFFFu), __NV_E4M3);
+    const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&h));
+    out[2 * i] = f.x; out[2 * i + 1] = f.y;
+  }
+}
+
 template <int BYTES>
 __device__ __forceinline__ uint32_t ld_codes(const uint8_t* p) {
   if constexpr (BYTES == 4) return *reinterpret_cast<const uint32_t*>(p);
@@ -25,6 +44,8 @@ __device__ __forceinline__ void load_cached_chunk(const void* base, const void* 
   constexpr int V = VecOf<T>::N;
   if constexpr (FMT == AKVS_KV_NATIVE) {
     ld16(reinterpret_cast<const T*>(base) + ((size_t)src * n_kv + h) * hd + dim0, out);
+  } else if constexpr (FMT == AKVS_KV_FP8) {
+    ld_fp8<V>(reinterpret_cast<const uint8_t*>(base) + ((size_t)src * n_kv + h) * hd + dim0, out);
   } else {
     constexpr int BITS = FMT;
     constexpr int BYTES = V * BITS / 8;
@@ -173,8 +194,10 @@ __global__ void scores_kernel(KvLayer kv, ReqMaps maps, const T* __restrict__ k_
 static int32_t check_kv_shape(int dtype, const KvLayer& kv, int hd) {
   const int V = dtype == AKVS_F32 ? 4 : 8;
   if (hd % (2 * V) != 0) return AKVS_ERR_UNSUPPORTED;
-  if (kv.fmt != AKVS_KV_NATIVE && kv.fmt != AKVS_KV_Q4 && kv.fmt != AKVS_KV_Q2) return AKVS_ERR_UNSUPPORTED;
-  if (kv.fmt != AKVS_KV_NATIVE && (hd % 64 != 0 || !kv.k_meta || !kv.v_meta)) return AKVS_ERR_UNSUPPORTED;
+  if (kv.fmt != AKVS_KV_NATIVE && kv.fmt != AKVS_KV_Q4 && kv.fmt != AKVS_KV_Q2 && kv.fmt != AKVS_KV_FP8)
+    return AKVS_ERR_UNSUPPORTED;
+  if ((kv.fmt == AKVS_KV_Q4 || kv.fmt == AKVS_KV_Q2) && (hd % 64 != 0 || !kv.k_meta || !kv.v_meta))
+    return AKVS_ERR_UNSUPPORTED;
   return AKVS_OK;
 }
 
@@ -359,6 +382,11 @@ offsets_kernel(KvLayer kv, ReqMaps maps, const int32_t* __restrict__ probe_off, 
         const TW* cp = reinterpret_cast<const TW*>(cbase) + ((size_t)src * n_kv + h) * hd;
         lo = to_f(cp[e]);
         hi = to_f(cp[half + e]);
+      } else if constexpr (FMT == AKVS_KV_FP8) {
+        const uint8_t* cp = reinterpret_cast<const uint8_t*>(cbase) + ((size_t)src * n_kv + h) * hd;
+        const __half_raw ra = __nv_cvt_fp8_to_halfraw(cp[e], __NV_E4M3), rb = __nv_cvt_fp8_to_halfraw(cp[half + e], __NV_E4M3);
+        lo = __half2float(*reinterpret_cast<const __half*>(&ra));
+        hi = __half2float(*reinterpret_cast<const __half*>(&rb));
       } else {
         const uint8_t* cp = reinterpret_cast<const uint8_t*>(cbase) + ((size_t)src * n_kv + h) * hd * FMT / 8;
         const __half2* mp = reinterpret_cast<const __half2*>(cmeta) + ((size_t)src * n_kv + h) * (hd / 64);
@@ -424,6 +452,7 @@ template <typename TW, int FMT> struct RawChunk;
 template <typename TW> struct RawChunk<TW, AKVS_KV_NATIVE> { uint4 v; };
 template <typename TW> struct RawChunk<TW, AKVS_KV_Q4> { uint32_t packed; __half2 sm; };
 template <typename TW> struct RawChunk<TW, AKVS_KV_Q2> { uint32_t packed; __half2 sm; };
+template <typename TW> struct RawChunk<TW, AKVS_KV_FP8> { uint32_t w[2]; };
 
 __device__ __forceinline__ void unpack16(const uint4& r, float (&o)[4], const float*) {
   o[0] = __uint_as_float(r.x); o[1] = __uint_as_float(r.y); o[2] = __uint_as_float(r.z); o[3] = __uint_as_float(r.w);
@@ -457,6 +486,14 @@ __device__ __forceinline__ void issue_chunk(bool from_fresh, const T* fresh_p, c
     fresh_raw = *reinterpret_cast<const uint4*>(fresh_p);
   } else if constexpr (FMT == AKVS_KV_NATIVE) {
     raw.v = *reinterpret_cast<const uint4*>(reinterpret_cast<const TW*>(base) + ((size_t)src * n_kv + h) * hd + dim0);
+  } else if constexpr (FMT == AKVS_KV_FP8) {
+    const uint8_t* cp = reinterpret_cast<const uint8_t*>(base) + ((size_t)src * n_kv + h) * hd + dim0;
+    if constexpr (V == 8) {
+      const uint2 t = *reinterpret_cast<const uint2*>(cp);
+      raw.w[0] = t.x; raw.w[1] = t.y;
+    } else {
+      raw.w[0] = *reinterpret_cast<const uint32_t*>(cp);
+    }
   } else {
     constexpr int BYTES = V * FMT / 8;
     raw.packed = ld_codes<BYTES>(reinterpret_cast<const uint8_t*>(base) + (((size_t)src * n_kv + h) * hd + dim0) * FMT / 8);
@@ -473,6 +510,13 @@ __device__ __forceinline__ void decode_chunk(bool from_fresh, const uint4& fresh
     unpack16(fresh_raw, out, (const T*)nullptr);
   } else if constexpr (FMT == AKVS_KV_NATIVE) {
     unpack16(raw.v, out, (const TW*)nullptr);
+  } else if constexpr (FMT == AKVS_KV_FP8) {
+#pragma unroll
+    for (int i = 0; i < V / 2; ++i) {
+      const __half2_raw h = __nv_cvt_fp8x2_to_halfraw2((__nv_fp8x2_storage_t)((raw.w[i >> 1] >> (16 * (i & 1))) & 0xFFFFu), __NV_E4M3);
+      const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&h));
+      out[2 * i] = f.x; out[2 * i + 1] = f.y;
+    }
   } else {
     const float s = __low2float(raw.sm), mn = __high2float(raw.sm);
 #pragma unroll
@@ -605,7 +649,8 @@ int32_t launch_correct(int dtype, const KvLayer& kv, const ReqMaps& maps, const 
   const int grid = (int)(want < 148 * 4 ? want : 148 * 4);   // grid-stride; two resident CTAs of 256 threads per SM
   // algorithmic bytes: every context K and V element read once in its cache format and
   // written once; fresh rows and query rows copied; 8 bytes of weights per context token
-  const double in_b = kv.fmt == AKVS_KV_NATIVE ? (double)dtype_size(dtype) : kv.fmt / 8.0 + 4.0 / 64.0;
+  const double in_b = kv.fmt == AKVS_KV_NATIVE ? (double)dtype_size(dtype)
+                      : kv.fmt == AKVS_KV_FP8  ? 1.0 : kv.fmt / 8.0 + 4.0 / 64.0;
   const double out_b = (double)dtype_size(dtype);
   const double bytes = 2.0 * n_kv * hd * ((double)N * (in_b + out_b) + (double)n_query * 2 * out_b) + 8.0 * N;
   ProfScope prof(2, kv.fmt, bytes, st);

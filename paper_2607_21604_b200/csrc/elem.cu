@@ -2,6 +2,7 @@
 // RoPE table + rotation, and the cache group quantiser.  All are HBM-bound; every global
 // access is a 16-byte vector where the layout allows it.
 #include "common.cuh"
+#include <cuda_fp8.h>
 
 // ---------------------------------------------------------------------------------------
 // h[r][:] = float(tok_emb[ids[gather ? gather[r] : r]][:])
@@ -239,9 +240,35 @@ __global__ void quantize_kernel(const T* __restrict__ x, int64_t n_groups, int b
   if (lane == 0) meta[g] = __halves2half2(s16, m16);
 }
 
+// FP8 (E4M3) cache: every value cast by itself, round to nearest even, saturating at 448.
+template <typename T>
+__global__ void fp8_cast_kernel(const T* __restrict__ x, int64_t n, uint8_t* __restrict__ codes) {
+  const int64_t i = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) * 4;
+  if (i >= n) return;
+  uint8_t c[4];
+#pragma unroll
+  for (int e = 0; e < 4; ++e)
+    c[e] = i + e < n ? (uint8_t)__nv_cvt_float_to_fp8(to_f(x[i + e]), __NV_SATFINITE, __NV_E4M3) : 0;
+  if (i + 3 < n) {
+    *reinterpret_cast<uchar4*>(codes + i) = make_uchar4(c[0], c[1], c[2], c[3]);
+  } else {
+    for (int e = 0; i + e < n; ++e) codes[i + e] = c[e];
+  }
+}
+
 int32_t launch_quantize(int dtype, const void* x, int n, int n_kv, int hd, int bits, void* codes, void* meta,
                         cudaStream_t st) {
   if (n == 0) return AKVS_OK;
+  if (bits == AKVS_KV_FP8) {
+    const int64_t total = (int64_t)n * n_kv * hd;          // rows of n_kv * hd bytes: 4-byte stores stay aligned
+    if ((n_kv * hd) % 4 != 0) return AKVS_ERR_UNSUPPORTED;
+    return dispatch_dtype(dtype, [&](auto tag) -> int32_t {
+      using T = decltype(tag);
+      fp8_cast_kernel<T><<<akvs_cdiv((total + 3) / 4, 256), 256, 0, st>>>((const T*)x, total, (uint8_t*)codes);
+      AKVS_LAUNCHED();
+      return AKVS_OK;
+    });
+  }
   if (hd % 64 != 0 || (bits != 2 && bits != 4)) return AKVS_ERR_UNSUPPORTED;
   const int64_t n_groups = (int64_t)n * n_kv * (hd / 64);
   const int blocks = akvs_cdiv(n_groups, 8);

@@ -60,7 +60,7 @@ def main():
     batches = [int(x) for x in args.batch.split(",")]
     gmodel = akvs.Model.from_layer_fn(m, testgen.embedding(m, SEED_W), lambda l: testgen.layer_weights(m, SEED_W, l),
                                       n_threads=12)
-    kvf = {"native": akvs.KV_NATIVE, "q4": akvs.KV_Q4, "q2": akvs.KV_Q2}[w0.kv_format]
+    kvf = {"native": akvs.KV_NATIVE, "q4": akvs.KV_Q4, "q2": akvs.KV_Q2, "fp8": akvs.KV_FP8}[w0.kv_format]
     print(f"# {w0.name}: {m.name}-class decoder L{m.n_layers} d{m.d_model}, units {w0.len_lo}-{w0.len_hi} tokens, "
           f"{w0.n_query} query tokens, check layer {args.check_layer}, cache {w0.kv_format}")
     print("| tok/req | batch | refresh | rows recomputed | corrected ms | full ms | naive ms | speedup vs full | "

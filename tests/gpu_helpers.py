@@ -64,6 +64,9 @@ class Case:
                 n = u["K"].shape[1]
                 u["K"], u["V"] = ks[:, o:o + n], vs[:, o:o + n]
                 o += n
+        elif self.kv_format == 8:
+            for name, dst in (("K", self.store.k), ("V", self.store.v)):
+                dst.copy_(torch.from_numpy(np.concatenate([u[name + "_codes"] for u in units], axis=1)))
         else:
             for name, dst, dmeta in (("K", self.store.k, self.store.k_meta), ("V", self.store.v, self.store.v_meta)):
                 codes = np.concatenate([u[name + "_codes"] for u in units], axis=1)

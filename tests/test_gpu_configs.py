@@ -33,10 +33,10 @@ def test_config_width_reduced_depth(name, n_layers, n_units):
     _run_all_modes(case, w.refresh_bp[0], 2, units)
 
 
-@pytest.mark.parametrize("name", ["c5q4", "c5q2"])
+@pytest.mark.parametrize("name", ["c5q4", "c5q2", "c5fp8"])
 def test_config5_quantised_cache(name):
     w = _reduced(name, 3, 4)
-    fmt = 4 if name.endswith("q4") else 2
+    fmt = {"c5q4": 4, "c5q2": 2, "c5fp8": 8}[name]
     case = Case(w, kv_format=fmt)
     case.encode()
     units = case.oracle_units()

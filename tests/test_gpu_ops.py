@@ -207,6 +207,23 @@ def test_quantize_bit_exact(akvs, bits, dtype):
     assert np.array_equal(m[..., 1].view(np.uint16), rm.view(np.uint16))
 
 
+@pytest.mark.parametrize("dtype", [torch.float32, torch.float16, torch.bfloat16])
+def test_fp8_cast_bit_exact(akvs, dtype):
+    """FP8 (E4M3) cache bytes equal the oracle's cast of the same stored values: random data,
+    ties, subnormals, saturation, signed zero."""
+    g = np.random.default_rng(8)
+    x = g.standard_normal((77, 2, 128)).astype(np.float32) * 3
+    x[0, 0, :16] = [1.0625, 1.1875, 1.07, 1.96, 447.0, 6e4, -3e4, 2.0 ** -10, 3 * 2.0 ** -10, 0.0, -0.0, 2.0 ** -9,
+                    -2.0 ** -6, 448.0, 0.0009, -0.0021]
+    x[1] *= 0.004                                          # subnormal range of the format
+    x[2] *= 100                                            # saturating range
+    xt = dev(x, dtype)
+    codes, meta = akvs.op_quantize(xt, 8)
+    torch.cuda.synchronize()
+    assert meta is None
+    assert np.array_equal(codes.cpu().numpy(), orc.e4m3_encode(xt.float().cpu().numpy()))
+
+
 # ----------------------------------------------------------------------------- offsets + correction
 
 def _correct_case(akvs, dtype_t, kv_format, N_units, len_lo, len_hi, nkv, hd, nq, bp, seed=0):
@@ -236,6 +253,11 @@ def _correct_case(akvs, dtype_t, kv_format, N_units, len_lo, len_hi, nkv, hd, nq
         ck_t, cv_t = dev(ck, dtype_t), dev(cv, dtype_t)
         ck_ref, cv_ref = n64(ck_t), n64(cv_t)
         km = vm = None
+    elif kv_format == 8:
+        kc, vc = orc.e4m3_encode(ck), orc.e4m3_encode(cv)
+        ck_t, cv_t = dev(kc), dev(vc)
+        km = vm = None
+        ck_ref, cv_ref = orc.e4m3_decode(kc), orc.e4m3_decode(vc)
     else:
         kc, ks, kmn = orc.quantize_groups(ck, kv_format)
         vc, vs, vmn = orc.quantize_groups(cv, kv_format)
@@ -278,14 +300,16 @@ def _correct_case(akvs, dtype_t, kv_format, N_units, len_lo, len_hi, nkv, hd, nq
 @pytest.mark.parametrize("dtype_t,kv_format,hd", [(torch.float32, 0, 64), (torch.float16, 0, 128),
                                                   (torch.bfloat16, 0, 128), (torch.bfloat16, 4, 64),
                                                   (torch.float16, 4, 128), (torch.float16, 2, 128),
-                                                  (torch.float32, 4, 64), (torch.float32, 2, 128)])
+                                                  (torch.float32, 4, 64), (torch.float32, 2, 128),
+                                                  (torch.float16, 8, 128), (torch.bfloat16, 8, 64),
+                                                  (torch.float32, 8, 64)])
 def test_correct_layer_small_ragged(akvs, dtype_t, kv_format, hd):
     _correct_case(akvs, dtype_t, kv_format, 5, 3, 41, 2, hd, 7, 2500)
     _correct_case(akvs, dtype_t, kv_format, 3, 1, 2, 1, hd, 0, 0, seed=1)         # no probes, no query
     _correct_case(akvs, dtype_t, kv_format, 2, 20, 30, 2, hd, 3, 10000, seed=2)   # everything is a probe
 
 
-@pytest.mark.parametrize("kv_format", [0, 4, 2])
+@pytest.mark.parametrize("kv_format", [0, 4, 2, 8])
 def test_correct_layer_full_size(akvs, kv_format):
     """One layer at the 8B-class shapes (8 kv heads x 128, ~8k / ~12k context tokens)."""
     if kv_format == 0:

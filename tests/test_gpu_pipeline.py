@@ -134,6 +134,23 @@ def test_small16_quantised_cache(kv_format, dtype, scale):
     _run_all_modes(case, 2000, 1, units)           # check layer 1: scores are the quantisation error
 
 
+@pytest.mark.parametrize("dtype,scale", SMALL16)
+def test_small16_fp8_cache(dtype, scale):
+    """FP8 (E4M3) cache: the library's own bytes sit within one format step of the oracle's
+    (its K/V are 16-bit), then all modes with the oracle's bytes on both sides."""
+    case = Case(small16(dtype), std_scale=scale, kv_format=8)
+    case.encode()
+    units = case.oracle_units()
+    kq = np.concatenate([u["K"] for u in units], axis=1)
+    got = orc.e4m3_decode(case.store.k.cpu().numpy())
+    assert np.all(np.abs(got - kq) <= np.maximum(np.abs(kq) / 8, 2.0 ** -9) + 0.02 * np.abs(kq).max())
+    _run_all_modes(case, 2500, 2, units)
+    if dtype == "f16":
+        # check layer 1: the scores ARE the FP8 rounding error (a few percent of |v|), which bf16
+        # storage of the fresh rows (0.4 % of |v|) cannot resolve to 1e-2; float16 can
+        _run_all_modes(case, 2000, 1, units)
+
+
 def test_invariants_on_gpu():
     """100 % refresh equals full recompute; 0 % refresh equals naive reuse (GPU vs GPU)."""
     case = Case(small16("f16"), std_scale=4.0)
