@@ -209,6 +209,37 @@ def pack_codes(codes, bits):
     return out.astype(np.uint8)
 
 
+# --------------------------------------------------------------------------- residual diagnostics
+
+def residual_stats(fresh, reuse, ctx_off, sel=None, mu=None, w=None):
+    """Diagnostics of the residual model r_i = mu + xi_i (Section 3.4 and the appendix on
+    mean-explained energy), per unit u with tokens a..e-1 and residual rows r_i = fresh_i -
+    reuse_i (flattened over heads):
+
+        mean[u]      = sum_i sel_i r_i / sum_i sel_i      (sel = 1: the exact unit mean; sel =
+                       sample multiplicities: a probe-mean estimate; 0 where the sum is 0)
+        total[u]     = sum_i |r_i|^2
+        remaining[u] = sum_i |r_i - w_i mu[u]|^2          (mu = 0, w = 1 when not given)
+
+    The mean-explained energy of a correction vector is 1 - remaining / total."""
+    ctx_off = np.asarray(ctx_off, np.int64)
+    M, N = len(ctx_off) - 1, int(ctx_off[-1])
+    r = (np.asarray(fresh, np.float64) - np.asarray(reuse, np.float64)).reshape(N, -1)
+    D = r.shape[1]
+    sel = np.ones(N) if sel is None else np.asarray(sel, np.float64)
+    w = np.ones(N) if w is None else np.asarray(w, np.float64)
+    mu = np.zeros((M, D)) if mu is None else np.asarray(mu, np.float64).reshape(M, D)
+    mean, total, remaining = np.zeros((M, D)), np.zeros(M), np.zeros(M)
+    for u in range(M):
+        a, e = int(ctx_off[u]), int(ctx_off[u + 1])
+        ssum = sel[a:e].sum()
+        if ssum > 0:
+            mean[u] = (sel[a:e, None] * r[a:e]).sum(axis=0) / ssum
+        total[u] = (r[a:e] ** 2).sum()
+        remaining[u] = ((r[a:e] - w[a:e, None] * mu[u]) ** 2).sum()
+    return mean, total, remaining
+
+
 # --------------------------------------------------------------------------- FP8 cache
 
 E4M3_MAX = 448.0

@@ -331,3 +331,33 @@ def test_e4m3_matches_the_library_cast_and_is_monotone():
     assert np.all(np.diff(orc.e4m3_decode(orc.e4m3_encode(xs))) >= 0)
     assert np.array_equal(orc.e4m3_encode(ours), orc.e4m3_encode(x))
     assert np.all(np.abs(ours - x) <= np.maximum(np.abs(x) / 16, 2.0 ** -10))   # half a step of 3 mantissa bits
+
+
+# ----------------------------------------------------------------------------- residual diagnostics
+
+def test_residual_stats_closed_forms():
+    """(i) subtracting the exact mean leaves total - n |mean|^2 (the variance identity);
+    (ii) a residual that IS a per-unit constant is removed entirely; (iii) no correction
+    leaves everything; (iv) the selection weights form a weighted mean (hand-computed)."""
+    g = np.random.default_rng(3)
+    off = np.array([0, 5, 5, 12])                            # the middle unit is empty
+    fresh, reuse = g.standard_normal((12, 2, 4)), g.standard_normal((12, 2, 4))
+    mean, total, rem0 = orc.residual_stats(fresh, reuse, off)
+    assert np.allclose(rem0, total) and total[1] == 0 and np.all(mean[1] == 0)
+    _, _, rem = orc.residual_stats(fresh, reuse, off, mu=mean)
+    n = np.diff(off)
+    assert np.allclose(rem, total - n * (mean ** 2).sum(axis=1))
+    const = np.repeat(g.standard_normal((3, 8)), n, axis=0).reshape(12, 2, 4)
+    m2, t2, _ = orc.residual_stats(reuse + const, reuse, off)
+    _, _, r2 = orc.residual_stats(reuse + const, reuse, off, mu=m2)
+    assert np.allclose(r2, 0, atol=1e-20) and np.allclose(t2, n * (m2 ** 2).sum(axis=1))
+    # weighted mean by hand: unit 0, weights 2,0,1,0,0 -> (2 r0 + r2) / 3
+    sel = np.zeros(12)
+    sel[[0, 2]] = [2, 1]
+    m3, _, _ = orc.residual_stats(fresh, reuse, off, sel=sel)
+    r = (fresh - reuse).reshape(12, 8)
+    assert np.allclose(m3[0], (2 * r[0] + r[2]) / 3) and np.all(m3[2] == 0)
+    # per-token weights scale the subtracted vector
+    w = g.random(12)
+    _, _, r4 = orc.residual_stats(fresh, reuse, off, mu=mean, w=w)
+    assert np.isclose(r4[2], sum(((r[i] - w[i] * mean[2]) ** 2).sum() for i in range(5, 12)))
