@@ -279,6 +279,26 @@ int32_t akvs_op_correct_layer(int32_t dtype, int32_t kv_format,
                               void* out_k, void* out_v, float* mu_k, float* mu_v,
                               void* scratch, void* stream);
 
+/* Diagnostics of the residual model r_i = mu + xi_i (Section 3.4; the appendix's mean-explained
+ * residual energy), for one layer of one request.  fresh_k / fresh_v: device [N][n_kv][hd],
+ * the fresh K (rotated at global positions) and V of EVERY context token, e.g. from
+ * AKVS_MODE_FULL; the cache arguments as in akvs_op_correct_layer; ctx_off: host [n_units+1].
+ * Per unit u and per K | V, with r_i = fresh_i - reuse_i (K re-aligned to the unit's offset):
+ *   mean[u]   = sum_i sel_i r_i / sum_i sel_i   (sel NULL: 1 -> the exact unit mean; sample
+ *               multiplicities -> a probe-mean estimate with replacement; 0 if the sum is 0)
+ *   energy[u] = { sum_i |r_i^K|^2, sum_i |r_i^K - w_i^K mu_K[u]|^2, the same two for V }
+ * mu_k / mu_v: device [n_units][n_kv*hd] or both NULL (zero); w_k / w_v: device [N] or NULL (1);
+ * sel_k / sel_v: device [N] or NULL; mean_k / mean_v: device [n_units][n_kv*hd] outputs or both
+ * NULL; energy: device [n_units][4] float.  The mean-explained energy of a correction vector is
+ * 1 - remaining / total.  scratch: akvs_op_scratch_bytes(N, 0, n_units, head_dim) bytes.
+ * Returns AKVS_ERR_TOO_LARGE when n_kv * hd exceeds 4096. */
+int32_t akvs_op_residual_stats(int32_t dtype, int32_t kv_format, const void* cache_k, const void* cache_v,
+                               const void* k_meta, const void* v_meta, const int32_t* src_tok, const void* fresh_k,
+                               const void* fresh_v, const int32_t* ctx_off, int32_t n_units, int32_t n_kv_heads,
+                               int32_t head_dim, float rope_base, const float* sel_k, const float* sel_v,
+                               const float* mu_k, const float* mu_v, const float* w_k, const float* w_v, float* mean_k,
+                               float* mean_v, float* energy, void* scratch, void* stream);
+
 /* Group quantiser of the cache (asymmetric min-max, groups of 64 along head_dim, float16
  * scale and minimum): x [n][n_kv][hd] -> codes [n][n_kv][hd*bits/8], meta half2 [n][n_kv][hd/64].
  * bits = 8 is the FP8 (E4M3) cast: one byte per value, meta unused (may be NULL). */

@@ -26,7 +26,7 @@ EXPORTS = ["akvs_workspace_bytes", "akvs_debug_set_linear_algo", "akvs_launch_co
            "akvs_prof_reset", "akvs_prof_read", "akvs_encode_units", "akvs_select_probes", "akvs_prefill_corrected",
            "akvs_free", "akvs_check", "akvs_op_linear", "akvs_op_rope", "akvs_op_attention",
            "akvs_op_scratch_bytes", "akvs_op_select", "akvs_op_select_static", "akvs_op_correct_layer",
-           "akvs_op_quantize"]
+           "akvs_op_quantize", "akvs_op_residual_stats"]
 STATIC_MAX_CTX, STATIC_MAX_UNITS = 16384, 1024
 
 
@@ -409,6 +409,26 @@ def op_correct_layer(dtype, kv_format, cache_k, cache_v, k_meta, v_meta, src_tok
                                    n_query, n_kv, hd, C.c_float(base), _ptr(out_k), _ptr(out_v), _ptr(mu_k),
                                    _ptr(mu_v), _ptr(scratch), _stream()), "akvs_op_correct_layer")
     return out_k, out_v, mu_k, mu_v
+
+
+def op_residual_stats(dtype, kv_format, cache_k, cache_v, k_meta, v_meta, src_tok, fresh_k, fresh_v, ctx_off, n_kv, hd,
+                      base, sel_k=None, sel_v=None, mu_k=None, mu_v=None, w_k=None, w_v=None):
+    """Unit means of the residual (under selection weights) and total / remaining residual energy.
+    Returns (mean_k, mean_v [M][n_kv*hd], energy [M][4] = K total, K remaining, V total, V remaining)."""
+    M = len(ctx_off) - 1
+    N = int(ctx_off[-1])
+    dev_ = fresh_k.device
+    off = (C.c_int32 * (M + 1))(*[int(x) for x in ctx_off])
+    mean_k = torch.zeros((M, n_kv * hd), dtype=torch.float32, device=dev_)
+    mean_v = torch.zeros_like(mean_k)
+    energy = torch.zeros((M, 4), dtype=torch.float32, device=dev_)
+    scratch = op_scratch(N, 0, M, hd, dev_)
+    _chk(lib.akvs_op_residual_stats(dtype, kv_format, _ptr(cache_k), _ptr(cache_v), _ptr(k_meta), _ptr(v_meta),
+                                    _ptr(src_tok), _ptr(fresh_k), _ptr(fresh_v), off, M, n_kv, hd, C.c_float(base),
+                                    _ptr(sel_k), _ptr(sel_v), _ptr(mu_k), _ptr(mu_v), _ptr(w_k), _ptr(w_v),
+                                    _ptr(mean_k), _ptr(mean_v), _ptr(energy), _ptr(scratch), _stream()),
+         "akvs_op_residual_stats")
+    return mean_k, mean_v, energy
 
 
 def op_quantize(x, bits):

@@ -852,6 +852,31 @@ int32_t akvs_op_correct_layer(int32_t dtype, int32_t kv_format, const void* cach
                         probes->n_probe_rows, n_kv_heads, head_dim, table, out_k, out_v, st);
 }
 
+int32_t akvs_op_residual_stats(int32_t dtype, int32_t kv_format, const void* cache_k, const void* cache_v,
+                               const void* k_meta, const void* v_meta, const int32_t* src_tok, const void* fresh_k,
+                               const void* fresh_v, const int32_t* ctx_off_host, int32_t n_units, int32_t n_kv_heads,
+                               int32_t head_dim, float rope_base, const float* sel_k, const float* sel_v,
+                               const float* mu_k, const float* mu_v, const float* w_k, const float* w_v, float* mean_k,
+                               float* mean_v, float* energy, void* scratch, void* stream) {
+  if (!ctx_off_host || !energy || !scratch || n_units < 0) return AKVS_ERR_INVALID_ARG;
+  if ((mu_k == nullptr) != (mu_v == nullptr) || (mean_k == nullptr) != (mean_v == nullptr)) return AKVS_ERR_INVALID_ARG;
+  if (dtype != AKVS_F32 && dtype != AKVS_BF16 && dtype != AKVS_F16) return AKVS_ERR_UNSUPPORTED;
+  if (ctx_off_host[0] != 0) return AKVS_ERR_SHAPE;
+  for (int u = 0; u < n_units; ++u)
+    if (ctx_off_host[u + 1] < ctx_off_host[u]) return AKVS_ERR_SHAPE;
+  const int N = ctx_off_host[n_units];
+  if (N > 0 && (!cache_k || !cache_v || !src_tok || !fresh_k || !fresh_v)) return AKVS_ERR_INVALID_ARG;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  Carver c(scratch);
+  int32_t* ctx_off = c.take<int32_t>(n_units + 1);
+  float2* table = c.take<float2>((int64_t)N * (head_dim / 2));
+  AKVS_CUDA(cudaMemcpyAsync(ctx_off, ctx_off_host, (n_units + 1) * sizeof(int32_t), cudaMemcpyHostToDevice, st));
+  AKVS_TRY(launch_rope_table(rope_base, head_dim, N, table, st));
+  KvLayer kv{cache_k, cache_v, k_meta, v_meta, kv_format};
+  return launch_residual_stats(dtype, kv, ctx_off, src_tok, fresh_k, fresh_v, n_units, n_kv_heads, head_dim, table,
+                               sel_k, sel_v, mu_k, mu_v, w_k, w_v, mean_k, mean_v, energy, st);
+}
+
 int32_t akvs_op_quantize(int32_t dtype, const void* x, int32_t n, int32_t n_kv_heads, int32_t head_dim, int32_t bits,
                          void* codes, void* meta, void* stream) {
   if (!x || !codes || (!meta && bits != AKVS_KV_FP8) || n < 0) return AKVS_ERR_INVALID_ARG;

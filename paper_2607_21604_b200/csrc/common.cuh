@@ -239,6 +239,11 @@ int32_t launch_select(const float* d_k, const float* d_v, const int32_t* ctx_off
 int32_t launch_offsets(int dtype, const KvLayer& kv, const ReqMaps& maps, const int32_t* probe_off,
                        const int32_t* sk_idx, const int32_t* sv_idx, const void* k_fresh, const void* v_fresh, int M,
                        int n_kv, int hd, const float2* table, float* mu_k, float* mu_v, cudaStream_t st);
+int32_t launch_residual_stats(int dtype, const KvLayer& kv, const int32_t* ctx_off, const int32_t* tok_src,
+                              const void* k_fresh, const void* v_fresh, int M, int n_kv, int hd, const float2* table,
+                              const float* sel_k, const float* sel_v, const float* mu_k, const float* mu_v,
+                              const float* w_k, const float* w_v, float* mean_k, float* mean_v, float* energy,
+                              cudaStream_t st);
 int32_t launch_correct(int dtype, const KvLayer& kv, const ReqMaps& maps, const void* k_fresh, const void* v_fresh,
                        const float* w_k, const float* w_v, const float* mu_k, const float* mu_v, int N, int n_query,
                        int n_probe_rows, int n_kv, int hd, const float2* table, void* out_k, void* out_v,

@@ -665,3 +665,142 @@ int32_t launch_correct(int dtype, const KvLayer& kv, const ReqMaps& maps, const 
     });
   });
 }
+
+// ---------------------------------------------------------------------------------------
+// Diagnostics of the residual model r_i = mu + xi_i (Section 3.4; the appendix's mean-explained
+// energy): per unit and per K | V, over ALL tokens of the unit (fresh K/V of every context row
+// come from a full recompute),
+//   mean      = sum_i sel_i r_i / sum_i sel_i
+//   total     = sum_i |r_i|^2,   remaining = sum_i |r_i - w_i mu|^2
+// One CTA per (unit, K | V); a thread owns RS_PAIRS rotation pairs of the row and walks the
+// unit's tokens in order (fixed summation order), so the per-dimension sums stay in registers.
+// ---------------------------------------------------------------------------------------
+constexpr int RS_THREADS = 256, RS_PAIRS = 8;
+
+template <typename T, int FMT>
+__global__ void __launch_bounds__(RS_THREADS)
+residual_stats_kernel(KvLayer kv, const int32_t* __restrict__ ctx_off, const int32_t* __restrict__ tok_src,
+                      const T* __restrict__ k_fresh, const T* __restrict__ v_fresh, int n_kv, int hd,
+                      const float2* __restrict__ table, const float* __restrict__ sel_k,
+                      const float* __restrict__ sel_v, const float* __restrict__ mu_k, const float* __restrict__ mu_v,
+                      const float* __restrict__ w_k, const float* __restrict__ w_v, float* __restrict__ mean_k,
+                      float* __restrict__ mean_v, float* __restrict__ energy) {
+  __shared__ double red[2][RS_THREADS / 32];
+  const int u = blockIdx.x, is_v = blockIdx.y;
+  const int half = hd / 2, P = n_kv * half;
+  const int a = ctx_off[u], e = ctx_off[u + 1];
+  const T* fresh = is_v ? v_fresh : k_fresh;
+  const void* cbase = is_v ? kv.v : kv.k;
+  const void* cmeta = is_v ? kv.v_meta : kv.k_meta;
+  const float* sel = is_v ? sel_v : sel_k;
+  const float* mu = is_v ? mu_v : mu_k;
+  const float* w = is_v ? w_v : w_k;
+  const float2* rot = table + (size_t)a * half;           // a single request: the unit starts at position a
+  float s_lo[RS_PAIRS], s_hi[RS_PAIRS], m_lo[RS_PAIRS], m_hi[RS_PAIRS];
+#pragma unroll
+  for (int i = 0; i < RS_PAIRS; ++i) {
+    s_lo[i] = s_hi[i] = 0.f;
+    const int p = threadIdx.x + i * RS_THREADS;
+    const int h = p / half, d = p - h * half;
+    m_lo[i] = mu && p < P ? mu[((size_t)u * n_kv + h) * hd + d] : 0.f;
+    m_hi[i] = mu && p < P ? mu[((size_t)u * n_kv + h) * hd + half + d] : 0.f;
+  }
+  double tot = 0.0, rem = 0.0;
+  float ssum = 0.f;
+  for (int j = a; j < e; ++j) {
+    const int64_t src = tok_src[j];
+    const float sj = sel ? sel[j] : 1.f, wj = w ? w[j] : 1.f;
+    ssum += sj;
+    float t_acc = 0.f, r_acc = 0.f;
+#pragma unroll
+    for (int i = 0; i < RS_PAIRS; ++i) {
+      const int p = threadIdx.x + i * RS_THREADS;
+      if (p >= P) break;
+      const int h = p / half, d = p - h * half;
+      float lo[1], hi[1];
+      {
+        // scalar decode of elements d and half + d of head h (every cache format)
+        if constexpr (FMT == AKVS_KV_NATIVE) {
+          const T* cp = reinterpret_cast<const T*>(cbase) + ((size_t)src * n_kv + h) * hd;
+          lo[0] = to_f(cp[d]);
+          hi[0] = to_f(cp[half + d]);
+        } else if constexpr (FMT == AKVS_KV_FP8) {
+          const uint8_t* cp = reinterpret_cast<const uint8_t*>(cbase) + ((size_t)src * n_kv + h) * hd;
+          const __half_raw ra = __nv_cvt_fp8_to_halfraw(cp[d], __NV_E4M3), rb = __nv_cvt_fp8_to_halfraw(cp[half + d], __NV_E4M3);
+          lo[0] = __half2float(*reinterpret_cast<const __half*>(&ra));
+          hi[0] = __half2float(*reinterpret_cast<const __half*>(&rb));
+        } else {
+          const uint8_t* cp = reinterpret_cast<const uint8_t*>(cbase) + ((size_t)src * n_kv + h) * hd * FMT / 8;
+          const __half2* mp = reinterpret_cast<const __half2*>(cmeta) + ((size_t)src * n_kv + h) * (hd / 64);
+          const int d2 = half + d;
+          const uint32_t qa = (cp[d * FMT / 8] >> ((d * FMT) & 7)) & ((1u << FMT) - 1u);
+          const uint32_t qb = (cp[d2 * FMT / 8] >> ((d2 * FMT) & 7)) & ((1u << FMT) - 1u);
+          const __half2 ma = mp[d / 64], mb = mp[d2 / 64];
+          lo[0] = __fmaf_rn((float)qa, __low2float(ma), __high2float(ma));
+          hi[0] = __fmaf_rn((float)qb, __low2float(mb), __high2float(mb));
+        }
+      }
+      if (!is_v) {
+        const float2 t = rot[d];
+        const float rl = lo[0] * t.x - hi[0] * t.y, rh = hi[0] * t.x + lo[0] * t.y;
+        lo[0] = rl;
+        hi[0] = rh;
+      }
+      const T* fp = fresh + ((size_t)j * n_kv + h) * hd;
+      const float r_lo = to_f(fp[d]) - lo[0], r_hi = to_f(fp[half + d]) - hi[0];
+      s_lo[i] = fmaf(sj, r_lo, s_lo[i]);
+      s_hi[i] = fmaf(sj, r_hi, s_hi[i]);
+      t_acc += r_lo * r_lo + r_hi * r_hi;
+      const float c_lo = r_lo - wj * m_lo[i], c_hi = r_hi - wj * m_hi[i];
+      r_acc += c_lo * c_lo + c_hi * c_hi;
+    }
+    tot += (double)t_acc;
+    rem += (double)r_acc;
+  }
+  float* mean = is_v ? mean_v : mean_k;
+  if (mean) {
+    const float inv = ssum > 0.f ? 1.f / ssum : 0.f;
+#pragma unroll
+    for (int i = 0; i < RS_PAIRS; ++i) {
+      const int p = threadIdx.x + i * RS_THREADS;
+      if (p >= P) break;
+      const int h = p / half, d = p - h * half;
+      mean[((size_t)u * n_kv + h) * hd + d] = s_lo[i] * inv;
+      mean[((size_t)u * n_kv + h) * hd + half + d] = s_hi[i] * inv;
+    }
+  }
+  // block sums in a fixed order: lanes by shuffle, warps by thread 0
+  for (int o = 16; o > 0; o >>= 1) {
+    tot += __shfl_down_sync(0xFFFFFFFFu, tot, o);
+    rem += __shfl_down_sync(0xFFFFFFFFu, rem, o);
+  }
+  if ((threadIdx.x & 31) == 0) { red[0][threadIdx.x >> 5] = tot; red[1][threadIdx.x >> 5] = rem; }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    double t2 = 0.0, r2 = 0.0;
+    for (int i = 0; i < RS_THREADS / 32; ++i) { t2 += red[0][i]; r2 += red[1][i]; }
+    energy[(size_t)u * 4 + is_v * 2] = (float)t2;
+    energy[(size_t)u * 4 + is_v * 2 + 1] = (float)r2;
+  }
+}
+
+int32_t launch_residual_stats(int dtype, const KvLayer& kv, const int32_t* ctx_off, const int32_t* tok_src,
+                              const void* k_fresh, const void* v_fresh, int M, int n_kv, int hd, const float2* table,
+                              const float* sel_k, const float* sel_v, const float* mu_k, const float* mu_v,
+                              const float* w_k, const float* w_v, float* mean_k, float* mean_v, float* energy,
+                              cudaStream_t st) {
+  if (M == 0) return AKVS_OK;
+  AKVS_TRY(check_kv_shape(dtype, kv, hd));
+  if (n_kv * (hd / 2) > RS_THREADS * RS_PAIRS) return AKVS_ERR_TOO_LARGE;
+  const dim3 grid(M, 2);
+  return dispatch_dtype(dtype, [&](auto tag) -> int32_t {
+    using T = decltype(tag);
+    return dispatch_fmt(kv.fmt, [&](auto f) -> int32_t {
+      residual_stats_kernel<T, decltype(f)::value><<<grid, RS_THREADS, 0, st>>>(
+          kv, ctx_off, tok_src, (const T*)k_fresh, (const T*)v_fresh, n_kv, hd, table, sel_k, sel_v, mu_k, mu_v, w_k,
+          w_v, mean_k, mean_v, energy);
+      AKVS_LAUNCHED();
+      return AKVS_OK;
+    });
+  });
+}

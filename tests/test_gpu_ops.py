@@ -317,3 +317,67 @@ def test_correct_layer_full_size(akvs, kv_format):
     else:
         N = _correct_case(akvs, torch.float16, kv_format, 48, 256, 256, 8, 128, 128, 2000, seed=4)
     assert N > 6000
+
+
+# ----------------------------------------------------------------------------- residual diagnostics
+
+@pytest.mark.parametrize("dtype_t,kv_format,nkv,hd", [(torch.float32, 0, 2, 64), (torch.float16, 0, 8, 128),
+                                                      (torch.float16, 4, 2, 128), (torch.bfloat16, 8, 2, 64)])
+def test_residual_stats_op(akvs, dtype_t, kv_format, nkv, hd):
+    """Unit means under selection weights and total / remaining residual energy against the oracle:
+    exact mean (sel = 1), a with-replacement sample (multiplicities), weighted correction."""
+    g = np.random.default_rng(11)
+    lens = np.array([37, 0, 5, 64, 1])
+    off = np.concatenate([[0], np.cumsum(lens)]).astype(np.int64)
+    N, M = int(off[-1]), len(lens)
+    src = g.permutation(N).astype(np.int32)                 # store rows in another order
+    ck = g.standard_normal((N, nkv, hd)).astype(np.float32)
+    cv = g.standard_normal((N, nkv, hd)).astype(np.float32)
+    dt = {torch.float32: akvs.F32, torch.bfloat16: akvs.BF16, torch.float16: akvs.F16}[dtype_t]
+    km = vm = None
+    if kv_format == 0:
+        ck_t, cv_t = dev(ck, dtype_t), dev(cv, dtype_t)
+        ck_ref, cv_ref = n64(ck_t), n64(cv_t)
+    elif kv_format == 8:
+        kc, vc = orc.e4m3_encode(ck), orc.e4m3_encode(cv)
+        ck_t, cv_t = dev(kc), dev(vc)
+        ck_ref, cv_ref = orc.e4m3_decode(kc), orc.e4m3_decode(vc)
+    else:
+        kc, ks, kmn = orc.quantize_groups(ck, kv_format)
+        vc, vs, vmn = orc.quantize_groups(cv, kv_format)
+        ck_t, cv_t = dev(orc.pack_codes(kc, kv_format)), dev(orc.pack_codes(vc, kv_format))
+        km, vm = dev(np.stack([ks, kmn], -1)), dev(np.stack([vs, vmn], -1))
+        ck_ref = orc.dequantize_groups(kc, ks, kmn).astype(np.float64)
+        cv_ref = orc.dequantize_groups(vc, vs, vmn).astype(np.float64)
+    inv = np.empty(N, np.int64)
+    inv[src] = np.arange(N)
+    st = lambda t: t[dev(inv)].contiguous() if t is not None else None
+    # fresh = reuse + a unit offset + noise, so that the mean explains part of the energy
+    kr = np.concatenate([orc.rope_rotate(ck_ref[off[u]:off[u + 1]], np.full(lens[u], off[u]), 1e4) for u in range(M)])
+    shift = np.repeat(g.standard_normal((M, nkv, hd)), lens, axis=0)
+    fk_t = dev((kr + shift + 0.5 * g.standard_normal(kr.shape)).astype(np.float32), dtype_t)
+    fv_t = dev((cv_ref + 0.7 * shift + 0.5 * g.standard_normal(kr.shape)).astype(np.float32), dtype_t)
+    fk, fv = n64(fk_t), n64(fv_t)
+    sel = np.bincount(np.concatenate([off[u] + g.integers(0, lens[u], max(1, lens[u] // 8))
+                                      for u in range(M) if lens[u] > 0]), minlength=N).astype(np.float32)
+    w = g.random(N).astype(np.float32)
+    args = (dt, kv_format, st(ck_t), st(cv_t), st(km), st(vm), dev(src), fk_t, fv_t, off, nkv, hd, 1e4)
+    tol = 2e-5
+
+    def check(got, ref_k, ref_v):
+        mk, mv, en = got
+        en = n64(en)
+        assert np.allclose(n64(mk), ref_k[0], rtol=tol, atol=tol) and np.allclose(n64(mv), ref_v[0], rtol=tol, atol=tol)
+        assert np.allclose(en[:, 0], ref_k[1], rtol=tol) and np.allclose(en[:, 1], ref_k[2], rtol=tol, atol=1e-6)
+        assert np.allclose(en[:, 2], ref_v[1], rtol=tol) and np.allclose(en[:, 3], ref_v[2], rtol=tol, atol=1e-6)
+
+    exact = akvs.op_residual_stats(*args)
+    check(exact, orc.residual_stats(fk, kr, off), orc.residual_stats(fv, cv_ref, off))
+    # subtract the exact mean the op just returned; means from a sample with replacement
+    mu_k, mu_v = n64(exact[0]), n64(exact[1])
+    got = akvs.op_residual_stats(*args, sel_k=dev(sel), sel_v=dev(sel), mu_k=exact[0], mu_v=exact[1])
+    check(got, orc.residual_stats(fk, kr, off, sel=sel, mu=mu_k), orc.residual_stats(fv, cv_ref, off, sel=sel, mu=mu_v))
+    assert np.all(n64(got[2])[:, 1] <= n64(got[2])[:, 0] + 1e-6)          # the exact mean never adds energy
+    # per-token weights on the subtracted vector (the method's w = min(d, 1))
+    got = akvs.op_residual_stats(*args, mu_k=exact[0], mu_v=exact[1], w_k=dev(w), w_v=dev(w))
+    check(got, orc.residual_stats(fk, kr, off, mu=mu_k, w=w), orc.residual_stats(fv, cv_ref, off, mu=mu_v, w=w))
