@@ -102,6 +102,24 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
   float* m_part = m_ref + 3 * 128;                                // [2][128]
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  pdl_trigger();
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < B_COUNT; ++i) {
+      int count = 1;
+      if (i == B_QFULL || i == B_PFULL || (i >= B_SEMPTY && i < B_SEMPTY + 2)) count = 4;   // the warps of a group
+      if (i >= B_FIN && i < B_FIN + 4) count = 2;                                           // one warp of each group
+      tc::mbar_init(&bar[i], count);
+    }
+    *abort_flag = 0;
+    tc::fence_barrier_init();
+    tc::fence_proxy_async();
+  }
+  if (threadIdx.x < 128) m_ref[threadIdx.x] = -1.0e30f;
+  if (warp == 1) {
+    tc::tmem_alloc(tmem_slot, 512);
+    tc::tmem_relinquish();
+  }
+  pdl_wait();                       // the key ranges below are the first global memory this kernel reads
   // 1-D grid, kv head fastest: CTAs are handed out longest row block first across ALL heads
   // (the last rows see the most keys), so the tail of the launch is made of short CTAs
   const int hk = blockIdx.x % p.n_kv;
@@ -128,22 +146,6 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
   // first key of tile j
   auto tile_key = [&](int j) { return j < n_tiles1 ? key_lo + j * BN : key_lo2 + (j - n_tiles1) * BN; };
 
-  if (threadIdx.x == 0) {
-    for (int i = 0; i < B_COUNT; ++i) {
-      int count = 1;
-      if (i == B_QFULL || i == B_PFULL || (i >= B_SEMPTY && i < B_SEMPTY + 2)) count = 4;   // the warps of a group
-      if (i >= B_FIN && i < B_FIN + 4) count = 2;                                           // one warp of each group
-      tc::mbar_init(&bar[i], count);
-    }
-    *abort_flag = 0;
-    tc::fence_barrier_init();
-    tc::fence_proxy_async();
-  }
-  if (threadIdx.x < 128) m_ref[threadIdx.x] = -1.0e30f;
-  if (warp == 1) {
-    tc::tmem_alloc(tmem_slot, 512);
-    tc::tmem_relinquish();
-  }
   tc::fence_before_sync();
   __syncthreads();
   tc::fence_after_sync();
@@ -435,8 +437,8 @@ int32_t launch_attention_tc(int dtype, const void* q, const void* k, const void*
   const dim3 grid((unsigned)p.row_blocks * n_kv);
   double flops = 0;   // filled by the caller's accounting when profiling attention
   ProfScope prof(3, 0, flops, st);
-  if (dtype == AKVS_BF16) attention_tc_kernel<bf16><<<grid, ATT_THREADS, ATT_SMEM, st>>>(tmK, tmV, p);
-  else attention_tc_kernel<f16><<<grid, ATT_THREADS, ATT_SMEM, st>>>(tmK, tmV, p);
+  if (dtype == AKVS_BF16) AKVS_CUDA(launch_pdl(attention_tc_kernel<bf16>, grid, dim3(ATT_THREADS), ATT_SMEM, st, tmK, tmV, p));
+  else AKVS_CUDA(launch_pdl(attention_tc_kernel<f16>, grid, dim3(ATT_THREADS), ATT_SMEM, st, tmK, tmV, p));
   AKVS_LAUNCHED();
   return AKVS_OK;
 }

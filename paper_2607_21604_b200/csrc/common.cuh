@@ -165,6 +165,32 @@ __device__ __forceinline__ float warp_min(float v) {
   return v;
 }
 
+// Programmatic dependent launch: a kernel launched with launch_pdl() may be scheduled while
+// the kernel before it in the stream is still draining, so that its launch latency and its
+// local prologue (barrier set-up, tensor-memory allocation, descriptor prefetch) overlap the
+// predecessor's tail.  Such a kernel calls pdl_trigger() first thing (its own successor may be
+// scheduled as soon as SM resources free up) and pdl_wait() before its first access to global
+// memory that an earlier kernel may have written or may still read: the wait returns when every
+// earlier kernel has completed and its writes are visible.  Both are no-ops under a plain launch.
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+static inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                                     Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 // Device status word: first error wins.
 __device__ __forceinline__ void set_status(int32_t* status, int32_t code) {
   if (status) atomicCAS(status, 0, code);

@@ -359,6 +359,8 @@ offsets_kernel(KvLayer kv, ReqMaps maps, const int32_t* __restrict__ probe_off, 
                const int32_t* __restrict__ sv_idx, const T* __restrict__ k_fresh, const T* __restrict__ v_fresh,
                int n_kv, int hd, const float2* __restrict__ table, float* __restrict__ mu_k, float* __restrict__ mu_v) {
   extern __shared__ float part[];                 // [OFF_WARPS][hd]
+  pdl_trigger();
+  pdl_wait();
   const int u = blockIdx.x, h = blockIdx.y, is_v = blockIdx.z;
   const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
   const int half = hd / 2;
@@ -427,8 +429,8 @@ int32_t launch_offsets(int dtype, const KvLayer& kv, const ReqMaps& maps, const 
   return dispatch_dtype(dtype, [&](auto tag) -> int32_t {
     using T = decltype(tag);
     return dispatch_fmt(kv.fmt, [&](auto f) -> int32_t {
-      offsets_kernel<T, T, decltype(f)::value><<<grid, OFF_WARPS * 32, smem, st>>>(
-          kv, maps, probe_off, sk_idx, sv_idx, (const T*)k_fresh, (const T*)v_fresh, n_kv, hd, table, mu_k, mu_v);
+      AKVS_CUDA(launch_pdl(offsets_kernel<T, T, decltype(f)::value>, grid, dim3(OFF_WARPS * 32), smem, st, kv, maps,
+                           probe_off, sk_idx, sv_idx, (const T*)k_fresh, (const T*)v_fresh, n_kv, hd, table, mu_k, mu_v));
       AKVS_LAUNCHED();
       return AKVS_OK;
     });
@@ -549,6 +551,8 @@ correct_kernel(KvLayer kv, ReqMaps maps, const T* __restrict__ k_fresh, const T*
                const float* __restrict__ mu_v, int N, int T_tok, int n_probe_rows, int n_kv, int hd,
                const float2* __restrict__ table, T* __restrict__ out_k, T* __restrict__ out_v) {
   constexpr int V = VecOf<T>::N;
+  pdl_trigger();
+  pdl_wait();
   const int half = hd / 2, ch = half / V;
   const int groups = (T_tok + COR_TOK - 1) / COR_TOK;
   const int total = groups * n_kv * ch;                 // < 2^31: checked by the launcher
@@ -657,9 +661,9 @@ int32_t launch_correct(int dtype, const KvLayer& kv, const ReqMaps& maps, const 
   return dispatch_dtype(dtype, [&](auto tag) -> int32_t {
     using T = decltype(tag);
     return dispatch_fmt(kv.fmt, [&](auto f) -> int32_t {
-      correct_kernel<T, T, decltype(f)::value><<<grid, 256, 0, st>>>(kv, maps, (const T*)k_fresh, (const T*)v_fresh, w_k,
-                                                                    w_v, mu_k, mu_v, N, T_tok, n_probe_rows, n_kv, hd,
-                                                                    table, (T*)out_k, (T*)out_v);
+      AKVS_CUDA(launch_pdl(correct_kernel<T, T, decltype(f)::value>, dim3(grid), dim3(256), 0, st, kv, maps,
+                           (const T*)k_fresh, (const T*)v_fresh, w_k, w_v, mu_k, mu_v, N, T_tok, n_probe_rows, n_kv, hd,
+                           table, (T*)out_k, (T*)out_v));
       AKVS_LAUNCHED();
       return AKVS_OK;
     });

@@ -73,6 +73,8 @@ constexpr int RMS_MAX_V = 8;           // float4 per thread: d <= 8192
 template <typename TO>
 __global__ void __launch_bounds__(RMS_THREADS)
 rmsnorm_kernel(const float* __restrict__ h, const float* __restrict__ gain, float eps, int d, TO* __restrict__ x) {
+  pdl_trigger();
+  pdl_wait();
   const int r = blockIdx.x;
   const float4* hp = reinterpret_cast<const float4*>(h + (size_t)r * d);
   const float4* gp = reinterpret_cast<const float4*>(gain);
@@ -121,7 +123,7 @@ int32_t launch_rmsnorm(int out_dtype, const float* h, const float* gain, float e
   if (d % 4 != 0 || d > RMS_THREADS * 4 * RMS_MAX_V) return AKVS_ERR_UNSUPPORTED;
   return dispatch_dtype(out_dtype, [&](auto tag) -> int32_t {
     using T = decltype(tag);
-    rmsnorm_kernel<T><<<n, RMS_THREADS, 0, st>>>(h, gain, eps, d, (T*)x);
+    AKVS_CUDA(launch_pdl(rmsnorm_kernel<T>, dim3(n), dim3(RMS_THREADS), 0, st, h, gain, eps, d, (T*)x));
     AKVS_LAUNCHED();
     return AKVS_OK;
   });

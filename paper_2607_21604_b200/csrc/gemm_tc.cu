@@ -69,6 +69,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int KB = (p.K + BK - 1) / BK;
   const int n_tiles = p.tiles_m * p.tiles_n;
+  pdl_trigger();
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < STAGES; ++i) { tc::mbar_init(&full[i], 1); tc::mbar_init(&empty[i], 1); }
@@ -85,6 +86,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   __syncthreads();
   tc::fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
+  pdl_wait();                       // everything above touched only this CTA's own state
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
@@ -383,7 +385,8 @@ int32_t launch_linear_tc(int dtype, int epi, const void* x, int M, int K, int n_
   for (int i = 0; i < n_seg; ++i) flops += 2.0 * M * (double)n[i] * K;
   ProfScope prof(1, epi, flops, st);
   if (epi < 0 || epi > 2) return AKVS_ERR_INVALID_ARG;
-#define AKVS_GEMM_LAUNCH(E, T) gemm_tc_kernel<E, T><<<grid, THREADS, SMEM_BYTES, st>>>(tmA, tmB[0], tmB[1], tmB[2], p)
+#define AKVS_GEMM_LAUNCH(E, T) \
+  AKVS_CUDA(launch_pdl(gemm_tc_kernel<E, T>, dim3(grid), dim3(THREADS), SMEM_BYTES, st, tmA, tmB[0], tmB[1], tmB[2], p))
   if (dtype == AKVS_BF16) {
     if (epi == EPI_STORE) AKVS_GEMM_LAUNCH(EPI_STORE, bf16);
     else if (epi == EPI_RESID) AKVS_GEMM_LAUNCH(EPI_RESID, bf16);
