@@ -69,6 +69,9 @@ class ClockSampler:
     def mark(self):
         """The timed region starts now (the sampler itself was started earlier: nvidia-smi takes
         a few hundred ms to deliver its first line)."""
+        deadline = time.time() + 2.0
+        while self.p is not None and not self.rows and time.time() < deadline:
+            time.sleep(0.02)
         self.t0 = time.time()
 
     def stop(self):

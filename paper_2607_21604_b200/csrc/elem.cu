@@ -157,6 +157,8 @@ template <typename T>
 __global__ void rope_kernel(T* __restrict__ x, const int32_t* __restrict__ pos, int n, int n_heads, int hd, int ld,
                             const float2* __restrict__ table, double base) {
   constexpr int V = VecOf<T>::N;
+  pdl_trigger();
+  pdl_wait();
   const int half = hd / 2, ch = half / V;
   const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (idx >= (int64_t)n * n_heads * ch) return;
@@ -199,7 +201,7 @@ int32_t launch_rope(int dtype, void* x, const int32_t* pos, int n, int n_heads, 
   const int blocks = akvs_cdiv(total, 256);
   return dispatch_dtype(dtype, [&](auto tag) -> int32_t {
     using T = decltype(tag);
-    rope_kernel<T><<<blocks, 256, 0, st>>>((T*)x, pos, n, n_heads, hd, ld, table, (double)base);
+    AKVS_CUDA(launch_pdl(rope_kernel<T>, dim3(blocks), dim3(256), 0, st, (T*)x, pos, n, n_heads, hd, ld, table, (double)base));
     AKVS_LAUNCHED();
     return AKVS_OK;
   });

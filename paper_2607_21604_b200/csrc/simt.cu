@@ -14,6 +14,8 @@ __global__ void __launch_bounds__(256)
 linear_simt_kernel(const T* __restrict__ x, const TW* __restrict__ w, const TW* __restrict__ w2, T* __restrict__ y,
                    float* __restrict__ resid, int M, int N, int K, int ldy) {
   __shared__ float xs[SG_BK][SG_BM + 4];
+  pdl_trigger();
+  pdl_wait();
   __shared__ float ws[SG_BK][SG_BN + 4];
   __shared__ float ws2[DUAL ? SG_BK : 1][SG_BN + 4];
   const int m0 = blockIdx.y * SG_BM, n0 = blockIdx.x * SG_BN;
@@ -70,8 +72,8 @@ int32_t launch_linear_simt(int dtype, const void* x, const void* w, const void* 
   const dim3 grid(akvs_cdiv(N, SG_BN), akvs_cdiv(M, SG_BM));
   return dispatch_dtype(dtype, [&](auto tag) -> int32_t {
     using T = decltype(tag);
-    if (w2) linear_simt_kernel<T, T, true><<<grid, 256, 0, st>>>((const T*)x, (const T*)w, (const T*)w2, (T*)y, resid, M, N, K, ldy);
-    else linear_simt_kernel<T, T, false><<<grid, 256, 0, st>>>((const T*)x, (const T*)w, nullptr, (T*)y, resid, M, N, K, ldy);
+    if (w2) AKVS_CUDA(launch_pdl(linear_simt_kernel<T, T, true>, grid, dim3(256), 0, st, (const T*)x, (const T*)w, (const T*)w2, (T*)y, resid, M, N, K, ldy));
+    else AKVS_CUDA(launch_pdl(linear_simt_kernel<T, T, false>, grid, dim3(256), 0, st, (const T*)x, (const T*)w, (const T*)nullptr, (T*)y, resid, M, N, K, ldy));
     AKVS_LAUNCHED();
     return AKVS_OK;
   });
@@ -90,6 +92,8 @@ attention_simt_kernel(const T* __restrict__ q, const T* __restrict__ k, const T*
                       const int32_t* __restrict__ k_lo, const int32_t* __restrict__ k_hi,
                       const int32_t* __restrict__ k_lo2, const int32_t* __restrict__ k_hi2, int R, int n_q, int n_kv) {
   extern __shared__ float smem[];
+  pdl_trigger();
+  pdl_wait();
   float* qs = smem;                               // [SA_ROWS][HD]
   float* ks = qs + SA_ROWS * HD;                  // [SA_KEYS][HD + 1]
   float* vs = ks + SA_KEYS * (HD + 1);            // [SA_KEYS][HD]
@@ -192,8 +196,8 @@ static int32_t launch_attention_simt_t(const void* q, const void* k, const void*
                                        int n_kv, cudaStream_t st) {
   const size_t smem = sizeof(float) * (SA_ROWS * HD + SA_KEYS * (HD + 1) + SA_KEYS * HD + SA_ROWS * SA_KEYS);
   const dim3 grid(akvs_cdiv(R, SA_ROWS), n_q);
-  attention_simt_kernel<T, HD><<<grid, 128, smem, st>>>((const T*)q, (const T*)k, (const T*)v, (T*)out, k_lo, k_hi, k_lo2,
-                                                       k_hi2, R, n_q, n_kv);
+  AKVS_CUDA(launch_pdl(attention_simt_kernel<T, HD>, grid, dim3(128), smem, st, (const T*)q, (const T*)k, (const T*)v, (T*)out,
+                       k_lo, k_hi, k_lo2, k_hi2, R, n_q, n_kv));
   AKVS_LAUNCHED();
   return AKVS_OK;
 }
