@@ -245,10 +245,13 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
     const int r_local = m / p.g, head = m - r_local * p.g;
     const int r = r0 + r_local;
     const bool valid = r_local < p.BR && r < p.R;
-    const int hi1 = valid ? p.k_hi[r] : -1;
-    const int lo1 = valid && p.k_lo[r] <= hi1 ? p.k_lo[r] : 0x40000000;   // nothing visible: no key reaches lo
-    const int hi2 = valid && p.k_lo2 ? p.k_hi2[r] : -1;
-    const int lo2 = valid && p.k_lo2 && p.k_lo2[r] <= hi2 ? p.k_lo2[r] : 0x40000000;
+    // Rows of the M tile that belong to no query row (g does not divide 128, or the last row
+    // block is short) have Q = 0 and are never written: they take every key as visible, so that
+    // their warp does not run the masking pass on every tile for their sake.
+    const int hi1 = valid ? p.k_hi[r] : 0x3fffffff;
+    const int lo1 = !valid ? -0x40000000 : (p.k_lo[r] <= hi1 ? p.k_lo[r] : 0x40000000);   // nothing visible: no key reaches lo
+    const int hi2 = !valid ? 0x3fffffff : (p.k_lo2 ? p.k_hi2[r] : -1);
+    const int lo2 = !valid ? -0x40000000 : (p.k_lo2 && p.k_lo2[r] <= hi2 ? p.k_lo2[r] : 0x40000000);
     // key visible  <=>  lo <= key <= hi  <=>  (unsigned)(key - lo) <= hi - lo: one compare and a
     // select per element (a per-element && / || compiles to divergent branches, measured 2x slower)
     const unsigned span1 = hi1 >= lo1 ? (unsigned)(hi1 - lo1) : 0u;
