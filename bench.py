@@ -276,8 +276,11 @@ def main():
     g_ms = sum(r[0] for r in gemm)
     g_fl = sum(r[1] for r in gemm)
     by_epi = {}
+    by_shape = {}
     for ms_, fl, sub in gemm:
         a = by_epi.setdefault(sub & 255, [0.0, 0.0, 0])
+        a[0] += ms_; a[1] += fl; a[2] += 1
+        a = by_shape.setdefault((sub & 255, round(fl / 1e9, 1)), [0.0, 0.0, 0])
         a[0] += ms_; a[1] += fl; a[2] += 1
     # attention flops of one step from the recomputed rows: 4 * dq * sum_r (keys visible to r);
     # the dense first layer sees every row, the selective layers the probe and query rows
@@ -303,7 +306,11 @@ def main():
                 "share_of_step": g_ms / (ms_step_prof * args.steps), "instrumented_ms_per_step": ms_step_prof,
                 "by_epilogue": {{0: "qkv_store", 1: "residual", 2: "swiglu"}.get(k, str(k)):
                                 {"tflops": v[1] / (v[0] * 1e-3) / 1e12, "ms_per_step": v[0] / args.steps,
-                                 "launches": v[2]} for k, v in sorted(by_epi.items())}}
+                                 "launches": v[2]} for k, v in sorted(by_epi.items())},
+                # one entry per distinct launch shape: epilogue kind, GFLOP per launch, us per launch, TFLOP/s
+                "by_shape": [{"epilogue": {0: "qkv_store", 1: "residual", 2: "swiglu"}.get(k[0], str(k[0])),
+                              "gflop": k[1], "us": 1e3 * v[0] / v[2], "tflops": v[1] / (v[0] * 1e-3) / 1e12,
+                              "launches": v[2]} for k, v in sorted(by_shape.items())]}
 
     # the same build's full recompute, for context (not the metric)
     def full():
