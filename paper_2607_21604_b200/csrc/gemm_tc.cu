@@ -234,9 +234,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 float* o = reinterpret_cast<float*>(p.seg_out[seg]) + (size_t)row * ldc + col;
 #pragma unroll
                 for (int v = 0; v < 8; ++v) {
-                  float4 t = *reinterpret_cast<float4*>(o + v * 4);
-                  t.x += a[v * 4]; t.y += a[v * 4 + 1]; t.z += a[v * 4 + 2]; t.w += a[v * 4 + 3];
-                  *reinterpret_cast<float4*>(o + v * 4) = t;
+                  // h += acc as a reduction at the L2: one add per element as before (every element
+                  // belongs to exactly one tile), but nothing comes back to the SM, so the epilogue
+                  // does not sit through a load round trip per chunk
+                  asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(o + v * 4), "f"(a[v * 4]),
+                               "f"(a[v * 4 + 1]), "f"(a[v * 4 + 2]), "f"(a[v * 4 + 3]) : "memory");
                 }
               } else {
                 T* o = reinterpret_cast<T*>(p.seg_out[seg]) + (size_t)row * ldc + col;
