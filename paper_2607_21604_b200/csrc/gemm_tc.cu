@@ -86,28 +86,55 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   __syncthreads();
   tc::fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
-  pdl_wait();                       // everything above touched only this CTA's own state
+  // Everything above touched only this CTA's own state.  From here on each role waits for the
+  // kernels before this one (pdl_wait) right before its first access to memory they may have
+  // written: the producer only before its first ACTIVATION tile - the weights are nobody's
+  // output, so their first stages are already in flight while the predecessor drains.
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
       tc::prefetch_tmap(&tmA);
       tc::prefetch_tmap(&tmB0);
-      int s = 0;
-      uint32_t ph = 0;
-      bool ok = true;
-      for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
-        const int tn = tile / p.tiles_m, tm = tile % p.tiles_m;
-        int seg0, row0, seg1, row1;
+      auto b_tiles = [&](int tile, const CUtensorMap*& m0, const CUtensorMap*& m1, int& row0, int& row1) {
+        const int tn = tile / p.tiles_m;
+        int seg0, seg1;
         if (EPI == EPI_SWIGLU) {
           seg0 = 0; seg1 = 1; row0 = row1 = tn * BNH;
         } else {
           locate(p, 2 * tn, seg0, row0);
           locate(p, 2 * tn + 1, seg1, row1);
         }
-        const CUtensorMap* m0 = seg0 == 0 ? &tmB0 : (seg0 == 1 ? &tmB1 : &tmB2);
-        const CUtensorMap* m1 = seg1 == 0 ? &tmB0 : (seg1 == 1 ? &tmB1 : &tmB2);
-        for (int kb = 0; kb < KB; ++kb) {
+        m0 = seg0 == 0 ? &tmB0 : (seg0 == 1 ? &tmB1 : &tmB2);
+        m1 = seg1 == 0 ? &tmB0 : (seg1 == 1 ? &tmB1 : &tmB2);
+      };
+      // weight tiles of the first stages (every stage is free at the start: no wait), then the
+      // dependency on the earlier kernels, then the activation tiles of the same stages
+      const int pre = blockIdx.x < n_tiles ? (KB < STAGES ? KB : STAGES) : 0;
+      if (pre > 0) {
+        const CUtensorMap *m0, *m1;
+        int row0, row1;
+        b_tiles(blockIdx.x, m0, m1, row0, row1);
+        for (int kb = 0; kb < pre; ++kb) {
+          uint8_t* st = smem + kb * STAGE_BYTES;
+          tc::mbar_expect_tx(&full[kb], STAGE_BYTES);
+          tc::tma_load_2d(st + A_BYTES, m0, kb * BK, row0, &full[kb]);
+          tc::tma_load_2d(st + A_BYTES + BH_BYTES, m1, kb * BK, row1, &full[kb]);
+        }
+      }
+      pdl_wait();
+      for (int kb = 0; kb < pre; ++kb)
+        tc::tma_load_2d(smem + kb * STAGE_BYTES, &tmA, kb * BK, (blockIdx.x % p.tiles_m) * BM, &full[kb]);
+      int s = pre % STAGES;
+      uint32_t ph = pre == STAGES ? 1u : 0u;
+      int kb_start = pre;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+        const int tm = tile % p.tiles_m;
+        const CUtensorMap *m0, *m1;
+        int row0, row1;
+        b_tiles(tile, m0, m1, row0, row1);
+        for (int kb = kb_start; kb < KB; ++kb) {
           if (!tc::mbar_wait(&empty[s], ph ^ 1, abort_flag)) { ok = false; break; }
           uint8_t* st = smem + s * STAGE_BYTES;
           tc::mbar_expect_tx(&full[s], STAGE_BYTES);
@@ -116,6 +143,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           tc::tma_load_2d(st + A_BYTES + BH_BYTES, m1, kb * BK, row1, &full[s]);
           if (++s == STAGES) { s = 0; ph ^= 1; }
         }
+        kb_start = 0;
       }
       if (!ok) { *abort_flag = 1; set_status(p.status, AKVS_ERR_TIMEOUT); }
     }
@@ -153,6 +181,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   } else {
     // ------------------------------------------------------------------ epilogue
     const int quad = warp & 3;                 // tensor-memory lane quadrant of this warp
+    pdl_wait();                                // outputs, residual and positions are other kernels' memory
     bool ok = true;
     int it = 0;
     for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++it) {
