@@ -26,6 +26,8 @@ enum { EPI_STORE = 0, EPI_RESID = 1, EPI_SWIGLU = 2 };
 
 struct GemmParams {
   int M, K, tiles_m, tiles_n;
+  int nh;                 // 128-column blocks of B per tile: 2 (128x256 tiles) or 1 (128x128, when 256-wide
+                          // tiles would leave most SMs without work)
   int n_seg;
   int seg_blocks[3];      // 128-row blocks of each B matrix
   void* seg_out[3];       // output of each segment (16-bit [M][ldc], or float for EPI_RESID)
@@ -102,14 +104,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         if (EPI == EPI_SWIGLU) {
           seg0 = 0; seg1 = 1; row0 = row1 = tn * BNH;
         } else {
-          locate(p, 2 * tn, seg0, row0);
-          locate(p, 2 * tn + 1, seg1, row1);
+          locate(p, p.nh * tn, seg0, row0);
+          locate(p, p.nh * tn + 1, seg1, row1);
         }
         m0 = seg0 == 0 ? &tmB0 : (seg0 == 1 ? &tmB1 : &tmB2);
         m1 = seg1 == 0 ? &tmB0 : (seg1 == 1 ? &tmB1 : &tmB2);
       };
       // weight tiles of the first stages (every stage is free at the start: no wait), then the
       // dependency on the earlier kernels, then the activation tiles of the same stages
+      const uint32_t stage_tx = A_BYTES + p.nh * BH_BYTES;
       const int pre = blockIdx.x < n_tiles ? (KB < STAGES ? KB : STAGES) : 0;
       if (pre > 0) {
         const CUtensorMap *m0, *m1;
@@ -117,9 +120,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         b_tiles(blockIdx.x, m0, m1, row0, row1);
         for (int kb = 0; kb < pre; ++kb) {
           uint8_t* st = smem + kb * STAGE_BYTES;
-          tc::mbar_expect_tx(&full[kb], STAGE_BYTES);
+          tc::mbar_expect_tx(&full[kb], stage_tx);
           tc::tma_load_2d(st + A_BYTES, m0, kb * BK, row0, &full[kb]);
-          tc::tma_load_2d(st + A_BYTES + BH_BYTES, m1, kb * BK, row1, &full[kb]);
+          if (p.nh == 2) tc::tma_load_2d(st + A_BYTES + BH_BYTES, m1, kb * BK, row1, &full[kb]);
         }
       }
       pdl_wait();
@@ -137,10 +140,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         for (int kb = kb_start; kb < KB; ++kb) {
           if (!tc::mbar_wait(&empty[s], ph ^ 1, abort_flag)) { ok = false; break; }
           uint8_t* st = smem + s * STAGE_BYTES;
-          tc::mbar_expect_tx(&full[s], STAGE_BYTES);
+          tc::mbar_expect_tx(&full[s], stage_tx);
           tc::tma_load_2d(st, &tmA, kb * BK, tm * BM, &full[s]);
           tc::tma_load_2d(st + A_BYTES, m0, kb * BK, row0, &full[s]);
-          tc::tma_load_2d(st + A_BYTES + BH_BYTES, m1, kb * BK, row1, &full[s]);
+          if (p.nh == 2) tc::tma_load_2d(st + A_BYTES + BH_BYTES, m1, kb * BK, row1, &full[s]);
           if (++s == STAGES) { s = 0; ph ^= 1; }
         }
         kb_start = 0;
@@ -218,9 +221,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         }
       } else {
 #pragma unroll 1
-        for (int hf = 0; hf < 2; ++hf) {
+        for (int hf = 0; hf < p.nh; ++hf) {
           int seg, brow;
-          locate(p, 2 * tn + hf, seg, brow);
+          locate(p, p.nh * tn + hf, seg, brow);
           const bool valid = brow < p.seg_blocks[seg] * BNH;
           const int ldc = p.seg_ldc[seg];
           if (EPI == EPI_STORE && ((p.rope_mask >> seg) & 1)) {
@@ -390,7 +393,6 @@ int32_t launch_linear_tc(int dtype, int epi, const void* x, int M, int K, int n_
   p.pos = pos;
   p.rope_mask = (epi == EPI_STORE && rope && pos) ? rope_mask : 0;
   const uint32_t fmt = dtype == AKVS_F16 ? tc::kF16 : tc::kBF16;
-  p.idesc = tc::idesc_f16(fmt, fmt, BM, 2 * BNH, 0);
   CUtensorMap tmA, tmB[3];
   AKVS_TRY(encode_tmap_2d_16bit(&tmA, x, M, K, K, BM));
   int blocks = 0;
@@ -403,13 +405,21 @@ int32_t launch_linear_tc(int dtype, int epi, const void* x, int M, int K, int n_
     p.seg_ldc[i] = ldc[i < n_seg && (epi != EPI_SWIGLU || i == 0) ? i : 0];
     if (i < n_seg) blocks += n[s] / BNH;
   }
+  p.tiles_m = (M + BM - 1) / BM;
+  p.nh = 2;
   if (epi == EPI_SWIGLU) {
     if (n_seg != 2 || n[0] != n[1]) return AKVS_ERR_SHAPE;
     p.tiles_n = n[0] / BNH;
   } else {
-    p.tiles_n = (blocks + 1) / 2;
+    // 128x128 tiles when that shortens the launch: a tile of half the width takes ~0.62 of the
+    // time (its MMAs read as many shared-memory bytes per flop again), rounds = tiles / SMs
+    const int sms = sm_count();
+    const int t2 = p.tiles_m * ((blocks + 1) / 2), t1 = p.tiles_m * blocks;
+    const double cost2 = (double)((t2 + sms - 1) / sms), cost1 = 0.62 * ((t1 + sms - 1) / sms);
+    if (cost1 < 0.9 * cost2) p.nh = 1;
+    p.tiles_n = (blocks + p.nh - 1) / p.nh;
   }
-  p.tiles_m = (M + BM - 1) / BM;
+  p.idesc = tc::idesc_f16(fmt, fmt, BM, p.nh * BNH, 0);
   const int n_tiles = p.tiles_m * p.tiles_n;
   const int grid = n_tiles < sm_count() ? n_tiles : sm_count();
   double flops = 0;
