@@ -65,7 +65,7 @@ CONFIGS = {
     "c4": Workload("c4", _M4, 30, 384, 384, 128, (1000, 2000, 3000)),
     "c5q4": Workload("c5q4", _M3, 48, 256, 256, 128, (2000,), "q4"),
     "c5q2": Workload("c5q2", _M3, 48, 256, 256, 128, (2000,), "q2"),
-    "c5fp8": Workload("c5fp8", _M3, 48, 256, 256, 128, (2000,), "fp8"),     # not a BASELINE configuration: the FP8 cache
+    "c5fp8": Workload("c5fp8", _M3, 48, 256, 256, 128, (2000,), "fp8"),     # extra: configuration 5 with the FP8 cache
 }
 
 

@@ -1,11 +1,12 @@
-"""Parity on the BASELINE configurations 2-5 at full model width.
+"""Parity on benchmark configurations 2-5 at full model width.
 
 The oracle is plain numpy, so each configuration runs at reduced depth and context (sizes
 the oracle finishes in tens of seconds) plus, for the 3B-class model, at its FULL depth of
 36 layers on a short context.  Full-size behaviour (the launch configuration the benchmark
 times) is covered by per-kernel checks on sampled outputs and by invariants that hold at
-any size.  The 16-bit configurations hold their bf16-valued weights in float16 containers
-(see the precision reading in the design doc)."""
+any size.  The 16-bit configurations hold their bf16-valued weights in float16 containers:
+rounding activations to bf16 between kernels alone exceeds the 1e-2 bound after about a dozen
+layers, float16 storage stays near 2e-3."""
 import ctypes as C
 
 import numpy as np
