@@ -129,6 +129,19 @@ def test_batch_f16_tensor_core_paths(check_layer):
     _run(case, [[0, 1, 2, 3, 4], [3, 1], [4, 0, 2], [2]], [2, 1, 3, 1], 2500, check_layer)
 
 
+@pytest.mark.parametrize("kv_format", [4, 8])
+def test_batch_quantised_caches(kv_format):
+    """Batched requests over a 4-bit group-quantised and an FP8 cache (dequantisation fused into
+    the scores / offsets / correction reads of every request)."""
+    case = Case(small16("f16"), std_scale=4.0, kv_format=kv_format)
+    _run(case, [[4, 3, 2, 1, 0], [0, 2], [1, 4, 3]], [1, 2, 1], 2500, 2)
+
+
+def test_batch_bf16_storage():
+    case = Case(small16("bf16"), std_scale=1.0)
+    _run(case, [[0, 1, 2], [4, 3]], [1, 1], 2500, 2)
+
+
 def test_batch_request_without_context():
     """A request with no units (query only) inside a batch: its rows see only its own query."""
     case = Case(small16("f16"), std_scale=4.0)
