@@ -371,43 +371,68 @@ offsets_kernel(KvLayer kv, ReqMaps maps, const int32_t* __restrict__ probe_off, 
   const void* cbase = is_v ? kv.v : kv.k;
   const void* cmeta = is_v ? kv.v_meta : kv.k_meta;
 
-  for (int e = lane; e < half; e += 32) { part[wid * hd + e] = 0.f; part[wid * hd + half + e] = 0.f; }
-  for (int i = wid; i < b; i += OFF_WARPS) {
-    const int j = S[i];
-    const int row = maps.row_of_pos[j];
-    const int64_t src = maps.tok_src[j];
-    if (row < 0) continue;                         // inconsistent caller-supplied sets: skip
-    const T* fp = fresh + ((size_t)row * n_kv + h) * hd;
-    for (int e = lane; e < half; e += 32) {
-      float lo, hi;
-      if constexpr (FMT == AKVS_KV_NATIVE) {
-        const TW* cp = reinterpret_cast<const TW*>(cbase) + ((size_t)src * n_kv + h) * hd;
-        lo = to_f(cp[e]);
-        hi = to_f(cp[half + e]);
-      } else if constexpr (FMT == AKVS_KV_FP8) {
-        const uint8_t* cp = reinterpret_cast<const uint8_t*>(cbase) + ((size_t)src * n_kv + h) * hd;
-        const __half_raw ra = __nv_cvt_fp8_to_halfraw(cp[e], __NV_E4M3), rb = __nv_cvt_fp8_to_halfraw(cp[half + e], __NV_E4M3);
-        lo = __half2float(*reinterpret_cast<const __half*>(&ra));
-        hi = __half2float(*reinterpret_cast<const __half*>(&rb));
-      } else {
-        const uint8_t* cp = reinterpret_cast<const uint8_t*>(cbase) + ((size_t)src * n_kv + h) * hd * FMT / 8;
-        const __half2* mp = reinterpret_cast<const __half2*>(cmeta) + ((size_t)src * n_kv + h) * (hd / 64);
-        const int e2 = half + e;
-        const uint32_t qa = (cp[e * FMT / 8] >> ((e * FMT) & 7)) & ((1u << FMT) - 1u);
-        const uint32_t qb = (cp[e2 * FMT / 8] >> ((e2 * FMT) & 7)) & ((1u << FMT) - 1u);
-        const __half2 ma = mp[e / 64], mb = mp[e2 / 64];
-        lo = __fmaf_rn((float)qa, __low2float(ma), __high2float(ma));
-        hi = __fmaf_rn((float)qb, __low2float(mb), __high2float(mb));
-      }
-      if (!is_v) {
-        const float2 t = rot[e];
-        const float rlo = lo * t.x - hi * t.y, rhi = hi * t.x + lo * t.y;
-        lo = rlo;
-        hi = rhi;
-      }
-      part[wid * hd + e] += to_f(fp[e]) - lo;
-      part[wid * hd + half + e] += to_f(fp[half + e]) - hi;
+  // A lane owns the rotation pairs e = lane, lane + 32, ... and keeps their sums in registers.
+  // The warp's probes (every 8th of the unit) are taken 32 at a time: each lane first fetches
+  // the row and store indices of one probe, so that the dependent index loads are paid once per
+  // batch and not once per probe; the probes are then walked in their original order.
+  constexpr int OFF_Q = 4;                        // pairs per lane: head_dim <= 256
+  float acc_lo[OFF_Q], acc_hi[OFF_Q];
+#pragma unroll
+  for (int q = 0; q < OFF_Q; ++q) acc_lo[q] = acc_hi[q] = 0.f;
+  for (int base = wid; base < b; base += OFF_WARPS * 32) {
+    const int i = base + lane * OFF_WARPS;
+    int row_l = -1, src_l = 0;
+    if (i < b) {
+      const int j = S[i];
+      row_l = maps.row_of_pos[j];
+      src_l = maps.tok_src[j];
     }
+    const int left = (b - base + OFF_WARPS - 1) / OFF_WARPS;
+    const int cnt = left < 32 ? left : 32;
+    for (int k = 0; k < cnt; ++k) {
+      const int row = __shfl_sync(0xFFFFFFFFu, row_l, k);
+      const int64_t src = __shfl_sync(0xFFFFFFFFu, src_l, k);
+      if (row < 0) continue;                       // inconsistent caller-supplied sets: skip
+      const T* fp = fresh + ((size_t)row * n_kv + h) * hd;
+#pragma unroll
+      for (int q = 0; q < OFF_Q; ++q) {
+        const int e = lane + 32 * q;
+        if (e >= half) break;
+        float lo, hi;
+        if constexpr (FMT == AKVS_KV_NATIVE) {
+          const TW* cp = reinterpret_cast<const TW*>(cbase) + ((size_t)src * n_kv + h) * hd;
+          lo = to_f(cp[e]);
+          hi = to_f(cp[half + e]);
+        } else if constexpr (FMT == AKVS_KV_FP8) {
+          const uint8_t* cp = reinterpret_cast<const uint8_t*>(cbase) + ((size_t)src * n_kv + h) * hd;
+          const __half_raw ra = __nv_cvt_fp8_to_halfraw(cp[e], __NV_E4M3), rb = __nv_cvt_fp8_to_halfraw(cp[half + e], __NV_E4M3);
+          lo = __half2float(*reinterpret_cast<const __half*>(&ra));
+          hi = __half2float(*reinterpret_cast<const __half*>(&rb));
+        } else {
+          const uint8_t* cp = reinterpret_cast<const uint8_t*>(cbase) + ((size_t)src * n_kv + h) * hd * FMT / 8;
+          const __half2* mp = reinterpret_cast<const __half2*>(cmeta) + ((size_t)src * n_kv + h) * (hd / 64);
+          const int e2 = half + e;
+          const uint32_t qa = (cp[e * FMT / 8] >> ((e * FMT) & 7)) & ((1u << FMT) - 1u);
+          const uint32_t qb = (cp[e2 * FMT / 8] >> ((e2 * FMT) & 7)) & ((1u << FMT) - 1u);
+          const __half2 ma = mp[e / 64], mb = mp[e2 / 64];
+          lo = __fmaf_rn((float)qa, __low2float(ma), __high2float(ma));
+          hi = __fmaf_rn((float)qb, __low2float(mb), __high2float(mb));
+        }
+        if (!is_v) {
+          const float2 t = rot[e];
+          const float rlo = lo * t.x - hi * t.y, rhi = hi * t.x + lo * t.y;
+          lo = rlo;
+          hi = rhi;
+        }
+        acc_lo[q] += to_f(fp[e]) - lo;
+        acc_hi[q] += to_f(fp[half + e]) - hi;
+      }
+    }
+  }
+#pragma unroll
+  for (int q = 0; q < OFF_Q; ++q) {
+    const int e = lane + 32 * q;
+    if (e < half) { part[wid * hd + e] = acc_lo[q]; part[wid * hd + half + e] = acc_hi[q]; }
   }
   __syncthreads();
   float* mu = (is_v ? mu_v : mu_k) + ((size_t)u * n_kv + h) * hd;
@@ -424,6 +449,7 @@ int32_t launch_offsets(int dtype, const KvLayer& kv, const ReqMaps& maps, const 
                        int n_kv, int hd, const float2* table, float* mu_k, float* mu_v, cudaStream_t st) {
   if (M == 0) return AKVS_OK;
   AKVS_TRY(check_kv_shape(dtype, kv, hd));
+  if (hd > 256) return AKVS_ERR_UNSUPPORTED;      // a lane keeps at most 4 rotation pairs
   const dim3 grid(M, n_kv, 2);
   const size_t smem = (size_t)OFF_WARPS * hd * sizeof(float);
   return dispatch_dtype(dtype, [&](auto tag) -> int32_t {
