@@ -143,7 +143,7 @@ def reference_arm(args, w):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours")
     ap.add_argument("--workload", default="c3")
@@ -232,17 +232,22 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
+    step_times = []
+
     def timed(fn, steps, warmup):
+        """Mean time per step over `steps` steps (max over ranks).  An event after every step also
+        gives the single-step times of the last call (rank-local), for the median and the best."""
         for _ in range(warmup):
             fn()
         barrier()
-        a, b = ev(), ev()
-        a.record()
-        for _ in range(steps):
+        marks = [ev() for _ in range(steps + 1)]
+        marks[0].record()
+        for i in range(steps):
             fn()
-        b.record()
+            marks[i + 1].record()
         barrier()
-        return max_over_ranks(a.elapsed_time(b), world) / steps
+        step_times[:] = [marks[i].elapsed_time(marks[i + 1]) for i in range(steps)]
+        return max_over_ranks(marks[0].elapsed_time(marks[-1]), world) / steps
 
     # ---------------------------------------------------------------- device-resident timing
     # The headline time comes from K plain steps.  The per-kernel figures of the roofline object come
@@ -257,6 +262,7 @@ def main():
     launches0 = akvs.launch_count()
     sampler.mark()
     ms_step = timed(step, args.steps, 0)
+    ms_median, ms_best = float(np.median(step_times)), float(min(step_times))
     launches = akvs.launch_count() - launches0
     akvs.prof_enable((1 << 1) | (1 << 2) | (1 << 3), 8192)
     step()
@@ -363,7 +369,8 @@ def main():
         cpu = {"value": val, "unit": UNIT, "cores": ccores, "kind": "oracle", "sample": sample}
     out = {
         "metric": metric, "value": whole_job_rate(T, world, ms_step), "unit": UNIT, "n_gpus": world,
-        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "ms_per_step_median": ms_median,
+        "ms_per_step_best": ms_best, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None,
         "dtype": {"f16": "f16 storage (bf16-valued random-init weights), f32 accumulate",
                   "bf16": "bf16 storage, f32 accumulate", "f32": "f32"}[m.dtype],
