@@ -148,6 +148,35 @@ def test_attention_tensor_core_many_tiles(akvs, dtype, nq, nkv):
     assert orc.rel_l2(n64(out), n64(out1)) < 4 * EPS[dtype]
 
 
+@pytest.mark.parametrize("dtype", H16)
+@pytest.mark.parametrize("shape", ["rising", "falling", "spiky"])
+def test_attention_tensor_core_moving_maximum(akvs, dtype, shape):
+    """Scores whose maximum moves by far more than 2^8 between key tiles: the shared reference
+    maximum is raised again and again (the output accumulator is rescaled in tensor memory), stays
+    put while later tiles fall far below it, or jumps on single keys."""
+    g = np.random.default_rng(17)
+    T, hd, nq, nkv = 1500, 128, 8, 2
+    kk = g.standard_normal((T, nkv, hd)).astype(np.float32)
+    ramp = np.linspace(0.05, 6.0, T, dtype=np.float32)
+    if shape == "rising":
+        kk *= ramp[:, None, None]
+    elif shape == "falling":
+        kk *= ramp[::-1, None, None]
+    else:
+        kk *= 0.2
+        kk[g.choice(T, 25, replace=False)] *= 40.0
+    k, v = dev(kk, dtype), dev(g.standard_normal((T, nkv, hd)).astype(np.float32), dtype)
+    rows = np.sort(g.choice(T, 150, replace=False)).astype(np.int32)
+    rows[-1] = T - 1
+    q = dev((g.standard_normal((len(rows), nq, hd)) * 2.0).astype(np.float32), dtype)
+    out = akvs.op_attention(q, k, v, dev(np.zeros_like(rows)), dev(rows), 0)
+    torch.cuda.synchronize()
+    ref = orc.attention(n64(q), n64(k), n64(v), rows, np.arange(T))
+    per_row = np.linalg.norm((n64(out) - ref).reshape(len(rows), -1), axis=1) / np.linalg.norm(ref.reshape(len(rows), -1), axis=1)
+    assert per_row.max() < 8 * EPS[dtype], (per_row.argmax(), per_row.max())
+    assert torch.isfinite(out.float()).all()
+
+
 # ----------------------------------------------------------------------------- selection (bit-exact)
 
 def _check_select(akvs, dk, dv, off, nq, bp):
