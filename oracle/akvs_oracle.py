@@ -26,14 +26,20 @@ heads; `check_layer` is 1-based and layers before it are computed densely for ev
 ties in the top-b are broken towards the smaller token index; b is computed from the
 ratio in integer basis points.
 
+* Section 4.5 (quantised caches): 2/4-bit asymmetric groups of 64 and the FP8 (E4M3) cast,
+  the paper naming only the formats.
+* Section 3.4 and the appendix on mean-explained residual energy: `residual_stats`.
+
 Arithmetic: float64 by default (`dtype=np.float32` gives the single-precision variant).
-The group quantiser is the exception: its decisions are taken in float32 with float16
-scale and minimum, because those decide integer codes.
+The quantisers are the exception: their decisions are taken on float32 values (float16
+scale and minimum for the groups), because those decide integer codes.
 
 Pins (tests/test_oracle_*.py): closed forms for the mean and the correction, brute-force
 top-b, brute-force attention, an independent composition of stock library ops for the
 transformer, Lemma 1's inequality, the Proposition 2 residual identity, quantiser error
-bounds, and the invariants 100 % refresh == full recompute, first unit has zero
+bounds, the E4M3 cast by brute force over every code, hand-computed ties and an independent
+library cast, the residual statistics by the variance identity and hand-computed weighted
+means, and the invariants 100 % refresh == full recompute, first unit has zero
 residual, 0 % refresh == naive reuse, exact constant-offset caches are recovered exactly.
 No function here is "parity unpinned".
 """
