@@ -12,6 +12,11 @@
 // The 256 accumulator columns are two 128-row blocks of B that may come from different
 // weight matrices: (Wq | Wk | Wv) share one launch, and (W_gate, W_up) land side by side
 // so that silu(gate) * up is formed in registers and only the activation is written.
+// Epilogues: store (16-bit; a 128-column block that is one attention head gets its RoPE rotation
+// in registers), residual (h += acc as a vector reduction at the L2, nothing is read back),
+// SwiGLU.  A launch whose 128x256 tiles would occupy well under all SMs runs 128x128 tiles
+// (one B block per tile, `nh` = 1).  The kernel is launched as a programmatic dependent: its
+// set-up and the first weight tiles overlap the tail of the kernel before it.
 #include "tc_common.cuh"
 
 namespace {
