@@ -34,6 +34,30 @@ def test_config_width_reduced_depth(name, n_layers, n_units):
     _run_all_modes(case, w.refresh_bp[0], 2, units)
 
 
+def _run_corrected_only(case, bp, check_layer, units):
+    ref = orc.corrected_reuse(case.omodel, units, list(case.order), case.ctx, case.qry, bp, check_layer)
+    probes, ctx, ws = case.gpu_select(bp, check_layer)
+    assert np.array_equal(probes.probe_off.cpu().numpy()[:case.M + 1], ref["probes"]["probe_off"])
+    case.set_probes(probes, ref["probes"])
+    hid, k, v = case.gpu_prefill(case.akvs.MODE_CORRECTED, ws, probes, ctx, check_layer)
+    case.akvs.free(ctx)
+    assert orc.rel_l2(hid, ref["hidden"]) < case.tol
+    assert max_layer_err(k, ref["K"]) < case.tol and max_layer_err(v, ref["V"]) < case.tol
+
+
+@pytest.mark.parametrize("name,n_layers,n_units,ratios", [("c2", 3, 4, (2000, 3000)), ("c4", 2, 2, (3000,))])
+def test_config_other_refresh_ratios(name, n_layers, n_units, ratios):
+    """Configurations 2 and 4 are specified at 10, 20 and 30 % refresh: the higher ratios on the
+    corrected path (the first ratio runs in test_config_width_reduced_depth)."""
+    w = _reduced(name, n_layers, n_units)
+    case = Case(w)
+    case.encode()
+    units = case.oracle_units()
+    case.load_oracle_cache(units)
+    for bp in ratios:
+        _run_corrected_only(case, bp, 2, units)
+
+
 @pytest.mark.parametrize("name", ["c5q4", "c5q2", "c5fp8"])
 def test_config5_quantised_cache(name):
     w = _reduced(name, 3, 4)
