@@ -174,7 +174,13 @@ int32_t akvs_select_probes(const akvs_model_desc* model, const akvs_cache* cache
  *  AKVS_MODE_FULL:  probes/ctx may be NULL; everything recomputed (cache K/V unused).
  * Outputs: out_hidden float [n_query][d_model] (after the final RMSNorm);
  *          out_k, out_v [L][n_ctx+n_query][n_kv][head_dim] in the model dtype, K after
- *          RoPE at global positions.  Asynchronous. */
+ *          RoPE at global positions.  Asynchronous.
+ * In AKVS_MODE_CORRECTED the call only enqueues work on `stream` (kernels and device-to-device
+ * copies; no host reads, no host buffers of its own), so after one eager call with the same
+ * model (which sets the kernels' function attributes) it may be recorded into a CUDA graph by
+ * stream capture and replayed, as long as every pointer argument, the probe counts and the
+ * cache's layer_ready events stay what they were at capture.  The other two modes upload small
+ * host tables and are not meant for capture. */
 int32_t akvs_prefill_corrected(const akvs_model_desc* model, const akvs_cache* cache,
                                const akvs_request* req, const akvs_probes* probes, int32_t mode,
                                float* out_hidden, void* out_k, void* out_v,

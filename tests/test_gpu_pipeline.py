@@ -245,3 +245,32 @@ def test_cache_streamed_in_behind_layer_events():
     case.store.set_layer_events(None)
     for x, y in zip(got, want):
         assert np.array_equal(x, y)
+
+
+def test_corrected_prefill_replays_from_a_cuda_graph():
+    """The corrected prefill enqueues only stream work: captured once, its replay writes the same
+    bits as the eager call."""
+    case = Case(small16("f16"), std_scale=4.0)
+    a = case.akvs
+    case.encode()
+    probes, ctx, ws = case.gpu_select(2500, 2)
+    hid, k, v = a.alloc_outputs(case.gmodel, case.N, case.nq)
+    run = lambda: a.prefill_corrected(case.gmodel, case.store, case.req, probes, a.MODE_CORRECTED, hid, k, v, ctx, ws)
+    run()                                             # eager: also the warm-up the header asks for
+    torch.cuda.synchronize()
+    want = (hid.clone(), k.clone(), v.clone())
+    for t in (hid, k, v):
+        t.zero_()
+    side = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            run()
+    torch.cuda.synchronize()
+    assert float(hid.abs().max()) == 0.0              # capture records, it does not run
+    for _ in range(2):
+        graph.replay()
+    torch.cuda.synchronize()
+    assert a.check(ws) == 0
+    assert torch.equal(hid, want[0]) and torch.equal(k, want[1]) and torch.equal(v, want[2])
+    a.free(ctx)
