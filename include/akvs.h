@@ -19,6 +19,10 @@
  *    (scratch comes from the caller's workspace);
  *  - all work is enqueued on the caller's stream (a cudaStream_t passed as void*; NULL is
  *    the default stream); only akvs_select_probes and akvs_check synchronise it;
+ *  - a process drives ONE device through this library (one process per GPU): kernel
+ *    attributes are set once per process on the device current at the first call, the
+ *    measurement hooks keep process-wide state, and calls are not re-entrant across host
+ *    threads that share a workspace;
  *  - linear weights are row-major [out_features][in_features] (y = x W^T), no biases;
  *  - model dtype AKVS_F32 / AKVS_BF16 / AKVS_F16: weights, the native unit cache, every
  *    activation tensor and the K/V outputs have that type; accumulation, the residual
