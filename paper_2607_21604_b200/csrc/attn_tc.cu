@@ -101,15 +101,17 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
 }
 
 enum { B_QFULL = 0,     // Q sits in tensor memory (4 warps)
-       B_KFULL = 1, B_KEMPTY = 4, B_VFULL = 7, B_VEMPTY = 11,
-       B_SFULL = 15,    // [2] S of an even / odd tile is complete
-       B_SEMPTY = 17,   // [2] the group has taken S into registers (4 warps)
-       B_PFULL = 19,    // P of the next tile is in tensor memory (4 warps)
-       B_ODONE = 20,    // [4] P V of tile j (slot j mod 4) has completed
-       B_OFINAL = 24,   // the last P V has completed
-       B_DEC = 25,      // [2][4] the warp of this quad has settled the reference maximum of an even / odd tile
-       B_FIN = 33,      // [4] both warps of this quad have published their row sums
-       B_COUNT = 37 };
+       B_KFULL = 1, B_KEMPTY = B_KFULL + K_STAGES, B_VFULL = B_KEMPTY + K_STAGES, B_VEMPTY = B_VFULL + V_STAGES,
+       B_SFULL = B_VEMPTY + V_STAGES,   // [2] S of an even / odd tile is complete
+       B_SEMPTY = B_SFULL + 2,          // [2] the group has taken S into registers (4 warps)
+       B_PFULL = B_SEMPTY + 2,          // P of the next tile is in tensor memory (4 warps)
+       B_ODONE = B_PFULL + 1,           // [4] P V of tile j (slot j mod 4) has completed
+       B_OFINAL = B_ODONE + 4,          // the last P V has completed
+       B_DEC = B_OFINAL + 1,            // [2][4] the warp of this quad has settled the reference maximum of an even / odd tile
+       B_FIN = B_DEC + 8,               // [4] both warps of this quad have published their row sums
+       B_COUNT = B_FIN + 4 };
+static_assert(B_COUNT * 8 + 16 <= 512, "barriers, the tensor-memory slot and the abort flag share 512 bytes");
+static_assert((K_STAGES + V_STAGES) * TILE + 512 + 5 * 128 * 4 <= 232448, "shared memory of one CTA");
 
 template <typename T>
 __global__ void __launch_bounds__(ATT_THREADS, 1)
