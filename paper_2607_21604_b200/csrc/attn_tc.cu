@@ -349,7 +349,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
       if (raise) m_ref[m] = m_new;
       __syncwarp();
       if (lane == 0 && j + 1 < n_tiles) tc::mbar_arrive(&bar[B_DEC + (j & 1) * 4 + quad]);
-      l_mine *= ex2(m_mine - m_new);
+      if (m_mine != m_new) l_mine *= ex2(m_mine - m_new);       // rare: keeps a special-function round trip off the usual path
       m_mine = m_new;
       if (j > 0 && __any_sync(0xffffffffu, raise)) {
         // rows of O accumulated so far move to the new maximum, once P(j-1) V(j-1) has landed
