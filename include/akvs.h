@@ -199,7 +199,9 @@ int32_t akvs_check(void* workspace, void* stream);
 
 /* Cross-check switch for the tests: bit 0 set routes the 16-bit linear layers, bit 1 set the
  * 16-bit attention, to the CUDA-core kernels instead of the tcgen05 ones (default 0: tensor
- * cores for both).  Process-wide; not part of the serving surface. */
+ * cores for both).  Bits 2-3: tiling of the tcgen05 linear layers - 0 picked by shape
+ * (default), 1 single CTAs, 2 CTA pairs wherever M > 128.  Process-wide; not part of the
+ * serving surface. */
 int32_t akvs_debug_set_linear_algo(int32_t algo);
 
 /* Number of kernels this library has launched in this process so far. */
@@ -223,7 +225,9 @@ int32_t akvs_prof_read(int32_t capacity, float* ms, double* work, int32_t* sub, 
  * ------------------------------------------------------------------------------------ */
 
 /* y[M][N] = x[M][K] * w[N][K]^T, float accumulation.  algo 0: the path's default for the
- * dtype (tcgen05 tensor cores for the 16-bit types, CUDA cores for float); algo 1: CUDA cores. */
+ * dtype (tcgen05 tensor cores for the 16-bit types, CUDA cores for float); algo 1: CUDA cores;
+ * algo 2 / 3 (16-bit types): the tensor-core kernel forced onto single CTAs / onto CTA pairs
+ * (pairs need M > 128; otherwise single CTAs run) - the default picks between them by shape. */
 int32_t akvs_op_linear(int32_t dtype, const void* x, const void* w, void* y,
                        int32_t M, int32_t N, int32_t K, int32_t algo, void* stream);
 

@@ -162,6 +162,7 @@ struct Ctx {                   // host object that carries a request from select
 
 // ----------------------------------------------------------------------------- linear layers
 int g_bf16_linear_algo = 0;    // 16-bit models: 0 = tcgen05; 1 = CUDA cores (kept for cross-checking)
+int g_linear_tiling = 0;       // tcgen05 linear layers: 0 = by shape; 1 = single CTAs; 2 = CTA pairs (cross-checking)
 
 // Projections that share the input x.  Segments whose bit is set in rope_mask are [M][heads][hd]
 // tensors that get RoPE at pos[row]: fused into the tensor-core epilogue when hd == 128,
@@ -175,7 +176,7 @@ int32_t linear_multi(const Dims& D, const void* x, int M, int K, int n_seg, cons
   const bool fuse = tc_ok && D.hd == 128;
   if (tc_ok) {
     AKVS_TRY(launch_linear_tc(D.dtype, 0, x, M, K, n_seg, w, n, out, ldc, status, st, fuse ? rope : nullptr, pos,
-                              rope_mask));
+                              rope_mask, g_linear_tiling));
   } else {
     for (int i = 0; i < n_seg; ++i)
       AKVS_TRY(launch_linear_simt(D.dtype, x, w[i], nullptr, out[i], nullptr, M, n[i], K, ldc[i], st));
@@ -190,7 +191,7 @@ int32_t linear_resid(const Dims& D, const void* x, int M, int K, const void* w, 
                      cudaStream_t st) {
   if (D.dtype != AKVS_F32 && g_bf16_linear_algo == 0 && K % 8 == 0 && n % 128 == 0) {
     void* out = h;
-    return launch_linear_tc(D.dtype, 1, x, M, K, 1, &w, &n, &out, &n, status, st);
+    return launch_linear_tc(D.dtype, 1, x, M, K, 1, &w, &n, &out, &n, status, st, nullptr, nullptr, 0, g_linear_tiling);
   }
   return launch_linear_simt(D.dtype, x, w, nullptr, nullptr, h, M, n, K, n, st);
 }
@@ -201,7 +202,7 @@ int32_t linear_swiglu(const Dims& D, const void* x, int M, int K, const void* wg
     const int ns[2] = {n, n};
     void* out[2] = {act, act};
     const int ld[2] = {n, n};
-    return launch_linear_tc(D.dtype, 2, x, M, K, 2, w, ns, out, ld, status, st);
+    return launch_linear_tc(D.dtype, 2, x, M, K, 2, w, ns, out, ld, status, st, nullptr, nullptr, 0, g_linear_tiling);
   }
   return launch_linear_simt(D.dtype, x, wg, wu, act, nullptr, M, n, K, n, st);
 }
@@ -450,6 +451,8 @@ extern "C" {
 int32_t akvs_debug_set_linear_algo(int32_t algo) {
   g_bf16_linear_algo = algo & 1;
   g_attention_algo = (algo >> 1) & 1;
+  g_linear_tiling = (algo >> 2) & 3;
+  if (g_linear_tiling == 3) g_linear_tiling = 0;
   return AKVS_OK;
 }
 
@@ -743,9 +746,11 @@ int32_t akvs_op_linear(int32_t dtype, const void* x, const void* w, void* y, int
   if (!x || !w || !y || M < 0 || N <= 0 || K <= 0) return AKVS_ERR_INVALID_ARG;
   if (dtype != AKVS_F32 && dtype != AKVS_BF16 && dtype != AKVS_F16) return AKVS_ERR_UNSUPPORTED;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
-  if (dtype != AKVS_F32 && algo == 0) {
+  if (algo < 0 || algo > 3) return AKVS_ERR_INVALID_ARG;
+  if (dtype != AKVS_F32 && algo != 1) {
     if (N % 128 != 0 || K % 8 != 0) return AKVS_ERR_SHAPE;
-    return launch_linear_tc(dtype, 0, x, M, K, 1, &w, &N, &y, &N, nullptr, st);
+    return launch_linear_tc(dtype, 0, x, M, K, 1, &w, &N, &y, &N, nullptr, st, nullptr, nullptr, 0,
+                            algo == 0 ? 0 : algo - 1);
   }
   return launch_linear_simt(dtype, x, w, nullptr, y, nullptr, M, N, K, N, st);
 }

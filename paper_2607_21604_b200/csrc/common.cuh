@@ -237,9 +237,10 @@ int32_t launch_linear_simt(int dtype, const void* x, const void* w, const void* 
 // 2: out[0] = silu(x w[0]^T) * (x w[1]^T).
 // With epi 0, segments whose bit is set in rope_mask (heads of 128 columns) are rotated through
 // rope[pos[row]] in the epilogue (rope: [positions][64] (cos, sin); null = no rotation).
+// tiling 0: single CTAs or CTA pairs, whichever the shape favours; 1: single CTAs; 2: pairs (M > 128).
 int32_t launch_linear_tc(int dtype, int epi, const void* x, int M, int K, int n_seg, const void* const* w, const int* n,
                          void* const* out, const int* ldc, int32_t* status, cudaStream_t st,
-                         const float2* rope = nullptr, const int32_t* pos = nullptr, int rope_mask = 0);
+                         const float2* rope = nullptr, const int32_t* pos = nullptr, int rope_mask = 0, int tiling = 0);
 
 // tcgen05 attention (attn_tc.cu): 16-bit types, head_dim 128.
 int32_t launch_attention_tc(int dtype, const void* q, const void* k, const void* v, void* out, const int32_t* k_lo,

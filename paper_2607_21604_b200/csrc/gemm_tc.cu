@@ -15,8 +15,9 @@
 // Epilogues: store (16-bit; a 128-column block that is one attention head gets its RoPE rotation
 // in registers), residual (h += acc as a vector reduction at the L2, nothing is read back),
 // SwiGLU.  A launch whose 128x256 tiles would occupy well under all SMs runs 128x128 tiles
-// (one B block per tile, `nh` = 1).  The kernel is launched as a programmatic dependent: its
-// set-up and the first weight tiles overlap the tail of the kernel before it.
+// (one B block per tile, `nh` = 1); a long launch runs on CTA pairs with 256x256 tiles
+// (gemm_tc_pair_kernel below, tcgen05.mma.cta_group::2).  The kernels are launched as
+// programmatic dependents: set-up and the first weight tiles overlap the tail of the kernel before.
 #include "tc_common.cuh"
 
 namespace {
@@ -56,6 +57,105 @@ __device__ __forceinline__ void locate(const GemmParams& p, int block, int& seg,
     ++seg;
   }
   row = block * BNH;
+}
+
+// Epilogue of one accumulator tile for one thread: its row `row` of the output, the 2 (or `nh`)
+// 128-column blocks of tile column `tn`; t_addr = the accumulator's tensor-memory address in the
+// warp's lane quadrant.
+template <int EPI, typename T>
+__device__ __forceinline__ void epilogue_row(const GemmParams& p, uint32_t t_addr, int row, int tn, int nh) {
+  if (EPI == EPI_SWIGLU) {
+    T* out = reinterpret_cast<T*>(p.seg_out[0]);
+    const int ldc = p.seg_ldc[0];
+    const int n_valid = p.seg_blocks[0] * BNH;
+#pragma unroll 1
+    for (int c = 0; c < BNH / 32; ++c) {
+      float g[32], u[32];
+      tc::tmem_ld32(t_addr + c * 32, g);
+      tc::tmem_ld32(t_addr + BNH + c * 32, u);
+      tc::tmem_ld_wait();
+      const int col = tn * BNH + c * 32;
+      if (row < p.M && col < n_valid) {
+        T* o = out + (size_t)row * ldc + col;
+#pragma unroll
+        for (int v = 0; v < 4; ++v) {
+          float r[8];
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            const float x = g[v * 8 + i];
+            r[i] = x / (1.f + __expf(-x)) * u[v * 8 + i];
+          }
+          st16(o + v * 8, r);
+        }
+      }
+    }
+  } else {
+#pragma unroll 1
+    for (int hf = 0; hf < nh; ++hf) {
+      int seg, brow;
+      locate(p, nh * tn + hf, seg, brow);
+      const bool valid = brow < p.seg_blocks[seg] * BNH;
+      const int ldc = p.seg_ldc[seg];
+      if (EPI == EPI_STORE && ((p.rope_mask >> seg) & 1)) {
+        // this 128-column block is one head: rotate the pairs (i, i + 64) in registers
+        const float2* rt = p.rope + (size_t)(row < p.M ? p.pos[row] : 0) * 64;
+#pragma unroll 1
+        for (int c = 0; c < 2; ++c) {
+          float lo[32], hi[32];
+          tc::tmem_ld32(t_addr + hf * BNH + c * 32, lo);
+          tc::tmem_ld32(t_addr + hf * BNH + 64 + c * 32, hi);
+          tc::tmem_ld_wait();
+          if (row < p.M && valid) {
+            T* o = reinterpret_cast<T*>(p.seg_out[seg]) + (size_t)row * ldc + brow + c * 32;
+#pragma unroll
+            for (int v = 0; v < 4; ++v) {
+              float rl[8], rh[8];
+#pragma unroll
+              for (int i = 0; i < 8; i += 2) {
+                const float4 cs = *reinterpret_cast<const float4*>(rt + c * 32 + v * 8 + i);   // two (cos, sin)
+                rl[i] = lo[v * 8 + i] * cs.x - hi[v * 8 + i] * cs.y;
+                rh[i] = hi[v * 8 + i] * cs.x + lo[v * 8 + i] * cs.y;
+                rl[i + 1] = lo[v * 8 + i + 1] * cs.z - hi[v * 8 + i + 1] * cs.w;
+                rh[i + 1] = hi[v * 8 + i + 1] * cs.z + lo[v * 8 + i + 1] * cs.w;
+              }
+              st16(o + v * 8, rl);
+              st16(o + 64 + v * 8, rh);
+            }
+          }
+        }
+        continue;
+      }
+#pragma unroll 1
+      for (int c = 0; c < BNH / 32; ++c) {
+        float a[32];
+        tc::tmem_ld32(t_addr + hf * BNH + c * 32, a);
+        tc::tmem_ld_wait();
+        if (row < p.M && valid) {
+          const int col = brow + c * 32;
+          if (EPI == EPI_RESID) {
+            float* o = reinterpret_cast<float*>(p.seg_out[seg]) + (size_t)row * ldc + col;
+#pragma unroll
+            for (int v = 0; v < 8; ++v) {
+              // h += acc as a reduction at the L2: one add per element as before (every element
+              // belongs to exactly one tile), but nothing comes back to the SM, so the epilogue
+              // does not sit through a load round trip per chunk
+              asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(o + v * 4), "f"(a[v * 4]),
+                           "f"(a[v * 4 + 1]), "f"(a[v * 4 + 2]), "f"(a[v * 4 + 3]) : "memory");
+            }
+          } else {
+            T* o = reinterpret_cast<T*>(p.seg_out[seg]) + (size_t)row * ldc + col;
+#pragma unroll
+            for (int v = 0; v < 4; ++v) {
+              float r[8];
+#pragma unroll
+              for (int i = 0; i < 8; ++i) r[i] = a[v * 8 + i];
+              st16(o + v * 8, r);
+            }
+          }
+        }
+      }
+    }
+  }
 }
 
 template <int EPI, typename T>
@@ -197,100 +297,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       const int tn = tile / p.tiles_m, tm = tile % p.tiles_m;
       if (!tc::mbar_wait(&acc_full[acc], (it >> 1) & 1, abort_flag)) { ok = false; break; }
       tc::fence_after_sync();
-      const int row = tm * BM + quad * 32 + lane;
-      const uint32_t t_addr = tmem_base + acc * (2 * BNH) + ((uint32_t)(quad * 32) << 16);
-      if (EPI == EPI_SWIGLU) {
-        T* out = reinterpret_cast<T*>(p.seg_out[0]);
-        const int ldc = p.seg_ldc[0];
-        const int n_valid = p.seg_blocks[0] * BNH;
-#pragma unroll 1
-        for (int c = 0; c < BNH / 32; ++c) {
-          float g[32], u[32];
-          tc::tmem_ld32(t_addr + c * 32, g);
-          tc::tmem_ld32(t_addr + BNH + c * 32, u);
-          tc::tmem_ld_wait();
-          const int col = tn * BNH + c * 32;
-          if (row < p.M && col < n_valid) {
-            T* o = out + (size_t)row * ldc + col;
-#pragma unroll
-            for (int v = 0; v < 4; ++v) {
-              float r[8];
-#pragma unroll
-              for (int i = 0; i < 8; ++i) {
-                const float x = g[v * 8 + i];
-                r[i] = x / (1.f + __expf(-x)) * u[v * 8 + i];
-              }
-              st16(o + v * 8, r);
-            }
-          }
-        }
-      } else {
-#pragma unroll 1
-        for (int hf = 0; hf < p.nh; ++hf) {
-          int seg, brow;
-          locate(p, p.nh * tn + hf, seg, brow);
-          const bool valid = brow < p.seg_blocks[seg] * BNH;
-          const int ldc = p.seg_ldc[seg];
-          if (EPI == EPI_STORE && ((p.rope_mask >> seg) & 1)) {
-            // this 128-column block is one head: rotate the pairs (i, i + 64) in registers
-            const float2* rt = p.rope + (size_t)(row < p.M ? p.pos[row] : 0) * 64;
-#pragma unroll 1
-            for (int c = 0; c < 2; ++c) {
-              float lo[32], hi[32];
-              tc::tmem_ld32(t_addr + hf * BNH + c * 32, lo);
-              tc::tmem_ld32(t_addr + hf * BNH + 64 + c * 32, hi);
-              tc::tmem_ld_wait();
-              if (row < p.M && valid) {
-                T* o = reinterpret_cast<T*>(p.seg_out[seg]) + (size_t)row * ldc + brow + c * 32;
-#pragma unroll
-                for (int v = 0; v < 4; ++v) {
-                  float rl[8], rh[8];
-#pragma unroll
-                  for (int i = 0; i < 8; i += 2) {
-                    const float4 cs = *reinterpret_cast<const float4*>(rt + c * 32 + v * 8 + i);   // two (cos, sin)
-                    rl[i] = lo[v * 8 + i] * cs.x - hi[v * 8 + i] * cs.y;
-                    rh[i] = hi[v * 8 + i] * cs.x + lo[v * 8 + i] * cs.y;
-                    rl[i + 1] = lo[v * 8 + i + 1] * cs.z - hi[v * 8 + i + 1] * cs.w;
-                    rh[i + 1] = hi[v * 8 + i + 1] * cs.z + lo[v * 8 + i + 1] * cs.w;
-                  }
-                  st16(o + v * 8, rl);
-                  st16(o + 64 + v * 8, rh);
-                }
-              }
-            }
-            continue;
-          }
-#pragma unroll 1
-          for (int c = 0; c < BNH / 32; ++c) {
-            float a[32];
-            tc::tmem_ld32(t_addr + hf * BNH + c * 32, a);
-            tc::tmem_ld_wait();
-            if (row < p.M && valid) {
-              const int col = brow + c * 32;
-              if (EPI == EPI_RESID) {
-                float* o = reinterpret_cast<float*>(p.seg_out[seg]) + (size_t)row * ldc + col;
-#pragma unroll
-                for (int v = 0; v < 8; ++v) {
-                  // h += acc as a reduction at the L2: one add per element as before (every element
-                  // belongs to exactly one tile), but nothing comes back to the SM, so the epilogue
-                  // does not sit through a load round trip per chunk
-                  asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(o + v * 4), "f"(a[v * 4]),
-                               "f"(a[v * 4 + 1]), "f"(a[v * 4 + 2]), "f"(a[v * 4 + 3]) : "memory");
-                }
-              } else {
-                T* o = reinterpret_cast<T*>(p.seg_out[seg]) + (size_t)row * ldc + col;
-#pragma unroll
-                for (int v = 0; v < 4; ++v) {
-                  float r[8];
-#pragma unroll
-                  for (int i = 0; i < 8; ++i) r[i] = a[v * 8 + i];
-                  st16(o + v * 8, r);
-                }
-              }
-            }
-          }
-        }
-      }
+      epilogue_row<EPI, T>(p, tmem_base + acc * (2 * BNH) + ((uint32_t)(quad * 32) << 16), tm * BM + quad * 32 + lane, tn,
+                           p.nh);
       tc::fence_before_sync();
       __syncwarp();
       if (lane == 0) tc::mbar_arrive(&acc_empty[acc]);
@@ -306,6 +314,182 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     __syncwarp();
     tc::fence_after_sync();
     tc::tmem_dealloc(tmem_base, 512);
+  }
+}
+
+// ---------------------------------------------------------------------------------------
+// The same GEMM on CTA pairs: a cluster of two CTAs (two SMs) works on one 256x256 tile with
+// tcgen05.mma.cta_group::2.  Each CTA stages its own 128 rows of x and only ITS 128 of the
+// tile's 256 weight rows (the pair's other half is read from the neighbour's shared memory by
+// the tensor core), so a k slab costs 32 KB of L2 -> SM traffic per SM instead of 48 KB, and
+// the ring is 6 stages deep.  Rank 0 issues the MMAs for both; each CTA holds the accumulator
+// of its 128 rows (2 x 256 columns, double-buffered) and runs the same epilogue as above.
+//   full[s]      rank 0's only: its producer announces the bytes of BOTH CTAs' slabs, both
+//                producers' loads report there
+//   empty[s]     one per CTA, signalled by one commit to both (the MMAs that read the stage)
+//   acc_full[a]  one per CTA, signalled by one commit to both
+//   acc_empty[a] rank 0's only: the 8 epilogue warps of the pair arrive there
+// ---------------------------------------------------------------------------------------
+constexpr int STAGES2 = 6;
+constexpr int PAIR_MIN_SLABS = 400;                           // k slabs per CTA from which pairs are used
+constexpr int STAGE2_BYTES = A_BYTES + BH_BYTES;             // 32768 per CTA
+constexpr int SMEM2_BYTES = STAGES2 * STAGE2_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+static_assert(SMEM2_BYTES <= 227 * 1024, "shared memory of the paired GEMM");
+static_assert((2 * STAGES2 + 4) * 8 + 8 <= 256, "barrier block of the paired GEMM");
+
+template <int EPI, typename T>
+__global__ void __launch_bounds__(THREADS, 1)
+gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB0,
+                    const __grid_constant__ CUtensorMap tmB1, const __grid_constant__ CUtensorMap tmB2,
+                    const GemmParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  // the dynamic shared memory starts at the same offset in both CTAs, so the aligned ring does too
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + STAGES2 * STAGE2_BYTES);
+  uint64_t* full = bars;                     // [STAGES2]
+  uint64_t* empty = bars + STAGES2;          // [STAGES2]
+  uint64_t* acc_full = bars + 2 * STAGES2;   // [2]
+  uint64_t* acc_empty = acc_full + 2;        // [2]
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = tc::cluster_ctarank();          // 0 issues the MMAs
+  const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+  const int KB = (p.K + BK - 1) / BK;
+  const int n_tiles = p.tiles_m * p.tiles_n;            // tiles_m counts 256-row tiles here
+  pdl_trigger();
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < STAGES2; ++i) { tc::mbar_init(&full[i], 1); tc::mbar_init(&empty[i], 1); }
+    for (int i = 0; i < 2; ++i) { tc::mbar_init(&acc_full[i], 1); tc::mbar_init(&acc_empty[i], 8); }
+    *abort_flag = 0;
+    tc::fence_barrier_init();
+    tc::fence_proxy_async();
+  }
+  if (warp == 1) {
+    tc::tmem_alloc_pair(tmem_slot, 512);
+    tc::tmem_relinquish_pair();
+  }
+  tc::fence_before_sync();
+  __syncthreads();
+  tc::cluster_sync_all();                    // the neighbour's barriers exist before anything is sent there
+  tc::fence_after_sync();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer (both CTAs)
+    if (lane == 0) {
+      tc::prefetch_tmap(&tmA);
+      tc::prefetch_tmap(&tmB0);
+      // this CTA's half of the tile's weight rows: block 2 tn + rank of the concatenated columns
+      auto b_half = [&](int tile, const CUtensorMap*& m, int& row) {
+        const int tn = tile / p.tiles_m;
+        int seg;
+        if (EPI == EPI_SWIGLU) {
+          seg = (int)rank; row = tn * BNH;
+        } else {
+          locate(p, 2 * tn + (int)rank, seg, row);
+        }
+        m = seg == 0 ? &tmB0 : (seg == 1 ? &tmB1 : &tmB2);
+      };
+      uint32_t full0[STAGES2];                // rank 0's full barriers as shared::cluster addresses
+      for (int i = 0; i < STAGES2; ++i) full0[i] = tc::map_to_rank(tc::smem_u32(&full[i]), 0);
+      const int pre = pair < n_tiles ? (KB < STAGES2 ? KB : STAGES2) : 0;
+      if (pre > 0) {
+        const CUtensorMap* m;
+        int row;
+        b_half(pair, m, row);
+        for (int kb = 0; kb < pre; ++kb) {
+          if (rank == 0) tc::mbar_expect_tx(&full[kb], 2 * STAGE2_BYTES);
+          tc::tma_load_2d_pair(smem + kb * STAGE2_BYTES + A_BYTES, m, kb * BK, row, full0[kb]);
+        }
+      }
+      pdl_wait();
+      for (int kb = 0; kb < pre; ++kb)
+        tc::tma_load_2d_pair(smem + kb * STAGE2_BYTES, &tmA, kb * BK, ((pair % p.tiles_m) * 2 + (int)rank) * BM, full0[kb]);
+      int s = pre % STAGES2;
+      uint32_t ph = pre == STAGES2 ? 1u : 0u;
+      int kb_start = pre;
+      bool ok = true;
+      for (int tile = pair; tile < n_tiles && ok; tile += n_pairs) {
+        const int tm = tile % p.tiles_m;
+        const CUtensorMap* m;
+        int row;
+        b_half(tile, m, row);
+        for (int kb = kb_start; kb < KB; ++kb) {
+          if (!tc::mbar_wait(&empty[s], ph ^ 1, abort_flag)) { ok = false; break; }
+          uint8_t* st = smem + s * STAGE2_BYTES;
+          if (rank == 0) tc::mbar_expect_tx(&full[s], 2 * STAGE2_BYTES);
+          tc::tma_load_2d_pair(st, &tmA, kb * BK, (tm * 2 + (int)rank) * BM, full0[s]);
+          tc::tma_load_2d_pair(st + A_BYTES, m, kb * BK, row, full0[s]);
+          if (++s == STAGES2) { s = 0; ph ^= 1; }
+        }
+        kb_start = 0;
+      }
+      if (!ok) { *abort_flag = 1; set_status(p.status, AKVS_ERR_TIMEOUT); }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer (rank 0 only)
+    if (lane == 0 && rank == 0) {
+      const uint32_t idesc = p.idesc;
+      int s = 0;
+      uint32_t ph = 0;
+      bool ok = true;
+      int it = 0;
+      for (int tile = pair; tile < n_tiles && ok; tile += n_pairs, ++it) {
+        const int acc = it & 1;
+        if (!tc::mbar_wait(&acc_empty[acc], ((it >> 1) & 1) ^ 1, abort_flag)) { ok = false; break; }
+        tc::fence_after_sync();
+        const uint32_t d_tmem = tmem_base + acc * (2 * BNH);
+        for (int kb = 0; kb < KB; ++kb) {
+          if (!tc::mbar_wait(&full[s], ph, abort_flag)) { ok = false; break; }
+          tc::fence_after_sync();
+          const uint32_t a_addr = tc::smem_u32(smem + s * STAGE2_BYTES);
+          const uint32_t b_addr = a_addr + A_BYTES;
+#pragma unroll
+          for (int k = 0; k < BK / 16; ++k) {
+            const uint64_t da = tc::smem_desc_k_sw128(a_addr + k * 32);
+            const uint64_t db = tc::smem_desc_k_sw128(b_addr + k * 32);
+            tc::mma_f16_pair(d_tmem, da, db, idesc, (kb | k) != 0);
+          }
+          tc::mma_commit_pair(&empty[s], 3);            // frees the stage in both CTAs
+          if (++s == STAGES2) { s = 0; ph ^= 1; }
+        }
+        if (ok) tc::mma_commit_pair(&acc_full[acc], 3);
+      }
+      if (!ok) { *abort_flag = 1; set_status(p.status, AKVS_ERR_TIMEOUT); }
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue (both CTAs)
+    const int quad = warp & 3;
+    const uint32_t acc_empty0[2] = {tc::map_to_rank(tc::smem_u32(&acc_empty[0]), 0),
+                                    tc::map_to_rank(tc::smem_u32(&acc_empty[1]), 0)};
+    pdl_wait();
+    bool ok = true;
+    int it = 0;
+    for (int tile = pair; tile < n_tiles && ok; tile += n_pairs, ++it) {
+      const int acc = it & 1;
+      const int tn = tile / p.tiles_m, tm = tile % p.tiles_m;
+      if (!tc::mbar_wait(&acc_full[acc], (it >> 1) & 1, abort_flag)) { ok = false; break; }
+      tc::fence_after_sync();
+      epilogue_row<EPI, T>(p, tmem_base + acc * (2 * BNH) + ((uint32_t)(quad * 32) << 16),
+                           (tm * 2 + (int)rank) * BM + quad * 32 + lane, tn, 2);
+      tc::fence_before_sync();
+      __syncwarp();
+      if (lane == 0) tc::mbar_arrive_cluster(acc_empty0[acc]);
+    }
+    if (!ok && lane == 0) { *abort_flag = 1; set_status(p.status, AKVS_ERR_TIMEOUT); }
+  }
+
+  // ---------------------------------------------------------------------- teardown
+  if (*abort_flag) __nanosleep(200000);       // let loads already in flight land before the CTA exits
+  tc::fence_before_sync();
+  __syncthreads();
+  tc::cluster_sync_all();                     // neither CTA's shared or tensor memory goes while the other may use it
+  if (warp == 1) {
+    tc::fence_after_sync();
+    tc::tmem_dealloc_pair(tmem_base, 512);
   }
 }
 
@@ -335,6 +519,51 @@ int sm_count() {
     if (g_sm_count <= 0) g_sm_count = 148;
   }
   return g_sm_count;
+}
+
+// Launch with clusters of two CTAs, as a programmatic dependent of the kernel before it.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl_pair(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  attr[1].id = cudaLaunchAttributeClusterDimension;
+  attr[1].val.clusterDim.x = 2;
+  attr[1].val.clusterDim.y = 1;
+  attr[1].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 2;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
+// How many CTA pairs of the paired GEMM the device runs at once (0: none, use single CTAs).
+int g_pair_count = -1;
+int pair_count() {
+  if (g_pair_count < 0) {
+    g_pair_count = 0;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2 * sm_count());
+    cfg.blockDim = dim3(THREADS);
+    cfg.dynamicSmemBytes = SMEM2_BYTES;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, gemm_tc_pair_kernel<EPI_STORE, f16>, &cfg) == cudaSuccess && n > 0)
+      g_pair_count = n;
+    else
+      cudaGetLastError();
+  }
+  return g_pair_count;
 }
 
 }  // namespace
@@ -375,7 +604,7 @@ int32_t encode_tmap_3d_16bit(CUtensorMap* map, const void* base, uint64_t d0, ui
 //   epi 2: out[0] = silu(x w[0]^T) * (x w[1]^T) (16-bit), n[0] == n[1].
 int32_t launch_linear_tc(int dtype, int epi, const void* x, int M, int K, int n_seg, const void* const* w, const int* n,
                          void* const* out, const int* ldc, int32_t* status, cudaStream_t st, const float2* rope,
-                         const int32_t* pos, int rope_mask) {
+                         const int32_t* pos, int rope_mask, int tiling) {
   if (M == 0) return AKVS_OK;
   if (K % 8 != 0 || n_seg < 1 || n_seg > 3) return AKVS_ERR_SHAPE;
   if (dtype != AKVS_BF16 && dtype != AKVS_F16) return AKVS_ERR_UNSUPPORTED;
@@ -387,6 +616,12 @@ int32_t launch_linear_tc(int dtype, int epi, const void* x, int M, int K, int n_
     AKVS_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI_STORE, f16>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES));
     AKVS_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI_RESID, f16>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES));
     AKVS_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI_SWIGLU, f16>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES));
+    AKVS_CUDA(cudaFuncSetAttribute(gemm_tc_pair_kernel<EPI_STORE, bf16>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM2_BYTES));
+    AKVS_CUDA(cudaFuncSetAttribute(gemm_tc_pair_kernel<EPI_RESID, bf16>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM2_BYTES));
+    AKVS_CUDA(cudaFuncSetAttribute(gemm_tc_pair_kernel<EPI_SWIGLU, bf16>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM2_BYTES));
+    AKVS_CUDA(cudaFuncSetAttribute(gemm_tc_pair_kernel<EPI_STORE, f16>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM2_BYTES));
+    AKVS_CUDA(cudaFuncSetAttribute(gemm_tc_pair_kernel<EPI_RESID, f16>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM2_BYTES));
+    AKVS_CUDA(cudaFuncSetAttribute(gemm_tc_pair_kernel<EPI_SWIGLU, f16>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM2_BYTES));
     attr_set = true;
   }
   GemmParams p;
@@ -424,13 +659,44 @@ int32_t launch_linear_tc(int dtype, int epi, const void* x, int M, int K, int n_
     if (cost1 < 0.9 * cost2) p.nh = 1;
     p.tiles_n = (blocks + p.nh - 1) / p.nh;
   }
-  p.idesc = tc::idesc_f16(fmt, fmt, BM, p.nh * BNH, 0);
-  const int n_tiles = p.tiles_m * p.tiles_n;
-  const int grid = n_tiles < sm_count() ? n_tiles : sm_count();
   double flops = 0;
   for (int i = 0; i < n_seg; ++i) flops += 2.0 * M * (double)n[i] * K;
   ProfScope prof(1, epi, flops, st);
   if (epi < 0 || epi > 2) return AKVS_ERR_INVALID_ARG;
+  // CTA pairs on 256x256 tiles when that takes no more rounds than single CTAs on 128x256 tiles
+  // and the launch is long enough (k slabs per CTA) to repay the pair's slower start: measured
+  // on the 8B shapes, the pair's main loop is ~8 % faster (a third less operand data per SM)
+  // and its launch ~10 us longer.  tiling 1 / 2 force single CTAs / pairs (tests, comparisons).
+  const int pairs = tiling == 1 ? 0 : pair_count();
+  if ((p.nh == 2 || tiling == 2) && pairs > 0 && M > BM) {
+    if (p.nh == 1) { p.nh = 2; p.tiles_n = (blocks + 1) / 2; }
+    const int tiles_m2 = (M + 2 * BM - 1) / (2 * BM);
+    const int t_pair = tiles_m2 * p.tiles_n, t_single = p.tiles_m * p.tiles_n;
+    const int r_pair = (t_pair + pairs - 1) / pairs, r_single = (t_single + sm_count() - 1) / sm_count();
+    const int KB = (K + BK - 1) / BK;
+    if (tiling == 2 || (r_pair <= r_single && (long long)r_pair * KB >= PAIR_MIN_SLABS)) {
+      p.tiles_m = tiles_m2;
+      p.idesc = tc::idesc_f16(fmt, fmt, 2 * BM, 2 * BNH, 0);
+      const int n_pairs = t_pair < pairs ? t_pair : pairs;
+#define AKVS_GEMM_LAUNCH(E, T) \
+  AKVS_CUDA(launch_pdl_pair(gemm_tc_pair_kernel<E, T>, dim3(2 * n_pairs), dim3(THREADS), SMEM2_BYTES, st, tmA, tmB[0], tmB[1], tmB[2], p))
+      if (dtype == AKVS_BF16) {
+        if (epi == EPI_STORE) AKVS_GEMM_LAUNCH(EPI_STORE, bf16);
+        else if (epi == EPI_RESID) AKVS_GEMM_LAUNCH(EPI_RESID, bf16);
+        else AKVS_GEMM_LAUNCH(EPI_SWIGLU, bf16);
+      } else {
+        if (epi == EPI_STORE) AKVS_GEMM_LAUNCH(EPI_STORE, f16);
+        else if (epi == EPI_RESID) AKVS_GEMM_LAUNCH(EPI_RESID, f16);
+        else AKVS_GEMM_LAUNCH(EPI_SWIGLU, f16);
+      }
+#undef AKVS_GEMM_LAUNCH
+      AKVS_LAUNCHED();
+      return AKVS_OK;
+    }
+  }
+  p.idesc = tc::idesc_f16(fmt, fmt, BM, p.nh * BNH, 0);
+  const int n_tiles = p.tiles_m * p.tiles_n;
+  const int grid = n_tiles < sm_count() ? n_tiles : sm_count();
 #define AKVS_GEMM_LAUNCH(E, T) \
   AKVS_CUDA(launch_pdl(gemm_tc_kernel<E, T>, dim3(grid), dim3(THREADS), SMEM_BYTES, st, tmA, tmB[0], tmB[1], tmB[2], p))
   if (dtype == AKVS_BF16) {

@@ -31,7 +31,7 @@ H16 = [torch.bfloat16, torch.float16]
 
 @pytest.mark.parametrize("M,N,K", [(1, 128, 64), (77, 256, 200), (128, 128, 64), (130, 384, 1024), (1357, 1024, 4096),
                                    (300, 11008, 2048)])
-@pytest.mark.parametrize("algo", [0, 1])
+@pytest.mark.parametrize("algo", [0, 1, 2, 3])      # by shape, CUDA cores, single CTAs, CTA pairs
 @pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float16])
 def test_linear_16bit(akvs, M, N, K, algo, dtype):
     g = np.random.default_rng(M * 7 + N)
@@ -55,17 +55,19 @@ def test_linear_f32(akvs, M, N, K):
     assert orc.rel_l2(n64(y), n64(x) @ n64(w).T) < 1e-6
 
 
+@pytest.mark.parametrize("algo", [2, 3])
 @pytest.mark.parametrize("dtype", H16)
-def test_linear_16bit_full_size_sampled(akvs, dtype):
-    """Config-3 MLP shape; the oracle checks sampled outputs one by one."""
+def test_linear_16bit_full_size_sampled(akvs, dtype, algo):
+    """Config-3 MLP shape on single CTAs and on CTA pairs (the last pair's second CTA holds no
+    row: M = 10 x 256 + 26); the oracle checks sampled outputs one by one."""
     g = torch.Generator(device="cuda").manual_seed(5)
     M, N, K = 2586, 4096, 14336
     x = torch.randn((M, K), generator=g, device="cuda").to(dtype)
     w = (torch.randn((N, K), generator=g, device="cuda") * 0.02).to(dtype)
-    y = akvs.op_linear(x, w, 0)
+    y = akvs.op_linear(x, w, algo)
     torch.cuda.synchronize()
     rs = np.random.default_rng(0)
-    rows = np.concatenate([[0, 127, 128, M - 1], rs.integers(0, M, 60)])
+    rows = np.concatenate([[0, 127, 128, 255, 256, 2559, 2560, M - 1], rs.integers(0, M, 60)])
     cols = np.concatenate([[0, 255, 256, N - 1], rs.integers(0, N, 60)])
     xr, wc = n64(x[rows]), n64(w[cols])
     ref = xr @ wc.T

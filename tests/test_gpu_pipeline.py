@@ -113,6 +113,20 @@ def test_small16_all_modes(dtype, scale):
     _run_all_modes(case, 2500, 2, units)
 
 
+@pytest.mark.parametrize("dtype,scale", SMALL16)
+def test_small16_all_modes_linear_layers_on_cta_pairs(dtype, scale):
+    """The same with every tensor-core linear layer of more than 128 rows forced onto the
+    CTA-pair kernel (fused RoPE, residual and SwiGLU epilogues), which the shapes of this small
+    model would not pick by themselves."""
+    case = Case(small16(dtype), std_scale=scale)
+    case.akvs.lib.akvs_debug_set_linear_algo(2 << 2)
+    try:
+        units = _check_encode(case, case.tol)
+        _run_all_modes(case, 2500, 2, units)
+    finally:
+        case.akvs.lib.akvs_debug_set_linear_algo(0)
+
+
 @pytest.mark.parametrize("kv_format", [4, 2])
 @pytest.mark.parametrize("dtype,scale", SMALL16)
 def test_small16_quantised_cache(kv_format, dtype, scale):
