@@ -30,7 +30,7 @@ SEED_W, SEED_IDS, SEED_LEN = 1234, 1235, 1236
 METRIC = "context tokens/s prefilled (corrected reuse, 15% refresh)"
 UNIT = "tokens/s"
 CHECK_LAYER = 2
-# dram__bytes_read.sum + dram__bytes_write.sum per gemm_tc_kernel launch (bytes), averaged over
+# dram__bytes_read.sum + dram__bytes_write.sum per linear-layer launch (bytes), averaged over
 # the four linear-layer launches of one selective layer, from the ncu --set full capture
 # summarised in profiles/selective_layer_kernels_c3.md (algorithmic: 201 MB per launch)
 GEMM_TRAFFIC_PER_LAUNCH = {"c3": 202.2e6}
@@ -325,7 +325,7 @@ def main():
                            "frac": c_by / (c_ms * 1e-3) / 1e9 / pk["hbm"] if c_ms > 0 else None,
                            "ms_per_step": c_ms / args.steps, "launches_per_step": len(corr) / args.steps,
                            "bytes_per_launch": c_by / max(1, len(corr))}}
-    roofline = {"bound": "tensor", "kernel": "gemm_tc_kernel (all linear layers of the step)",
+    roofline = {"bound": "tensor", "kernel": "gemm_tc_kernel + gemm_tc_pair_kernel (all linear layers of the step)",
                 "achieved": achieved, "peak": pk["tensor"], "unit": "TFLOP/s", "frac": achieved / pk["tensor"],
                 "peak_source": pk["src"] + " bf16 cuBLAS sustained (f16 and bf16 MMAs run at the same rate)",
                 "traffic": GEMM_TRAFFIC_PER_LAUNCH.get(args.workload) if B == 1 else None, "launches": len(gemm),
