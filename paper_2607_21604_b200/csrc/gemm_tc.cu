@@ -15,8 +15,8 @@
 // Epilogues: store (16-bit; a 128-column block that is one attention head gets its RoPE rotation
 // in registers), residual (h += acc as a vector reduction at the L2, nothing is read back),
 // SwiGLU.  A launch whose 128x256 tiles would occupy well under all SMs runs 128x128 tiles
-// (one B block per tile, `nh` = 1); a long launch runs on CTA pairs with 256x256 tiles
-// (gemm_tc_pair_kernel below, tcgen05.mma.cta_group::2).  The kernels are launched as
+// (one B block per tile, `nh` = 1); every other launch of more than 128 rows runs on CTA pairs
+// with 256x256 tiles (gemm_tc_pair_kernel below, tcgen05.mma.cta_group::2).  The kernels are launched as
 // programmatic dependents: set-up and the first weight tiles overlap the tail of the kernel before.
 #include "tc_common.cuh"
 
@@ -331,7 +331,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 //   acc_empty[a] rank 0's only: the 8 epilogue warps of the pair arrive there
 // ---------------------------------------------------------------------------------------
 constexpr int STAGES2 = 6;
-constexpr int PAIR_MIN_SLABS = 400;                           // k slabs per CTA from which pairs are used
 constexpr int STAGE2_BYTES = A_BYTES + BH_BYTES;             // 32768 per CTA
 constexpr int SMEM2_BYTES = STAGES2 * STAGE2_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
 static_assert(SMEM2_BYTES <= 227 * 1024, "shared memory of the paired GEMM");
@@ -663,18 +662,17 @@ int32_t launch_linear_tc(int dtype, int epi, const void* x, int M, int K, int n_
   for (int i = 0; i < n_seg; ++i) flops += 2.0 * M * (double)n[i] * K;
   ProfScope prof(1, epi, flops, st);
   if (epi < 0 || epi > 2) return AKVS_ERR_INVALID_ARG;
-  // CTA pairs on 256x256 tiles when that takes no more rounds than single CTAs on 128x256 tiles
-  // and the launch is long enough (k slabs per CTA) to repay the pair's slower start: measured
-  // on the 8B shapes, the pair's main loop is ~8 % faster (a third less operand data per SM)
-  // and its launch ~10 us longer.  tiling 1 / 2 force single CTAs / pairs (tests, comparisons).
+  // CTA pairs on 256x256 tiles when that takes no more rounds than single CTAs on 128x256 tiles:
+  // a tile takes the same number of MMA cycles either way, and the pair moves a third less
+  // operand data per SM (measured on the 8B shapes: main loop ~8 % faster under the power cap).
+  // tiling 1 / 2 force single CTAs / pairs (tests, comparisons).
   const int pairs = tiling == 1 ? 0 : pair_count();
   if ((p.nh == 2 || tiling == 2) && pairs > 0 && M > BM) {
     if (p.nh == 1) { p.nh = 2; p.tiles_n = (blocks + 1) / 2; }
     const int tiles_m2 = (M + 2 * BM - 1) / (2 * BM);
     const int t_pair = tiles_m2 * p.tiles_n, t_single = p.tiles_m * p.tiles_n;
     const int r_pair = (t_pair + pairs - 1) / pairs, r_single = (t_single + sm_count() - 1) / sm_count();
-    const int KB = (K + BK - 1) / BK;
-    if (tiling == 2 || (r_pair <= r_single && (long long)r_pair * KB >= PAIR_MIN_SLABS)) {
+    if (tiling == 2 || r_pair <= r_single) {
       p.tiles_m = tiles_m2;
       p.idesc = tc::idesc_f16(fmt, fmt, 2 * BM, 2 * BNH, 0);
       const int n_pairs = t_pair < pairs ? t_pair : pairs;
