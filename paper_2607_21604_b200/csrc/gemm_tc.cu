@@ -25,7 +25,10 @@ namespace {
 constexpr int BM = 128, BNH = 128, BK = 64, STAGES = 4;
 constexpr int A_BYTES = BM * BK * 2, BH_BYTES = BNH * BK * 2;
 constexpr int STAGE_BYTES = A_BYTES + 2 * BH_BYTES;        // 49152
-constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr int EPI_PITCH = 144;                             // bytes between staged rows: 128 of payload + 16
+constexpr int EPI_STAGE_BYTES = 32 * EPI_PITCH;            // staging tile of one epilogue warp
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/ + 4 * EPI_STAGE_BYTES;
+static_assert(SMEM_BYTES <= 227 * 1024, "shared memory of the GEMM");
 constexpr int THREADS = 192;
 
 enum { EPI_STORE = 0, EPI_RESID = 1, EPI_SWIGLU = 2 };
@@ -59,98 +62,147 @@ __device__ __forceinline__ void locate(const GemmParams& p, int block, int& seg,
   row = block * BNH;
 }
 
-// Epilogue of one accumulator tile for one thread: its row `row` of the output, the 2 (or `nh`)
-// 128-column blocks of tile column `tn`; t_addr = the accumulator's tensor-memory address in the
-// warp's lane quadrant.
-template <int EPI, typename T>
-__device__ __forceinline__ void epilogue_row(const GemmParams& p, uint32_t t_addr, int row, int tn, int nh) {
-  if (EPI == EPI_SWIGLU) {
-    T* out = reinterpret_cast<T*>(p.seg_out[0]);
-    const int ldc = p.seg_ldc[0];
-    const int n_valid = p.seg_blocks[0] * BNH;
+// SwiGLU epilogue of one accumulator tile for one thread: its row `row` of the output, tile column
+// `tn`; t_addr = the accumulator's tensor-memory address in the warp's lane quadrant.  Stores
+// straight from the row-per-thread layout of tcgen05.ld (64 contiguous bytes per thread and
+// chunk).  Staging these through shared memory like the other epilogues measured 4 % SLOWER on
+// the 14-round W_gate/W_up launch: every tile but the last overlaps the next tile's main loop,
+// whose MMAs want the shared-memory bandwidth to themselves, and the tail is short here.
+template <typename T>
+__device__ __forceinline__ void epilogue_swiglu_row(const GemmParams& p, uint32_t t_addr, int row, int tn) {
+  T* out = reinterpret_cast<T*>(p.seg_out[0]);
+  const int ldc = p.seg_ldc[0];
+  const int n_valid = p.seg_blocks[0] * BNH;
 #pragma unroll 1
-    for (int c = 0; c < BNH / 32; ++c) {
-      float g[32], u[32];
-      tc::tmem_ld32(t_addr + c * 32, g);
-      tc::tmem_ld32(t_addr + BNH + c * 32, u);
-      tc::tmem_ld_wait();
-      const int col = tn * BNH + c * 32;
-      if (row < p.M && col < n_valid) {
-        T* o = out + (size_t)row * ldc + col;
+  for (int c = 0; c < BNH / 32; ++c) {
+    float g[32], u[32];
+    tc::tmem_ld32(t_addr + c * 32, g);
+    tc::tmem_ld32(t_addr + BNH + c * 32, u);
+    tc::tmem_ld_wait();
+    const int col = tn * BNH + c * 32;
+    if (row < p.M && col < n_valid) {
+      T* o = out + (size_t)row * ldc + col;
 #pragma unroll
-        for (int v = 0; v < 4; ++v) {
-          float r[8];
+      for (int v = 0; v < 4; ++v) {
+        float r[8];
 #pragma unroll
-          for (int i = 0; i < 8; ++i) {
-            const float x = g[v * 8 + i];
-            r[i] = x / (1.f + __expf(-x)) * u[v * 8 + i];
-          }
-          st16(o + v * 8, r);
+        for (int i = 0; i < 8; ++i) {
+          const float x = g[v * 8 + i];
+          r[i] = x / (1.f + __expf(-x)) * u[v * 8 + i];
         }
+        st16(o + v * 8, r);
       }
     }
-  } else {
+  }
+}
+
+// Store and residual epilogues of one accumulator tile for one warp: the 32 rows row0 .. row0+31
+// of the output, the 2 (or `nh`) 128-column blocks of tile column `tn`.  tcgen05.ld hands each
+// thread ONE ROW (32 columns per load); storing from that layout sends 32 rows x 16 bytes per
+// instruction - 32 separate lines - and the last tile's epilogue is the exposed tail of the
+// launch.  So each chunk goes through a per-warp staging tile in shared memory (32 rows x 128
+// bytes, row pitch 144 bytes so that 16-byte accesses of a quarter warp fall on distinct banks)
+// and leaves it as whole 128-byte (64 for the rotated heads) row segments, 8 lanes per row
+// (measured on the 8B shapes: QKV -5 us, W_o -10 us, W_down -7 us per launch).
+template <int EPI, typename T>
+__device__ __forceinline__ void epilogue_warp(const GemmParams& p, uint32_t t_addr, int row0, int lane, int tn, int nh,
+                                              uint8_t* stage) {
+  const int row = row0 + lane;                  // the row this thread holds after tcgen05.ld
+  uint8_t* mine = stage + lane * EPI_PITCH;
+  const int q = lane & 7, rsub = lane >> 3;     // on the way out: 16-byte piece q of staged row 4 i + rsub
 #pragma unroll 1
-    for (int hf = 0; hf < nh; ++hf) {
-      int seg, brow;
-      locate(p, nh * tn + hf, seg, brow);
-      const bool valid = brow < p.seg_blocks[seg] * BNH;
-      const int ldc = p.seg_ldc[seg];
-      if (EPI == EPI_STORE && ((p.rope_mask >> seg) & 1)) {
-        // this 128-column block is one head: rotate the pairs (i, i + 64) in registers
-        const float2* rt = p.rope + (size_t)(row < p.M ? p.pos[row] : 0) * 64;
+  for (int hf = 0; hf < nh; ++hf) {
+    int seg, brow;
+    locate(p, nh * tn + hf, seg, brow);
+    const bool valid = brow < p.seg_blocks[seg] * BNH;
+    const int ldc = p.seg_ldc[seg];
+    if (EPI == EPI_STORE && ((p.rope_mask >> seg) & 1)) {
+      // this 128-column block is one head: rotate the pairs (i, i + 64) in registers
+      const float2* rt = p.rope + (size_t)(row < p.M ? p.pos[row] : 0) * 64;
+      T* out = reinterpret_cast<T*>(p.seg_out[seg]);
 #pragma unroll 1
-        for (int c = 0; c < 2; ++c) {
-          float lo[32], hi[32];
-          tc::tmem_ld32(t_addr + hf * BNH + c * 32, lo);
-          tc::tmem_ld32(t_addr + hf * BNH + 64 + c * 32, hi);
-          tc::tmem_ld_wait();
-          if (row < p.M && valid) {
-            T* o = reinterpret_cast<T*>(p.seg_out[seg]) + (size_t)row * ldc + brow + c * 32;
+      for (int c = 0; c < 2; ++c) {
+        float lo[32], hi[32];
+        tc::tmem_ld32(t_addr + hf * BNH + c * 32, lo);
+        tc::tmem_ld32(t_addr + hf * BNH + 64 + c * 32, hi);
+        tc::tmem_ld_wait();
+        __syncwarp();
 #pragma unroll
-            for (int v = 0; v < 4; ++v) {
-              float rl[8], rh[8];
+        for (int v = 0; v < 4; ++v) {
+          float rl[8], rh[8];
 #pragma unroll
-              for (int i = 0; i < 8; i += 2) {
-                const float4 cs = *reinterpret_cast<const float4*>(rt + c * 32 + v * 8 + i);   // two (cos, sin)
-                rl[i] = lo[v * 8 + i] * cs.x - hi[v * 8 + i] * cs.y;
-                rh[i] = hi[v * 8 + i] * cs.x + lo[v * 8 + i] * cs.y;
-                rl[i + 1] = lo[v * 8 + i + 1] * cs.z - hi[v * 8 + i + 1] * cs.w;
-                rh[i + 1] = hi[v * 8 + i + 1] * cs.z + lo[v * 8 + i + 1] * cs.w;
-              }
-              st16(o + v * 8, rl);
-              st16(o + 64 + v * 8, rh);
-            }
+          for (int i = 0; i < 8; i += 2) {
+            const float4 cs = *reinterpret_cast<const float4*>(rt + c * 32 + v * 8 + i);   // two (cos, sin)
+            rl[i] = lo[v * 8 + i] * cs.x - hi[v * 8 + i] * cs.y;
+            rh[i] = hi[v * 8 + i] * cs.x + lo[v * 8 + i] * cs.y;
+            rl[i + 1] = lo[v * 8 + i + 1] * cs.z - hi[v * 8 + i + 1] * cs.w;
+            rh[i + 1] = hi[v * 8 + i + 1] * cs.z + lo[v * 8 + i + 1] * cs.w;
           }
+          st16(reinterpret_cast<T*>(mine + v * 16), rl);          // bytes 0..63: columns c*32 .. +31
+          st16(reinterpret_cast<T*>(mine + 64 + v * 16), rh);     // bytes 64..127: columns 64 + c*32 .. +31
         }
-        continue;
+        __syncwarp();
+        const int col = brow + (q < 4 ? c * 32 + q * 8 : 64 + c * 32 + (q - 4) * 8);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          const int rr = 4 * i + rsub, grow = row0 + rr;
+          if (grow < p.M && valid)
+            *reinterpret_cast<uint4*>(out + (size_t)grow * ldc + col) =
+                *reinterpret_cast<const uint4*>(stage + rr * EPI_PITCH + q * 16);
+        }
       }
+      continue;
+    }
+    if (EPI == EPI_RESID) {
+      float* out = reinterpret_cast<float*>(p.seg_out[seg]);
 #pragma unroll 1
       for (int c = 0; c < BNH / 32; ++c) {
         float a[32];
         tc::tmem_ld32(t_addr + hf * BNH + c * 32, a);
         tc::tmem_ld_wait();
-        if (row < p.M && valid) {
-          const int col = brow + c * 32;
-          if (EPI == EPI_RESID) {
-            float* o = reinterpret_cast<float*>(p.seg_out[seg]) + (size_t)row * ldc + col;
+        __syncwarp();
 #pragma unroll
-            for (int v = 0; v < 8; ++v) {
-              // h += acc as a reduction at the L2: one add per element as before (every element
-              // belongs to exactly one tile), but nothing comes back to the SM, so the epilogue
-              // does not sit through a load round trip per chunk
-              asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(o + v * 4), "f"(a[v * 4]),
-                           "f"(a[v * 4 + 1]), "f"(a[v * 4 + 2]), "f"(a[v * 4 + 3]) : "memory");
-            }
-          } else {
-            T* o = reinterpret_cast<T*>(p.seg_out[seg]) + (size_t)row * ldc + col;
+        for (int v = 0; v < 8; ++v)
+          *reinterpret_cast<float4*>(mine + v * 16) = make_float4(a[v * 4], a[v * 4 + 1], a[v * 4 + 2], a[v * 4 + 3]);
+        __syncwarp();
+        const int col = brow + c * 32 + q * 4;
 #pragma unroll
-            for (int v = 0; v < 4; ++v) {
-              float r[8];
+        for (int i = 0; i < 8; ++i) {
+          const int rr = 4 * i + rsub, grow = row0 + rr;
+          if (grow < p.M && valid) {
+            // h += acc as a reduction at the L2: one add per element (every element belongs to
+            // exactly one tile) and nothing comes back to the SM, so the epilogue does not sit
+            // through a load round trip per chunk
+            const float4 a4 = *reinterpret_cast<const float4*>(stage + rr * EPI_PITCH + q * 16);
+            asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(out + (size_t)grow * ldc + col), "f"(a4.x),
+                         "f"(a4.y), "f"(a4.z), "f"(a4.w) : "memory");
+          }
+        }
+      }
+    } else {
+      T* out = reinterpret_cast<T*>(p.seg_out[seg]);
+#pragma unroll 1
+      for (int c = 0; c < BNH / 32; ++c) {
+        float a[32];
+        tc::tmem_ld32(t_addr + hf * BNH + c * 32, a);
+        tc::tmem_ld_wait();
+        if ((c & 1) == 0) __syncwarp();
 #pragma unroll
-              for (int i = 0; i < 8; ++i) r[i] = a[v * 8 + i];
-              st16(o + v * 8, r);
-            }
+        for (int v = 0; v < 4; ++v) {
+          float r[8];
+#pragma unroll
+          for (int i = 0; i < 8; ++i) r[i] = a[v * 8 + i];
+          st16(reinterpret_cast<T*>(mine + (c & 1) * 64 + v * 16), r);
+        }
+        if (c & 1) {
+          __syncwarp();
+          const int col = brow + (c - 1) * 32 + q * 8;
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            const int rr = 4 * i + rsub, grow = row0 + rr;
+            if (grow < p.M && valid)
+              *reinterpret_cast<uint4*>(out + (size_t)grow * ldc + col) =
+                  *reinterpret_cast<const uint4*>(stage + rr * EPI_PITCH + q * 16);
           }
         }
       }
@@ -297,8 +349,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       const int tn = tile / p.tiles_m, tm = tile % p.tiles_m;
       if (!tc::mbar_wait(&acc_full[acc], (it >> 1) & 1, abort_flag)) { ok = false; break; }
       tc::fence_after_sync();
-      epilogue_row<EPI, T>(p, tmem_base + acc * (2 * BNH) + ((uint32_t)(quad * 32) << 16), tm * BM + quad * 32 + lane, tn,
-                           p.nh);
+      const uint32_t t_addr = tmem_base + acc * (2 * BNH) + ((uint32_t)(quad * 32) << 16);
+      if (EPI == EPI_SWIGLU)
+        epilogue_swiglu_row<T>(p, t_addr, tm * BM + quad * 32 + lane, tn);
+      else
+        epilogue_warp<EPI, T>(p, t_addr, tm * BM + quad * 32, lane, tn, p.nh,
+                              smem + STAGES * STAGE_BYTES + 256 + (warp - 2) * EPI_STAGE_BYTES);
       tc::fence_before_sync();
       __syncwarp();
       if (lane == 0) tc::mbar_arrive(&acc_empty[acc]);
@@ -332,7 +388,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 // ---------------------------------------------------------------------------------------
 constexpr int STAGES2 = 6;
 constexpr int STAGE2_BYTES = A_BYTES + BH_BYTES;             // 32768 per CTA
-constexpr int SMEM2_BYTES = STAGES2 * STAGE2_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr int SMEM2_BYTES = STAGES2 * STAGE2_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/ + 4 * EPI_STAGE_BYTES;
 static_assert(SMEM2_BYTES <= 227 * 1024, "shared memory of the paired GEMM");
 static_assert((2 * STAGES2 + 4) * 8 + 8 <= 256, "barrier block of the paired GEMM");
 
@@ -472,8 +528,13 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       const int tn = tile / p.tiles_m, tm = tile % p.tiles_m;
       if (!tc::mbar_wait(&acc_full[acc], (it >> 1) & 1, abort_flag)) { ok = false; break; }
       tc::fence_after_sync();
-      epilogue_row<EPI, T>(p, tmem_base + acc * (2 * BNH) + ((uint32_t)(quad * 32) << 16),
-                           (tm * 2 + (int)rank) * BM + quad * 32 + lane, tn, 2);
+      const uint32_t t_addr = tmem_base + acc * (2 * BNH) + ((uint32_t)(quad * 32) << 16);
+      const int row0 = (tm * 2 + (int)rank) * BM + quad * 32;
+      if (EPI == EPI_SWIGLU)
+        epilogue_swiglu_row<T>(p, t_addr, row0 + lane, tn);
+      else
+        epilogue_warp<EPI, T>(p, t_addr, row0, lane, tn, 2,
+                              smem + STAGES2 * STAGE2_BYTES + 256 + (warp - 2) * EPI_STAGE_BYTES);
       tc::fence_before_sync();
       __syncwarp();
       if (lane == 0) tc::mbar_arrive_cluster(acc_empty0[acc]);
