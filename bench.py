@@ -33,7 +33,7 @@ CHECK_LAYER = 2
 # dram__bytes_read.sum + dram__bytes_write.sum per linear-layer launch (bytes), averaged over
 # the four linear-layer launches of one selective layer, from the ncu --set full capture
 # summarised in profiles/selective_layer_kernels_c3.md (algorithmic: 201 MB per launch)
-GEMM_TRAFFIC_PER_LAUNCH = {"c3": 202.2e6}
+GEMM_TRAFFIC_PER_LAUNCH = {"c3": 203.3e6}
 
 
 def peaks():
