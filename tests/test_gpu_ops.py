@@ -30,7 +30,7 @@ H16 = [torch.bfloat16, torch.float16]
 # ----------------------------------------------------------------------------- linear layers
 
 @pytest.mark.parametrize("M,N,K", [(1, 128, 64), (77, 256, 200), (128, 128, 64), (130, 384, 1024), (1357, 1024, 4096),
-                                   (300, 11008, 2048)])
+                                   (300, 11008, 2048), (200, 384, 200), (257, 640, 72)])
 @pytest.mark.parametrize("algo", [0, 1, 2, 3])      # by shape, CUDA cores, single CTAs, CTA pairs
 @pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float16])
 def test_linear_16bit(akvs, M, N, K, algo, dtype):
