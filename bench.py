@@ -284,7 +284,7 @@ def main():
     ms_step = timed(step, args.steps, 0)
     ms_median, ms_best = float(np.median(step_times)), float(min(step_times))
     launches = akvs.launch_count() - launches0 + graph_launches * args.steps
-    akvs.prof_enable((1 << 1) | (1 << 2) | (1 << 3), 8192)
+    akvs.prof_enable((1 << 1) | (1 << 2) | (1 << 3) | (1 << 4) | (1 << 5), 8192)
     step()
     barrier()
     akvs.prof_reset()
@@ -299,6 +299,8 @@ def main():
     gemm = [r for r in recs if r[2] >> 8 == 1]
     corr = [r for r in recs if r[2] >> 8 == 2]
     attn = [r for r in recs if r[2] >> 8 == 3]
+    norm = [r for r in recs if r[2] >> 8 == 4]
+    offs = [r for r in recs if r[2] >> 8 == 5]
     g_ms = sum(r[0] for r in gemm)
     g_fl = sum(r[1] for r in gemm)
     by_epi = {}
@@ -324,7 +326,12 @@ def main():
         "correct_kernel": {"bound": "hbm", "gbs": c_by / (c_ms * 1e-3) / 1e9 if c_ms > 0 else None,
                            "frac": c_by / (c_ms * 1e-3) / 1e9 / pk["hbm"] if c_ms > 0 else None,
                            "ms_per_step": c_ms / args.steps, "launches_per_step": len(corr) / args.steps,
-                           "bytes_per_launch": c_by / max(1, len(corr))}}
+                           "bytes_per_launch": c_by / max(1, len(corr))},
+        "rmsnorm_kernel": {"bound": "hbm", "gbs": sum(r[1] for r in norm) / (sum(r[0] for r in norm) * 1e-3) / 1e9
+                           if norm else None, "ms_per_step": sum(r[0] for r in norm) / args.steps,
+                           "launches_per_step": len(norm) / args.steps},
+        "offsets_kernel": {"bound": "hbm/latency", "ms_per_step": sum(r[0] for r in offs) / args.steps,
+                           "launches_per_step": len(offs) / args.steps}}
     roofline = {"bound": "tensor", "kernel": "gemm_tc_kernel + gemm_tc_pair_kernel (all linear layers of the step)",
                 "achieved": achieved, "peak": pk["tensor"], "unit": "TFLOP/s", "frac": achieved / pk["tensor"],
                 "peak_source": pk["src"] + " bf16 cuBLAS sustained (f16 and bf16 MMAs run at the same rate)",

@@ -210,7 +210,8 @@ int64_t akvs_launch_count(void);
 /* Per-launch device timing of kernel classes with CUDA events recorded on the launching
  * stream.  kind_mask has bit k set for class k: 1 = tensor-core linear layers (sub =
  * epilogue: 0 store, 1 residual, 2 SwiGLU; work = flops), 2 = correction pass (sub = kv
- * format; work = algorithmic bytes), 3 = tensor-core attention (work not filled in);
+ * format; work = algorithmic bytes), 3 = tensor-core attention (work not filled in),
+ * 4 = RMSNorm (work = bytes read and written), 5 = offset estimation (work not filled in);
  * 0 = off.  akvs_prof_enable allocates max_records event pairs (host objects only);
  * akvs_prof_read waits for the recorded events and returns per launch the elapsed ms, the
  * work and (class << 8 | sub); akvs_prof_reset forgets the records but keeps the events.

@@ -452,6 +452,7 @@ int32_t launch_offsets(int dtype, const KvLayer& kv, const ReqMaps& maps, const 
   if (hd > 256) return AKVS_ERR_UNSUPPORTED;      // a lane keeps at most 4 rotation pairs
   const dim3 grid(M, n_kv, 2);
   const size_t smem = (size_t)OFF_WARPS * hd * sizeof(float);
+  ProfScope prof(5, kv.fmt, 0.0, st);
   return dispatch_dtype(dtype, [&](auto tag) -> int32_t {
     using T = decltype(tag);
     return dispatch_fmt(kv.fmt, [&](auto f) -> int32_t {

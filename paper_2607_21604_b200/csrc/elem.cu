@@ -121,6 +121,7 @@ int32_t launch_rmsnorm(int out_dtype, const float* h, const float* gain, float e
                        cudaStream_t st) {
   if (n == 0) return AKVS_OK;
   if (d % 4 != 0 || d > RMS_THREADS * 4 * RMS_MAX_V) return AKVS_ERR_UNSUPPORTED;
+  ProfScope prof(4, 0, (double)n * d * (4.0 + (out_dtype == AKVS_F32 ? 4.0 : 2.0)), st);
   return dispatch_dtype(out_dtype, [&](auto tag) -> int32_t {
     using T = decltype(tag);
     AKVS_CUDA(launch_pdl(rmsnorm_kernel<T>, dim3(n), dim3(RMS_THREADS), 0, st, h, gain, eps, d, (T*)x));
