@@ -18,7 +18,10 @@
  *    ordinary host memory owned by the caller; the library allocates no device memory
  *    (scratch comes from the caller's workspace);
  *  - all work is enqueued on the caller's stream (a cudaStream_t passed as void*; NULL is
- *    the default stream); only akvs_select_probes and akvs_check synchronise it;
+ *    the default stream).  These calls synchronise it (each says so below): akvs_select_probes
+ *    and akvs_check; akvs_op_select, akvs_op_select_static and akvs_op_correct_layer; and
+ *    akvs_select_probes / akvs_prefill_corrected (NAIVE and FULL modes) with n_requests > 1,
+ *    which upload per-token tables of a batch from host vectors;
  *  - a process drives ONE device through this library (one process per GPU): kernel
  *    attributes are set once per process on the device current at the first call, the
  *    measurement hooks keep process-wide state, and calls are not re-entrant across host
@@ -197,29 +200,6 @@ void akvs_free(void* ctx);
  * (AKVS_OK, AKVS_ERR_TIMEOUT, AKVS_ERR_NAN_SCORE), then clears it. */
 int32_t akvs_check(void* workspace, void* stream);
 
-/* Cross-check switch for the tests: bit 0 set routes the 16-bit linear layers, bit 1 set the
- * 16-bit attention, to the CUDA-core kernels instead of the tcgen05 ones (default 0: tensor
- * cores for both).  Bits 2-3: tiling of the tcgen05 linear layers - 0 picked by shape
- * (default), 1 single CTAs, 2 CTA pairs wherever M > 128.  Process-wide; not part of the
- * serving surface. */
-int32_t akvs_debug_set_linear_algo(int32_t algo);
-
-/* Number of kernels this library has launched in this process so far. */
-int64_t akvs_launch_count(void);
-
-/* Per-launch device timing of kernel classes with CUDA events recorded on the launching
- * stream.  kind_mask has bit k set for class k: 1 = tensor-core linear layers (sub =
- * epilogue: 0 store, 1 residual, 2 SwiGLU; work = flops), 2 = correction pass (sub = kv
- * format; work = algorithmic bytes), 3 = tensor-core attention (work not filled in),
- * 4 = RMSNorm (work = bytes read and written), 5 = offset estimation (work not filled in);
- * 0 = off.  akvs_prof_enable allocates max_records event pairs (host objects only);
- * akvs_prof_read waits for the recorded events and returns per launch the elapsed ms, the
- * work and (class << 8 | sub); akvs_prof_reset forgets the records but keeps the events.
- * Not thread-safe. */
-int32_t akvs_prof_enable(int32_t kind_mask, int32_t max_records);
-int32_t akvs_prof_reset(void);
-int32_t akvs_prof_read(int32_t capacity, float* ms, double* work, int32_t* sub, int32_t* n_out);
-
 /* ------------------------------------------------------------------------------------
  * Single steps of the path, exported so that each kernel can be checked on its own.
  * dtype names the element type of every `void*` tensor.  Asynchronous on `stream` unless stated.
@@ -319,6 +299,52 @@ int32_t akvs_op_residual_stats(int32_t dtype, int32_t kv_format, const void* cac
  * bits = 8 is the FP8 (E4M3) cast: one byte per value, meta unused (may be NULL). */
 int32_t akvs_op_quantize(int32_t dtype, const void* x, int32_t n, int32_t n_kv_heads, int32_t head_dim,
                          int32_t bits, void* codes, void* meta, void* stream);
+
+/* ====================================================================================
+ * NOT PART OF THE SERVING SURFACE.  Test and measurement hooks: process-wide state, not
+ * thread-safe, no paper passage behind any of them.  A serving caller needs none of these.
+ * ==================================================================================== */
+
+/* Cross-check switch for the tests: bit 0 set routes the 16-bit linear layers, bit 1 set the
+ * 16-bit attention, to the CUDA-core kernels instead of the tcgen05 ones (default 0: tensor
+ * cores for both).  Bits 2-3: tiling of the tcgen05 linear layers - 0 picked by shape
+ * (default), 1 single CTAs, 2 CTA pairs wherever M > 128.  Process-wide; not part of the
+ * serving surface. */
+int32_t akvs_debug_set_linear_algo(int32_t algo);
+
+/* Number of kernels this library has launched in this process so far. */
+int64_t akvs_launch_count(void);
+
+/* Per-launch device timing of kernel classes with CUDA events recorded on the launching
+ * stream.  kind_mask has bit k set for class k: 1 = tensor-core linear layers (sub =
+ * epilogue: 0 store, 1 residual, 2 SwiGLU; work = flops), 2 = correction pass (sub = kv
+ * format; work = algorithmic bytes), 3 = tensor-core attention (work not filled in),
+ * 4 = RMSNorm (work = bytes read and written), 5 = offset estimation (work not filled in);
+ * 0 = off.  akvs_prof_enable allocates max_records event pairs (host objects only);
+ * akvs_prof_read waits for the recorded events and returns per launch the elapsed ms, the
+ * work and (class << 8 | sub); akvs_prof_reset forgets the records but keeps the events.
+ * Not thread-safe. */
+int32_t akvs_prof_enable(int32_t kind_mask, int32_t max_records);
+int32_t akvs_prof_reset(void);
+int32_t akvs_prof_read(int32_t capacity, float* ms, double* work, int32_t* sub, int32_t* n_out);
+
+/* Launches ONLY the correction kernel of every layer from the check layer on, one after the
+ * other, with exactly the arguments akvs_prefill_corrected(AKVS_MODE_CORRECTED) gives it: the
+ * layer's cache slice in, the layer's out_k / out_v slice out, the request maps, offsets and
+ * fresh rows that the preceding prefill left in `workspace`.  For timing the kernel back to
+ * back over distinct buffers; the K/V it writes are those of the LAST layer's offsets and rows
+ * and are not meant to be used.  Arguments as for the prefill it follows.  Asynchronous. */
+int32_t akvs_debug_correct_repeat(const akvs_model_desc* model, const akvs_cache* cache, const akvs_request* req,
+                                  const akvs_probes* probes, void* out_k, void* out_v, void* ctx,
+                                  void* workspace, int64_t ws_bytes, void* stream);
+
+/* Makes one bounded device-side wait run out, to exercise AKVS_ERR_TIMEOUT without a hang, a
+ * trap or a fault: one CTA of one warp waits, with the same bounded wait the tensor-core kernels
+ * use on their barriers, on a shared-memory barrier that nothing ever arrives at; after
+ * `limit_cycles` SM clock cycles (clamped to [1000, 2e8], i.e. at most about 0.1 s) the wait gives
+ * up, the kernel writes AKVS_ERR_TIMEOUT to the status word at the start of `workspace` (the word
+ * akvs_check returns and clears) and exits normally.  The context stays usable.  Asynchronous. */
+int32_t akvs_debug_wait_timeout(void* workspace, int64_t limit_cycles, void* stream);
 
 #ifdef __cplusplus
 }

@@ -30,6 +30,12 @@ ratio in integer basis points.
   the paper naming only the formats.
 * Section 3.4 and the appendix on mean-explained residual energy: `residual_stats`.
 
+Run-time plumbing that changes no arithmetic: `ATTENTION_WORKERS` > 1 computes the query
+heads of one attention call in that many threads (each head is the same sequence of numpy
+calls on the same data); `Model.w` converts a layer's weights to the working precision once
+and keeps the last layer converted, and `encode_units` walks layer by layer over all units so
+that this happens once per layer.
+
 Arithmetic: float64 by default (`dtype=np.float32` gives the single-precision variant).
 The quantisers are the exception: their decisions are taken on float32 values (float16
 scale and minimum for the groups), because those decide integer codes.
@@ -46,7 +52,11 @@ No function here is "parity unpinned".
 from __future__ import annotations
 
 import math
+from concurrent.futures import ThreadPoolExecutor
+
 import numpy as np
+
+ATTENTION_WORKERS = 1        # threads over query heads inside attention(); 1 = plain loop
 
 # --------------------------------------------------------------------------- transformer parts
 
@@ -101,7 +111,8 @@ def attention(q, k, v, q_pos, k_pos, k_first=None, dtype=np.float64, row_block=1
     for r0 in range(0, R, row_block):
         r1 = min(R, r0 + row_block)
         visible = (k_pos[None, :] <= q_pos[r0:r1, None]) & (k_pos[None, :] >= lo[r0:r1, None])
-        for hq in range(nq):
+
+        def one_head(hq):
             hk = hq // g
             s = (q[r0:r1, hq, :] @ k[:, hk, :].T) * scale
             s = np.where(visible, s, -np.inf)
@@ -109,6 +120,13 @@ def attention(q, k, v, q_pos, k_pos, k_first=None, dtype=np.float64, row_block=1
             p = np.exp(s)
             p = p / np.sum(p, axis=1, keepdims=True)
             out[r0:r1, hq, :] = p @ v[:, hk, :]
+
+        if ATTENTION_WORKERS > 1 and nq > 1:
+            with ThreadPoolExecutor(ATTENTION_WORKERS) as ex:
+                list(ex.map(one_head, range(nq)))
+        else:
+            for hq in range(nq):
+                one_head(hq)
     return out
 
 
@@ -126,6 +144,16 @@ class Model:
         self.tok_emb = tok_emb
         self.layers = layers
         self.final_norm = np.ones(cfg.d_model, np.float32) if final_norm is None else final_norm
+        self._conv = (None, None, {})
+
+    def w(self, l, name, dtype=np.float64):
+        """Layer l's array `name` in the working precision; the last layer asked for stays converted."""
+        if self._conv[0] != l or self._conv[1] != dtype:
+            self._conv = (l, dtype, {})
+        c = self._conv[2]
+        if name not in c:
+            c[name] = np.asarray(self.layers[l][name], dtype)
+        return c[name]
 
 
 def embed(model, ids, dtype=np.float64):
@@ -135,12 +163,11 @@ def embed(model, ids, dtype=np.float64):
 def layer_qkv(model, l, h, positions, dtype=np.float64):
     """Pre-norm, q/k/v projections, RoPE on q and k at `positions`."""
     c = model.cfg
-    w = model.layers[l]
-    x = rmsnorm(h, w["attn_norm"], c.rms_eps, dtype)
+    x = rmsnorm(h, model.w(l, "attn_norm", dtype), c.rms_eps, dtype)
     n = x.shape[0]
-    q = (x @ np.asarray(w["wq"], dtype).T).reshape(n, c.n_q_heads, c.head_dim)
-    k = (x @ np.asarray(w["wk"], dtype).T).reshape(n, c.n_kv_heads, c.head_dim)
-    v = (x @ np.asarray(w["wv"], dtype).T).reshape(n, c.n_kv_heads, c.head_dim)
+    q = (x @ model.w(l, "wq", dtype).T).reshape(n, c.n_q_heads, c.head_dim)
+    k = (x @ model.w(l, "wk", dtype).T).reshape(n, c.n_kv_heads, c.head_dim)
+    v = (x @ model.w(l, "wv", dtype).T).reshape(n, c.n_kv_heads, c.head_dim)
     q = rope_rotate(q, positions, c.rope_base, dtype)
     k = rope_rotate(k, positions, c.rope_base, dtype)
     return q, k, v
@@ -149,12 +176,11 @@ def layer_qkv(model, l, h, positions, dtype=np.float64):
 def layer_out(model, l, h, attn, dtype=np.float64):
     """h + attn W_o, then the SwiGLU MLP with its own pre-norm and residual."""
     c = model.cfg
-    w = model.layers[l]
     n = h.shape[0]
-    h = h + attn.reshape(n, c.n_q_heads * c.head_dim) @ np.asarray(w["wo"], dtype).T
-    x = rmsnorm(h, w["mlp_norm"], c.rms_eps, dtype)
-    a = silu(x @ np.asarray(w["w_gate"], dtype).T) * (x @ np.asarray(w["w_up"], dtype).T)
-    return h + a @ np.asarray(w["w_down"], dtype).T
+    h = h + attn.reshape(n, c.n_q_heads * c.head_dim) @ model.w(l, "wo", dtype).T
+    x = rmsnorm(h, model.w(l, "mlp_norm", dtype), c.rms_eps, dtype)
+    a = silu(x @ model.w(l, "w_gate", dtype).T) * (x @ model.w(l, "w_up", dtype).T)
+    return h + a @ model.w(l, "w_down", dtype).T
 
 
 def dense_layer(model, l, h, positions, k_first=None, dtype=np.float64):
@@ -293,16 +319,18 @@ def encode_units(model, unit_ids_list, kv_bits=0, dtype=np.float64):
     values are the decoded bytes, kept beside them as codes."""
     c = model.cfg
     out = []
-    for ids in unit_ids_list:
-        n = len(ids)
-        pos = np.arange(n)
-        h = embed(model, ids, dtype)
-        Ks, Vs = [], []
-        for l in range(c.n_layers):
-            h, k, v = dense_layer(model, l, h, pos, None, dtype)
-            Ks.append(k)
-            Vs.append(v)
-        unit = {"K": np.stack(Ks), "V": np.stack(Vs), "hidden": h}
+    # every unit is its own sequence; the walk is layer by layer over all of them (the units do
+    # not interact, so the order of the two loops changes nothing)
+    hs = [embed(model, ids, dtype) for ids in unit_ids_list]
+    Ks = [[] for _ in unit_ids_list]
+    Vs = [[] for _ in unit_ids_list]
+    for l in range(c.n_layers):
+        for i, ids in enumerate(unit_ids_list):
+            hs[i], k, v = dense_layer(model, l, hs[i], np.arange(len(ids)), None, dtype)
+            Ks[i].append(k)
+            Vs[i].append(v)
+    for i in range(len(unit_ids_list)):
+        unit = {"K": np.stack(Ks[i]), "V": np.stack(Vs[i]), "hidden": hs[i]}
         if kv_bits == 8:
             for name in ("K", "V"):
                 unit[name + "_codes"] = e4m3_encode(unit[name])

@@ -26,7 +26,7 @@ EXPORTS = ["akvs_workspace_bytes", "akvs_debug_set_linear_algo", "akvs_launch_co
            "akvs_prof_reset", "akvs_prof_read", "akvs_encode_units", "akvs_select_probes", "akvs_prefill_corrected",
            "akvs_free", "akvs_check", "akvs_op_linear", "akvs_op_rope", "akvs_op_attention",
            "akvs_op_scratch_bytes", "akvs_op_select", "akvs_op_select_static", "akvs_op_correct_layer",
-           "akvs_op_quantize", "akvs_op_residual_stats"]
+           "akvs_op_quantize", "akvs_op_residual_stats", "akvs_debug_correct_repeat", "akvs_debug_wait_timeout"]
 STATIC_MAX_CTX, STATIC_MAX_UNITS = 16384, 1024
 
 
@@ -321,6 +321,18 @@ def prof_read(capacity=1 << 16):
     n = C.c_int32(0)
     _chk(lib.akvs_prof_read(capacity, ms, work, sub, C.byref(n)), "akvs_prof_read")
     return [(ms[i], work[i], sub[i]) for i in range(n.value)]
+
+
+def debug_correct_repeat(model, store, req, probes, out_k, out_v, ctx, workspace):
+    """Measurement hook: the correction kernel of every selective layer, back to back."""
+    _chk(lib.akvs_debug_correct_repeat(C.byref(model.desc), C.byref(store.desc), C.byref(req.desc),
+                                       C.byref(probes.desc), _ptr(out_k), _ptr(out_v), ctx, _ptr(workspace),
+                                       C.c_int64(workspace.numel()), _stream()), "akvs_debug_correct_repeat")
+
+
+def debug_wait_timeout(workspace, limit_cycles):
+    """Test hook: a bounded device wait that runs out and reports AKVS_ERR_TIMEOUT through `check`."""
+    _chk(lib.akvs_debug_wait_timeout(_ptr(workspace), C.c_int64(limit_cycles), _stream()), "akvs_debug_wait_timeout")
 
 
 def alloc_outputs(model, n_ctx, n_query, device="cuda"):

@@ -7,9 +7,9 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(os.path.dirname(HERE), "include")
 LIB = os.path.join(HERE, "libakvs.so")
-SOURCES = ["api.cu", "elem.cu", "correct.cu", "simt.cu", "gemm_tc.cu", "attn_tc.cu", "no_alloc.cu"]
+SOURCES = ["api.cu", "elem.cu", "correct.cu", "simt.cu", "gemm_tc.cu", "attn_tc.cu", "no_alloc.cu", "debug.cu"]
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-lineinfo",
-         "-Xcompiler", "-fPIC", "-I" + INCLUDE]
+         "-Xcompiler", "-fPIC", "-I" + INCLUDE] + os.environ.get("AKVS_NVCC_EXTRA", "").split()
 
 
 def _stale():

@@ -83,7 +83,7 @@ struct Workspace {
   int32_t* tok_unit;        // [N]
   int32_t* tok_src;         // [N]
   int32_t* row_of_pos;      // [T]
-  int4* tok_meta;           // [T]
+  int4* tok_meta;           // [2][T] K and V records of the correction pass
   uint8_t* flags;           // [2N]: kflag, vflag
   uint64_t* keys;           // [2N]
   int32_t* pos;             // [T] 0..T-1 (or unit-local positions while encoding)
@@ -107,6 +107,7 @@ struct Workspace {
   void* stash_k;            // [check_layer-1][T][dkv]
   void* stash_v;
   int64_t bytes;
+  int rope_n;               // positions the RoPE table was built for (host-side note for the bounds guards)
 };
 
 Workspace carve(const Dims& D, int N, int nq, int M, int check_layer, void* base) {
@@ -120,7 +121,7 @@ Workspace carve(const Dims& D, int N, int nq, int M, int check_layer, void* base
   w.tok_unit = c.take<int32_t>(N);
   w.tok_src = c.take<int32_t>(N);
   w.row_of_pos = c.take<int32_t>(T);
-  w.tok_meta = c.take<int4>(T);
+  w.tok_meta = c.take<int4>(2 * T);
   w.flags = c.take<uint8_t>(2 * (int64_t)N);
   w.keys = c.take<uint64_t>(2 * (int64_t)N);
   w.pos = c.take<int32_t>(T);
@@ -145,6 +146,7 @@ Workspace carve(const Dims& D, int N, int nq, int M, int check_layer, void* base
   w.stash_k = c.take_bytes(nd * T * D.dkv * D.es);
   w.stash_v = c.take_bytes(nd * T * D.dkv * D.es);
   w.bytes = akvs_align_up(c.off, 256);
+  w.rope_n = (int)T;
   return w;
 }
 
@@ -170,13 +172,13 @@ int g_linear_tiling = 0;       // tcgen05 linear layers: 0 = by shape; 1 = singl
 int32_t linear_multi(const Dims& D, const void* x, int M, int K, int n_seg, const void* const* w, const int* n,
                      void* const* out, const int* ldc, int32_t* status, cudaStream_t st,
                      const float2* rope = nullptr, const int32_t* pos = nullptr, int rope_mask = 0,
-                     float rope_base = 0.f) {
+                     float rope_base = 0.f, int n_pos = 0) {
   bool tc_ok = D.dtype != AKVS_F32 && g_bf16_linear_algo == 0 && K % 8 == 0;
   for (int i = 0; i < n_seg; ++i) tc_ok = tc_ok && n[i] % 128 == 0;
   const bool fuse = tc_ok && D.hd == 128;
   if (tc_ok) {
     AKVS_TRY(launch_linear_tc(D.dtype, 0, x, M, K, n_seg, w, n, out, ldc, status, st, fuse ? rope : nullptr, pos,
-                              rope_mask, g_linear_tiling));
+                              rope_mask, g_linear_tiling, n_pos));
   } else {
     for (int i = 0; i < n_seg; ++i)
       AKVS_TRY(launch_linear_simt(D.dtype, x, w[i], nullptr, out[i], nullptr, M, n[i], K, ldc[i], st));
@@ -184,7 +186,7 @@ int32_t linear_multi(const Dims& D, const void* x, int M, int K, int n_seg, cons
   if (!fuse)
     for (int i = 0; i < n_seg; ++i)
       if ((rope_mask >> i) & 1)
-        AKVS_TRY(launch_rope(D.dtype, out[i], pos, M, n[i] / D.hd, D.hd, ldc[i], rope, rope_base, st));
+        AKVS_TRY(launch_rope(D.dtype, out[i], pos, M, n[i] / D.hd, D.hd, ldc[i], rope, n_pos, status, rope_base, st));
   return AKVS_OK;
 }
 int32_t linear_resid(const Dims& D, const void* x, int M, int K, const void* w, int n, float* h, int32_t* status,
@@ -239,7 +241,8 @@ int32_t run_layer(const akvs_model_desc* m, const Dims& D, int l, const Workspac
     const void* w[3] = {m->wq[l], m->wk[l], m->wv[l]};
     const int ns[3] = {D.dq, D.dkv, D.dkv};
     void* out[3] = {ws.q, k_dst, v_dst};
-    AKVS_TRY(linear_multi(D, ws.x, n, D.d, 3, w, ns, out, ns, ws.status, st, ws.rope, g.pos, 0b011, m->rope_base));
+    AKVS_TRY(linear_multi(D, ws.x, n, D.d, 3, w, ns, out, ns, ws.status, st, ws.rope, g.pos, 0b011, m->rope_base,
+                          ws.rope_n));
   }
   if (between) AKVS_TRY(between());
   AKVS_TRY(attention(D, ws.q, attn_k, attn_v, ws.ao, g, n, n_keys, ws.status, st));
@@ -350,11 +353,16 @@ __global__ void local_pos_kernel(const int32_t* __restrict__ ctx_off, const int3
 }
 
 // Uploads the request's offsets and builds the maps every mode needs.
-__global__ void gather_i32_kernel(const int32_t* __restrict__ src, const int32_t* __restrict__ idx, int n, int stride_src,
-                                  int stride_dst, int n_arrays, int32_t* __restrict__ dst) {
+__global__ void gather_i32_kernel(const int32_t* __restrict__ src, const int32_t* __restrict__ idx, int n, int n_src,
+                                  int stride_src, int stride_dst, int n_arrays, int32_t* status,
+                                  int32_t* __restrict__ dst) {
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= n) return;
-  const int j = idx[i];
+  int j = idx[i];
+  if (j < 0 || j >= n_src) {                    // idx may be caller data (akvs_probes.rows)
+    set_status(status, AKVS_ERR_INVALID_ARG);
+    j = 0;
+  }
   for (int a = 0; a < n_arrays; ++a) dst[(size_t)a * stride_dst + i] = src[(size_t)a * stride_src + j];
 }
 
@@ -400,9 +408,9 @@ RowGeom token_geom(const Workspace& ws, const Batch& b, int T) {
 int32_t row_geom(const Workspace& ws, const Batch& b, const int32_t* rows, int R, int T, RowGeom& g, cudaStream_t st) {
   if (b.B == 1) { g = RowGeom{rows, ws.zeros, rows, nullptr, nullptr}; return AKVS_OK; }
   if (R > 0) {
-    gather_i32_kernel<<<akvs_cdiv(R, 256), 256, 0, st>>>(ws.tok_pos, rows, R, 0, 0, 1, ws.row_meta);
+    gather_i32_kernel<<<akvs_cdiv(R, 256), 256, 0, st>>>(ws.tok_pos, rows, R, T, 0, 0, 1, ws.status, ws.row_meta);
     AKVS_LAUNCHED();
-    gather_i32_kernel<<<akvs_cdiv(R, 256), 256, 0, st>>>(ws.tok_rng, rows, R, T, T, 4, ws.row_meta + T);
+    gather_i32_kernel<<<akvs_cdiv(R, 256), 256, 0, st>>>(ws.tok_rng, rows, R, T, T, T, 4, ws.status, ws.row_meta + T);
     AKVS_LAUNCHED();
   }
   g = RowGeom{ws.row_meta, ws.row_meta + T, ws.row_meta + 2 * (size_t)T, ws.row_meta + 3 * (size_t)T,
@@ -438,8 +446,9 @@ ReqMaps req_maps(const Workspace& ws, int N, bool batched = false) {
 // Embeds context (through the store's token ids) and query rows into ws.h.
 int32_t embed_all(const akvs_model_desc* m, const Dims& D, const akvs_cache* c, const akvs_request* r,
                   const Workspace& ws, int N, cudaStream_t st) {
-  AKVS_TRY(launch_embed(D.dtype, m->tok_emb, c->token_ids, ws.tok_src, N, D.d, ws.h, st));
-  AKVS_TRY(launch_embed(D.dtype, m->tok_emb, r->query_ids, nullptr, r->n_query, D.d, ws.h + (size_t)N * D.d, st));
+  AKVS_TRY(launch_embed(D.dtype, m->tok_emb, c->token_ids, ws.tok_src, N, D.d, D.vocab, ws.status, ws.h, st));
+  AKVS_TRY(launch_embed(D.dtype, m->tok_emb, r->query_ids, nullptr, r->n_query, D.d, D.vocab, ws.status,
+                        ws.h + (size_t)N * D.d, st));
   return AKVS_OK;
 }
 
@@ -515,10 +524,11 @@ int32_t akvs_encode_units(const akvs_model_desc* model, akvs_cache* cache, void*
   int max_len = 0;
   for (int u = 0; u < M; ++u) max_len = off[u + 1] - off[u] > max_len ? off[u + 1] - off[u] : max_len;
   AKVS_TRY(launch_rope_table(model->rope_base, D.hd, max_len, ws.rope, st));
+  ws.rope_n = max_len;
   local_pos_kernel<<<akvs_cdiv(N, 256), 256, 0, st>>>(ws.ctx_off, ws.tok_unit, N, ws.row_of_pos, ws.lo);
   AKVS_LAUNCHED();
   const int32_t* local_pos = ws.row_of_pos;     // unit-local positions; ws.pos stays 0..N-1 = row index
-  AKVS_TRY(launch_embed(D.dtype, model->tok_emb, cache->token_ids, nullptr, N, D.d, ws.h, st));
+  AKVS_TRY(launch_embed(D.dtype, model->tok_emb, cache->token_ids, nullptr, N, D.d, D.vocab, ws.status, ws.h, st));
   const bool native = cache->kv_format == AKVS_KV_NATIVE;
   const size_t lstride = (size_t)N * kv_row_bytes(D, cache->kv_format);
   const size_t mstride = (size_t)N * D.nkv * (D.hd / 64) * 4;
@@ -599,7 +609,7 @@ int32_t akvs_select_probes(const akvs_model_desc* model, const akvs_cache* cache
     const int ns[2] = {D.dkv, D.dkv};
     void* o[2] = {ws.k, ws.v};
     AKVS_TRY(linear_multi(D, ws.x, N, D.d, 2, w, ns, o, ns, ws.status, st, ws.rope, all_tokens.pos, 0b01,
-                          model->rope_base));
+                          model->rope_base, ws.rope_n));
     AKVS_TRY(wait_layer(cache, lc, st));
     AKVS_TRY(launch_scores(D.dtype, cache_layer(cache, D, lc), req_maps(ws, N, batch.B > 1), ws.k, ws.v, N, D.nkv, D.hd, ws.rope,
                            out->d_k, out->d_v, st));
@@ -659,7 +669,7 @@ int32_t akvs_prefill_corrected(const akvs_model_desc* model, const akvs_cache* c
     return launch_rmsnorm(AKVS_F32, ws.h + (size_t)N * D.d, model->final_norm, model->rms_eps, nq, D.d, out_hidden, st);
   }
 
-  int first_layer = 0, P = 0, R = nq;
+  int first_layer = 0, P = 0, R = nq, n_probe_total = 0;
   const int32_t* rows = nullptr;
   Workspace ws;
   if (mode == AKVS_MODE_NAIVE) {
@@ -670,8 +680,9 @@ int32_t akvs_prefill_corrected(const akvs_model_desc* model, const akvs_cache* c
     AKVS_TRY(launch_rope_table(model->rope_base, D.hd, T, ws.rope, st));
     rows = ws.pos + N;                                   // the query positions N..T-1
     AKVS_TRY(launch_row_maps(rows, nq, nullptr, nullptr, 0, N, T, ws.row_of_pos, ws.flags, ws.flags + N, st));
-    AKVS_TRY(launch_tok_meta(ws.tok_unit, ws.tok_src, ws.row_of_pos, ws.flags, ws.flags + N, N, T, 0, ws.tok_meta, st));
-    AKVS_TRY(launch_embed(D.dtype, model->tok_emb, req->query_ids, nullptr, nq, D.d, ws.h, st));
+    AKVS_TRY(launch_tok_meta(ws.tok_unit, ws.tok_src, ws.row_of_pos, ws.flags, ws.flags + N, nullptr, nullptr, N, T, 0,
+                             ws.tok_meta, st));
+    AKVS_TRY(launch_embed(D.dtype, model->tok_emb, req->query_ids, nullptr, nq, D.d, D.vocab, ws.status, ws.h, st));
   } else {
     const Ctx* ctx = reinterpret_cast<const Ctx*>(ctx_v);
     if (!ctx || ctx->magic != kCtxMagic || !probes) return AKVS_ERR_INVALID_ARG;
@@ -685,19 +696,21 @@ int32_t akvs_prefill_corrected(const akvs_model_desc* model, const akvs_cache* c
     ws = carve(D, N, nq, M, ctx->check_layer, workspace);
     AKVS_TRY(check_workspace(workspace, ws_bytes, ws.bytes));
     first_layer = ctx->check_layer - 1;
+    n_probe_total = ctx->n_probe_total;
     P = probes->n_probe_rows;
     R = probes->n_rows;
     rows = probes->rows;
     AKVS_TRY(launch_row_maps(rows, R, probes->sk_idx, probes->sv_idx, ctx->n_probe_total, N, T, ws.row_of_pos,
                              ws.flags, ws.flags + N, st));
-    AKVS_TRY(launch_tok_meta(ws.tok_unit, ws.tok_src, ws.row_of_pos, ws.flags, ws.flags + N, N, T, P, ws.tok_meta, st));
+    AKVS_TRY(launch_tok_meta(ws.tok_unit, ws.tok_src, ws.row_of_pos, ws.flags, ws.flags + N, probes->w_k, probes->w_v, N,
+                             T, P, ws.tok_meta, st));
     for (int l = 0; l < first_layer; ++l) {
       AKVS_CUDA(cudaMemcpyAsync(ok + l * kv_l, reinterpret_cast<char*>(ws.stash_k) + l * kv_l, kv_l,
                                 cudaMemcpyDeviceToDevice, st));
       AKVS_CUDA(cudaMemcpyAsync(ov + l * kv_l, reinterpret_cast<char*>(ws.stash_v) + l * kv_l, kv_l,
                                 cudaMemcpyDeviceToDevice, st));
     }
-    AKVS_TRY(launch_gather_rows(ws.stash_h, rows, R, D.d, ws.h, st));
+    AKVS_TRY(launch_gather_rows(ws.stash_h, rows, R, D.d, T, ws.status, ws.h, st));
   }
 
   const ReqMaps maps = req_maps(ws, N, batch.B > 1);
@@ -710,14 +723,41 @@ int32_t akvs_prefill_corrected(const akvs_model_desc* model, const akvs_cache* c
       AKVS_TRY(wait_layer(cache, l, st));
       if (corrected)
         AKVS_TRY(launch_offsets(D.dtype, kv, maps, probes->probe_off, probes->sk_idx, probes->sv_idx, ws.k, ws.v, M,
-                                D.nkv, D.hd, ws.rope, ws.mu_k, ws.mu_v, st));
-      return launch_correct(D.dtype, kv, maps, ws.k, ws.v, corrected ? probes->w_k : nullptr,
-                            corrected ? probes->w_v : nullptr, ws.mu_k, ws.mu_v, N, nq, P, D.nkv, D.hd, ws.rope,
+                                N, n_probe_total, D.nkv, D.hd, ws.rope, ws.mu_k, ws.mu_v, ws.status, st));
+      return launch_correct(D.dtype, kv, maps, ws.k, ws.v, corrected, ws.mu_k, ws.mu_v, N, nq, D.nkv, D.hd, ws.rope,
                             ok + l * kv_l, ov + l * kv_l, st);
     };
     AKVS_TRY(run_layer(model, D, l, ws, R, geom, ws.k, ws.v, ok + l * kv_l, ov + l * kv_l, T, assemble, st));
   }
   return launch_rmsnorm(AKVS_F32, ws.h + (size_t)P * D.d, model->final_norm, model->rms_eps, nq, D.d, out_hidden, st);
+}
+
+int32_t akvs_debug_correct_repeat(const akvs_model_desc* model, const akvs_cache* cache, const akvs_request* req,
+                                  const akvs_probes* probes, void* out_k, void* out_v, void* ctx_v, void* workspace,
+                                  int64_t ws_bytes, void* stream) {
+  Dims D;
+  AKVS_TRY(check_model(model, D));
+  AKVS_TRY(check_cache(cache, D, true));
+  if (!out_k || !out_v || !probes) return AKVS_ERR_INVALID_ARG;
+  std::vector<int32_t> ctx_off, slot_src;
+  AKVS_TRY(check_request(req, cache, ctx_off, slot_src));
+  Batch batch;
+  AKVS_TRY(check_batch(req, ctx_off, batch));
+  const Ctx* ctx = reinterpret_cast<const Ctx*>(ctx_v);
+  const int M = req->n_units, N = ctx_off[M], nq = req->n_query, T = N + nq;
+  if (!ctx || ctx->magic != kCtxMagic) return AKVS_ERR_INVALID_ARG;
+  if (ctx->N != N || ctx->nq != nq || ctx->M != M || ctx->B != batch.B || ctx->workspace != workspace)
+    return AKVS_ERR_SHAPE;
+  Workspace ws = carve(D, N, nq, M, ctx->check_layer, workspace);
+  AKVS_TRY(check_workspace(workspace, ws_bytes, ws.bytes));
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  const size_t kv_l = (size_t)T * D.dkv * D.es;
+  const ReqMaps maps = req_maps(ws, N, batch.B > 1);
+  for (int l = ctx->check_layer - 1; l < D.L; ++l)
+    AKVS_TRY(launch_correct(D.dtype, cache_layer(cache, D, l), maps, ws.k, ws.v, true, ws.mu_k, ws.mu_v, N, nq, D.nkv,
+                            D.hd, ws.rope, reinterpret_cast<char*>(out_k) + l * kv_l,
+                            reinterpret_cast<char*>(out_v) + l * kv_l, st));
+  return AKVS_OK;
 }
 
 void akvs_free(void* ctx) {
@@ -759,7 +799,7 @@ int32_t akvs_op_rope(int32_t dtype, void* x, const int32_t* pos, int32_t n, int3
                      float rope_base, void* stream) {
   if (!x || !pos || n < 0 || n_heads <= 0 || head_dim <= 0) return AKVS_ERR_INVALID_ARG;
   if (dtype != AKVS_F32 && dtype != AKVS_BF16 && dtype != AKVS_F16) return AKVS_ERR_UNSUPPORTED;
-  return launch_rope(dtype, x, pos, n, n_heads, head_dim, n_heads * head_dim, nullptr, rope_base,
+  return launch_rope(dtype, x, pos, n, n_heads, head_dim, n_heads * head_dim, nullptr, 0, nullptr, rope_base,
                      reinterpret_cast<cudaStream_t>(stream));
 }
 
@@ -776,7 +816,7 @@ int32_t akvs_op_attention(int32_t dtype, const void* q, const void* k, const voi
 
 int64_t akvs_op_scratch_bytes(int32_t n_ctx, int32_t n_query, int32_t n_units, int32_t head_dim) {
   const int64_t T = (int64_t)n_ctx + n_query;
-  return 4096 + 256 * 12 + T * (4 + 16 + head_dim * 4) + (int64_t)n_ctx * (4 + 2 + 16) + (int64_t)(n_units + 1) * 8;
+  return 4096 + 256 * 12 + T * (4 + 32 + head_dim * 4) + (int64_t)n_ctx * (4 + 2 + 16) + (int64_t)(n_units + 1) * 8;
 }
 
 int32_t akvs_op_select(const float* d_k, const float* d_v, const int32_t* ctx_off_host, int32_t n_units,
@@ -787,11 +827,14 @@ int32_t akvs_op_select(const float* d_k, const float* d_v, const int32_t* ctx_of
   if (!out->ctx_off || !out->probe_off || !out->sk_idx || !out->sv_idx || !out->w_k || !out->w_v || !out->rows)
     return AKVS_ERR_INVALID_ARG;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
-  const int M = n_units, N = ctx_off_host[M];
+  const int M = n_units;
+  if (ctx_off_host[0] != 0) return AKVS_ERR_SHAPE;
+  for (int u = 0; u < M; ++u)
+    if (ctx_off_host[u + 1] < ctx_off_host[u]) return AKVS_ERR_SHAPE;      // before N is used for anything
+  const int N = ctx_off_host[M];
   std::vector<int32_t> probe_off(M + 1, 0);
   for (int u = 0; u < M; ++u) {
     const int64_t n = ctx_off_host[u + 1] - ctx_off_host[u];
-    if (n < 0) return AKVS_ERR_SHAPE;
     int64_t b = (n * refresh_bp + 9999) / 10000;
     b = b > n ? n : b;
     probe_off[u + 1] = probe_off[u] + (int32_t)b;
@@ -836,8 +879,7 @@ int32_t akvs_op_correct_layer(int32_t dtype, int32_t kv_format, const void* cach
   int32_t* zero_src = c.take<int32_t>(M + 1);
   int32_t* dummy_src = c.take<int32_t>(N);
   float2* table = c.take<float2>((int64_t)T * (head_dim / 2));
-  int4* tok_meta = c.take<int4>(T);
-  (void)poff_host_dev;
+  int4* tok_meta = c.take<int4>(2 * (int64_t)T);
   // the number of probe indices is probe_off[M]; read it back (this helper may synchronise)
   int32_t n_probe = 0;
   AKVS_CUDA(cudaMemcpyAsync(&n_probe, probes->probe_off + M, sizeof(int32_t), cudaMemcpyDeviceToHost, st));
@@ -848,13 +890,16 @@ int32_t akvs_op_correct_layer(int32_t dtype, int32_t kv_format, const void* cach
   AKVS_TRY(launch_row_maps(probes->rows, probes->n_rows, probes->sk_idx, probes->sv_idx, n_probe, N, T, row_of_pos,
                            flags, flags + N, st));
   AKVS_TRY(launch_rope_table(rope_base, head_dim, T, table, st));
-  AKVS_TRY(launch_tok_meta(tok_unit, src_tok, row_of_pos, flags, flags + N, N, T, probes->n_probe_rows, tok_meta, st));
+  AKVS_TRY(launch_tok_meta(tok_unit, src_tok, row_of_pos, flags, flags + N, probes->w_k, probes->w_v, N, T,
+                           probes->n_probe_rows, tok_meta, st));
   KvLayer kv{cache_k, cache_v, k_meta, v_meta, kv_format};
   ReqMaps maps{probes->ctx_off, probes->ctx_off, tok_unit, src_tok, row_of_pos, flags, flags + N, tok_meta};
-  AKVS_TRY(launch_offsets(dtype, kv, maps, probes->probe_off, probes->sk_idx, probes->sv_idx, fresh_k, fresh_v, M,
-                          n_kv_heads, head_dim, table, mu_k, mu_v, st));
-  return launch_correct(dtype, kv, maps, fresh_k, fresh_v, probes->w_k, probes->w_v, mu_k, mu_v, N, n_query,
-                        probes->n_probe_rows, n_kv_heads, head_dim, table, out_k, out_v, st);
+  int32_t* status = poff_host_dev;                 // first words of the scratch: the status word of this call
+  AKVS_CUDA(cudaMemsetAsync(status, 0, 16 * sizeof(int32_t), st));
+  AKVS_TRY(launch_offsets(dtype, kv, maps, probes->probe_off, probes->sk_idx, probes->sv_idx, fresh_k, fresh_v, M, N,
+                          n_probe, n_kv_heads, head_dim, table, mu_k, mu_v, status, st));
+  return launch_correct(dtype, kv, maps, fresh_k, fresh_v, true, mu_k, mu_v, N, n_query, n_kv_heads, head_dim, table,
+                        out_k, out_v, st);
 }
 
 int32_t akvs_op_residual_stats(int32_t dtype, int32_t kv_format, const void* cache_k, const void* cache_v,

@@ -466,8 +466,8 @@ int32_t launch_attention_tc(int dtype, const void* q, const void* k, const void*
   p.q = q; p.k_lo = k_lo; p.k_hi = k_hi; p.k_lo2 = k_lo2; p.k_hi2 = k_lo2 ? k_hi2 : nullptr; p.out = out; p.status = status;
   p.scale_log2 = 1.4426950408889634f / sqrtf((float)HD);
   const uint32_t fmt = dtype == AKVS_F16 ? tc::kF16 : tc::kBF16;
-  p.idesc_qk = tc::idesc_f16(fmt, fmt, 128, BN, 0);
-  p.idesc_pv = tc::idesc_f16(fmt, fmt, 128, HD, 1);
+  p.idesc_qk = tc::idesc_f16(fmt, 128, BN, 0);
+  p.idesc_pv = tc::idesc_f16(fmt, 128, HD, 1);
   CUtensorMap tmK, tmV;
   AKVS_TRY(encode_tmap_2d_16bit(&tmK, k, T, (uint64_t)n_kv * HD, (uint64_t)n_kv * HD, BN));
   AKVS_TRY(encode_tmap_2d_16bit(&tmV, v, T, (uint64_t)n_kv * HD, (uint64_t)n_kv * HD, BN));

@@ -215,17 +215,18 @@ struct ReqMaps {            // per-request index maps (device)
   const int32_t* row_of_pos;// [T] index into the recomputed rows, or -1
   const uint8_t* kflag;     // [N] 1 if j in S^K
   const uint8_t* vflag;     // [N]
-  const int4* tok_meta;     // [T] (store row, fresh K row or -1, fresh V row or -1, unit slot)
+  const int4* tok_meta;     // [2][T] K records, then V records: (store row, fresh row or -1, unit slot, weight bits)
 };
 
 int32_t launch_embed(int dtype, const void* tok_emb, const int32_t* ids, const int32_t* gather, int n, int d,
-                     float* h, cudaStream_t st);
-int32_t launch_gather_rows(const float* src, const int32_t* rows, int n, int d, float* dst, cudaStream_t st);
+                     int vocab, int32_t* status, float* h, cudaStream_t st);
+int32_t launch_gather_rows(const float* src, const int32_t* rows, int n, int d, int n_src, int32_t* status, float* dst,
+                           cudaStream_t st);
 int32_t launch_rmsnorm(int out_dtype, const float* h, const float* gain, float eps, int n, int d, void* x,
                        cudaStream_t st);
 int32_t launch_rope_table(float base, int hd, int n_pos, float2* table, cudaStream_t st);
 int32_t launch_rope(int dtype, void* x, const int32_t* pos, int n, int n_heads, int hd, int ld,
-                    const float2* table, float base, cudaStream_t st);
+                    const float2* table, int n_pos, int32_t* status, float base, cudaStream_t st);
 int32_t launch_iota(int32_t* p, int n, int start, cudaStream_t st);
 int32_t launch_quantize(int dtype, const void* x, int n, int n_kv, int hd, int bits, void* codes, void* meta,
                         cudaStream_t st);
@@ -236,11 +237,13 @@ int32_t launch_linear_simt(int dtype, const void* x, const void* w, const void* 
 // 16-bit tensor-core linear layers (gemm_tc.cu), dtype AKVS_BF16 or AKVS_F16.  epi 0: out[i] = x w[i]^T; 1: out[0] (float) += x w[0]^T;
 // 2: out[0] = silu(x w[0]^T) * (x w[1]^T).
 // With epi 0, segments whose bit is set in rope_mask (heads of 128 columns) are rotated through
-// rope[pos[row]] in the epilogue (rope: [positions][64] (cos, sin); null = no rotation).
+// rope[pos[row]] in the epilogue (rope: [n_pos][64] (cos, sin); null = no rotation; a position
+// outside [0, n_pos) raises AKVS_ERR_INVALID_ARG in the status word and rotates by position 0).
 // tiling 0: single CTAs or CTA pairs, whichever the shape favours; 1: single CTAs; 2: pairs (M > 128).
 int32_t launch_linear_tc(int dtype, int epi, const void* x, int M, int K, int n_seg, const void* const* w, const int* n,
                          void* const* out, const int* ldc, int32_t* status, cudaStream_t st,
-                         const float2* rope = nullptr, const int32_t* pos = nullptr, int rope_mask = 0, int tiling = 0);
+                         const float2* rope = nullptr, const int32_t* pos = nullptr, int rope_mask = 0, int tiling = 0,
+                         int n_pos = 0);
 
 // tcgen05 attention (attn_tc.cu): 16-bit types, head_dim 128.
 int32_t launch_attention_tc(int dtype, const void* q, const void* k, const void* v, void* out, const int32_t* k_lo,
@@ -255,8 +258,8 @@ int32_t launch_tok_maps(const int32_t* ctx_off, const int32_t* slot_src_off, int
 int32_t launch_row_maps(const int32_t* rows, int n_rows, const int32_t* sk_idx, const int32_t* sv_idx, int n_probe,
                         int N, int T, int32_t* row_of_pos, uint8_t* kflag, uint8_t* vflag, cudaStream_t st);
 int32_t launch_tok_meta(const int32_t* tok_unit, const int32_t* tok_src, const int32_t* row_of_pos,
-                        const uint8_t* kflag, const uint8_t* vflag, int N, int T, int n_probe_rows, int4* tok_meta,
-                        cudaStream_t st);
+                        const uint8_t* kflag, const uint8_t* vflag, const float* w_k, const float* w_v, int N, int T,
+                        int n_probe_rows, int4* tok_meta /*[2][T]*/, cudaStream_t st);
 int32_t launch_scores(int dtype, const KvLayer& kv, const ReqMaps& maps, const void* k_fresh, const void* v_fresh,
                       int N, int n_kv, int hd, const float2* table, float* d_k, float* d_v, cudaStream_t st);
 int32_t launch_select(const float* d_k, const float* d_v, const int32_t* ctx_off, const int32_t* probe_off, int M,
@@ -265,13 +268,14 @@ int32_t launch_select(const float* d_k, const float* d_v, const int32_t* ctx_off
                       cudaStream_t st);
 int32_t launch_offsets(int dtype, const KvLayer& kv, const ReqMaps& maps, const int32_t* probe_off,
                        const int32_t* sk_idx, const int32_t* sv_idx, const void* k_fresh, const void* v_fresh, int M,
-                       int n_kv, int hd, const float2* table, float* mu_k, float* mu_v, cudaStream_t st);
+                       int N, int n_probe_cap, int n_kv, int hd, const float2* table, float* mu_k, float* mu_v,
+                       int32_t* status, cudaStream_t st);
 int32_t launch_residual_stats(int dtype, const KvLayer& kv, const int32_t* ctx_off, const int32_t* tok_src,
                               const void* k_fresh, const void* v_fresh, int M, int n_kv, int hd, const float2* table,
                               const float* sel_k, const float* sel_v, const float* mu_k, const float* mu_v,
                               const float* w_k, const float* w_v, float* mean_k, float* mean_v, float* energy,
                               cudaStream_t st);
+// weighted = false: no offsets are added (direct reuse); the weights themselves ride in tok_meta
 int32_t launch_correct(int dtype, const KvLayer& kv, const ReqMaps& maps, const void* k_fresh, const void* v_fresh,
-                       const float* w_k, const float* w_v, const float* mu_k, const float* mu_v, int N, int n_query,
-                       int n_probe_rows, int n_kv, int hd, const float2* table, void* out_k, void* out_v,
-                       cudaStream_t st);
+                       bool weighted, const float* mu_k, const float* mu_v, int N, int n_query, int n_kv, int hd,
+                       const float2* table, void* out_k, void* out_v, cudaStream_t st);

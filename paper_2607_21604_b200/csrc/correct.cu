@@ -59,6 +59,24 @@ __device__ __forceinline__ void load_cached_chunk(const void* base, const void* 
   }
 }
 
+// V consecutive floats / float2 as 16-byte loads (the addresses are 16-byte aligned by layout)
+template <int V>
+__device__ __forceinline__ void ld_f(const float* p, float (&o)[V]) {
+#pragma unroll
+  for (int i = 0; i < V; i += 4) {
+    const float4 t = *reinterpret_cast<const float4*>(p + i);
+    o[i] = t.x; o[i + 1] = t.y; o[i + 2] = t.z; o[i + 3] = t.w;
+  }
+}
+template <int V>
+__device__ __forceinline__ void ld_f2(const float2* p, float2 (&o)[V]) {
+#pragma unroll
+  for (int i = 0; i < V; i += 2) {
+    const float4 t = *reinterpret_cast<const float4*>(p + i);
+    o[i] = make_float2(t.x, t.y); o[i + 1] = make_float2(t.z, t.w);
+  }
+}
+
 // ---------------------------------------------------------------------------------------
 // Index maps of a request.
 // ---------------------------------------------------------------------------------------
@@ -102,29 +120,35 @@ __global__ void row_maps_fill_kernel(const int32_t* __restrict__ rows, int n_row
   }
 }
 
-// Per-token record of the correction pass: (store row, fresh row for K or -1, fresh row for V
-// or -1, unit slot).  Query tokens take both from the fresh rows that follow the probes.
+// Per-token records of the correction pass, one array for K and one for V ([2][T]):
+//   (store row, fresh row or -1, unit slot, bits of the weight w)
+// A token in S^K (S^V) takes its fresh K (V) row; query tokens take both from the fresh rows
+// that follow the probes.  The weights are fixed after selection, so they ride in the record
+// and the correction pass makes one 16-byte load per token and role.
 __global__ void tok_meta_kernel(const int32_t* __restrict__ tok_unit, const int32_t* __restrict__ tok_src,
                                 const int32_t* __restrict__ row_of_pos, const uint8_t* __restrict__ kflag,
-                                const uint8_t* __restrict__ vflag, int N, int T, int n_probe_rows,
+                                const uint8_t* __restrict__ vflag, const float* __restrict__ w_k,
+                                const float* __restrict__ w_v, int N, int T, int n_probe_rows,
                                 int4* __restrict__ tok_meta) {
   const int j = blockIdx.x * blockDim.x + threadIdx.x;
   if (j >= T) return;
   if (j >= N) {
     const int r = n_probe_rows + (j - N);
-    tok_meta[j] = make_int4(-1, r, r, 0);
+    tok_meta[j] = make_int4(-1, r, 0, 0);
+    tok_meta[(size_t)T + j] = make_int4(-1, r, 0, 0);
   } else {
     const int r = row_of_pos[j];
-    tok_meta[j] = make_int4(tok_src[j], kflag[j] ? r : -1, vflag[j] ? r : -1, tok_unit[j]);
+    tok_meta[j] = make_int4(tok_src[j], kflag[j] ? r : -1, tok_unit[j], __float_as_int(w_k ? w_k[j] : 0.f));
+    tok_meta[(size_t)T + j] = make_int4(tok_src[j], vflag[j] ? r : -1, tok_unit[j], __float_as_int(w_v ? w_v[j] : 0.f));
   }
 }
 
 int32_t launch_tok_meta(const int32_t* tok_unit, const int32_t* tok_src, const int32_t* row_of_pos,
-                        const uint8_t* kflag, const uint8_t* vflag, int N, int T, int n_probe_rows, int4* tok_meta,
-                        cudaStream_t st) {
+                        const uint8_t* kflag, const uint8_t* vflag, const float* w_k, const float* w_v, int N, int T,
+                        int n_probe_rows, int4* tok_meta, cudaStream_t st) {
   if (T == 0) return AKVS_OK;
-  tok_meta_kernel<<<akvs_cdiv(T, 256), 256, 0, st>>>(tok_unit, tok_src, row_of_pos, kflag, vflag, N, T, n_probe_rows,
-                                                    tok_meta);
+  tok_meta_kernel<<<akvs_cdiv(T, 256), 256, 0, st>>>(tok_unit, tok_src, row_of_pos, kflag, vflag, w_k, w_v, N, T,
+                                                    n_probe_rows, tok_meta);
   AKVS_LAUNCHED();
   return AKVS_OK;
 }
@@ -348,116 +372,104 @@ int32_t launch_select(const float* d_k, const float* d_v, const int32_t* ctx_off
 
 // ---------------------------------------------------------------------------------------
 // Mean estimation (Section 3.3; Algorithm 1 line 5): mu_u = (1/b_u) sum_{j in S_u} (fresh_j -
-// reuse_j).  One CTA per (unit, kv head, K|V); each warp takes every 8th probe, lanes own
-// rotation pairs; warps are combined through shared memory in a fixed order.
+// reuse_j).  One CTA per (unit, kv head, K|V).  A thread owns one pair chunk (16 bytes of the
+// lower half of the head and the RoPE partner 16 bytes in the upper half) of one probe slot:
+// every global access is a 16-byte vector, a head's row is read as two whole 128-byte lines
+// by neighbouring threads, and the 256 / (chunks per head) slots take the unit's probes side
+// by side (all of them at once for b_u up to the slot count), so the dependent index loads
+// (probe -> recomputed row, store row) are paid once.  Slots are summed in a fixed order.
+// The probe arrays may have been written by the caller: an index outside the context or a
+// probe range outside the arrays raises AKVS_ERR_INVALID_ARG and is skipped, never read.
 // ---------------------------------------------------------------------------------------
-constexpr int OFF_WARPS = 8;
+constexpr int OFF_THREADS = 256;
 
 template <typename T, typename TW, int FMT>
-__global__ void __launch_bounds__(OFF_WARPS * 32)
+__global__ void __launch_bounds__(OFF_THREADS)
 offsets_kernel(KvLayer kv, ReqMaps maps, const int32_t* __restrict__ probe_off, const int32_t* __restrict__ sk_idx,
                const int32_t* __restrict__ sv_idx, const T* __restrict__ k_fresh, const T* __restrict__ v_fresh,
-               int n_kv, int hd, const float2* __restrict__ table, float* __restrict__ mu_k, float* __restrict__ mu_v) {
-  extern __shared__ float part[];                 // [OFF_WARPS][hd]
+               int N, int n_probe_cap, int n_kv, int hd, const float2* __restrict__ table, float* __restrict__ mu_k,
+               float* __restrict__ mu_v, int32_t* status) {
+  constexpr int V = VecOf<T>::N;
+  extern __shared__ float part[];                 // [slots][hd]
   pdl_trigger();
   pdl_wait();
   const int u = blockIdx.x, h = blockIdx.y, is_v = blockIdx.z;
-  const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
-  const int half = hd / 2;
-  const int p0 = probe_off[u], b = probe_off[u + 1] - p0;
+  const int half = hd / 2, ch = half / V;
+  const int slots = OFF_THREADS / ch;
+  const int slot = threadIdx.x / ch, c = threadIdx.x - slot * ch;
+  int p0 = probe_off[u], b = probe_off[u + 1] - p0;
+  if (p0 < 0 || b < 0 || (int64_t)p0 + b > n_probe_cap) {
+    if (threadIdx.x == 0) set_status(status, AKVS_ERR_INVALID_ARG);
+    p0 = 0;
+    b = 0;
+  }
   const int32_t* S = (is_v ? sv_idx : sk_idx) + p0;
-  const float2* rot = table + (size_t)maps.unit_pos[u] * half;
   const T* fresh = is_v ? v_fresh : k_fresh;
   const void* cbase = is_v ? kv.v : kv.k;
   const void* cmeta = is_v ? kv.v_meta : kv.k_meta;
-
-  // A lane owns the rotation pairs e = lane, lane + 32, ... and keeps their sums in registers.
-  // The warp's probes (every 8th of the unit) are taken 32 at a time: each lane first fetches
-  // the row and store indices of one probe, so that the dependent index loads are paid once per
-  // batch and not once per probe; the probes are then walked in their original order.
-  constexpr int OFF_Q = 4;                        // pairs per lane: head_dim <= 256
-  float acc_lo[OFF_Q], acc_hi[OFF_Q];
+  float acc_lo[V], acc_hi[V];
 #pragma unroll
-  for (int q = 0; q < OFF_Q; ++q) acc_lo[q] = acc_hi[q] = 0.f;
-  for (int base = wid; base < b; base += OFF_WARPS * 32) {
-    const int i = base + lane * OFF_WARPS;
-    int row_l = -1, src_l = 0;
-    if (i < b) {
+  for (int i = 0; i < V; ++i) acc_lo[i] = acc_hi[i] = 0.f;
+  if (slot < slots) {
+    float2 rot[V];
+    if (!is_v) ld_f2<V>(table + (size_t)maps.unit_pos[u] * half + c * V, rot);
+    for (int i = slot; i < b; i += slots) {
       const int j = S[i];
-      row_l = maps.row_of_pos[j];
-      src_l = maps.tok_src[j];
-    }
-    const int left = (b - base + OFF_WARPS - 1) / OFF_WARPS;
-    const int cnt = left < 32 ? left : 32;
-    for (int k = 0; k < cnt; ++k) {
-      const int row = __shfl_sync(0xFFFFFFFFu, row_l, k);
-      const int64_t src = __shfl_sync(0xFFFFFFFFu, src_l, k);
-      if (row < 0) continue;                       // inconsistent caller-supplied sets: skip
-      const T* fp = fresh + ((size_t)row * n_kv + h) * hd;
+      if (j < 0 || j >= N) { set_status(status, AKVS_ERR_INVALID_ARG); continue; }
+      const int row = maps.row_of_pos[j];
+      const int64_t src = maps.tok_src[j];
+      if (row < 0) continue;                        // inconsistent caller-supplied sets: skip
+      float lo[V], hi[V], flo[V], fhi[V];
+      load_cached_chunk<TW, FMT>(cbase, cmeta, src, n_kv, hd, h, c * V, lo);
+      load_cached_chunk<TW, FMT>(cbase, cmeta, src, n_kv, hd, h, half + c * V, hi);
+      const T* fp = fresh + ((size_t)row * n_kv + h) * hd + c * V;
+      ld16(fp, flo);
+      ld16(fp + half, fhi);
 #pragma unroll
-      for (int q = 0; q < OFF_Q; ++q) {
-        const int e = lane + 32 * q;
-        if (e >= half) break;
-        float lo, hi;
-        if constexpr (FMT == AKVS_KV_NATIVE) {
-          const TW* cp = reinterpret_cast<const TW*>(cbase) + ((size_t)src * n_kv + h) * hd;
-          lo = to_f(cp[e]);
-          hi = to_f(cp[half + e]);
-        } else if constexpr (FMT == AKVS_KV_FP8) {
-          const uint8_t* cp = reinterpret_cast<const uint8_t*>(cbase) + ((size_t)src * n_kv + h) * hd;
-          const __half_raw ra = __nv_cvt_fp8_to_halfraw(cp[e], __NV_E4M3), rb = __nv_cvt_fp8_to_halfraw(cp[half + e], __NV_E4M3);
-          lo = __half2float(*reinterpret_cast<const __half*>(&ra));
-          hi = __half2float(*reinterpret_cast<const __half*>(&rb));
-        } else {
-          const uint8_t* cp = reinterpret_cast<const uint8_t*>(cbase) + ((size_t)src * n_kv + h) * hd * FMT / 8;
-          const __half2* mp = reinterpret_cast<const __half2*>(cmeta) + ((size_t)src * n_kv + h) * (hd / 64);
-          const int e2 = half + e;
-          const uint32_t qa = (cp[e * FMT / 8] >> ((e * FMT) & 7)) & ((1u << FMT) - 1u);
-          const uint32_t qb = (cp[e2 * FMT / 8] >> ((e2 * FMT) & 7)) & ((1u << FMT) - 1u);
-          const __half2 ma = mp[e / 64], mb = mp[e2 / 64];
-          lo = __fmaf_rn((float)qa, __low2float(ma), __high2float(ma));
-          hi = __fmaf_rn((float)qb, __low2float(mb), __high2float(mb));
-        }
+      for (int e = 0; e < V; ++e) {
+        float rl = lo[e], rh = hi[e];
         if (!is_v) {
-          const float2 t = rot[e];
-          const float rlo = lo * t.x - hi * t.y, rhi = hi * t.x + lo * t.y;
-          lo = rlo;
-          hi = rhi;
+          rl = lo[e] * rot[e].x - hi[e] * rot[e].y;
+          rh = hi[e] * rot[e].x + lo[e] * rot[e].y;
         }
-        acc_lo[q] += to_f(fp[e]) - lo;
-        acc_hi[q] += to_f(fp[half + e]) - hi;
+        acc_lo[e] += flo[e] - rl;
+        acc_hi[e] += fhi[e] - rh;
       }
     }
-  }
 #pragma unroll
-  for (int q = 0; q < OFF_Q; ++q) {
-    const int e = lane + 32 * q;
-    if (e < half) { part[wid * hd + e] = acc_lo[q]; part[wid * hd + half + e] = acc_hi[q]; }
+    for (int e = 0; e < V; ++e) {
+      part[slot * hd + c * V + e] = acc_lo[e];
+      part[slot * hd + half + c * V + e] = acc_hi[e];
+    }
   }
   __syncthreads();
   float* mu = (is_v ? mu_v : mu_k) + ((size_t)u * n_kv + h) * hd;
-  for (int e = threadIdx.x; e < hd; e += OFF_WARPS * 32) {
+  for (int e = threadIdx.x; e < hd; e += OFF_THREADS) {
     float s = 0.f;
-#pragma unroll
-    for (int w = 0; w < OFF_WARPS; ++w) s += part[w * hd + e];
+    for (int w = 0; w < slots; ++w) s += part[w * hd + e];
     mu[e] = b > 0 ? s / (float)b : 0.f;
   }
 }
 
 int32_t launch_offsets(int dtype, const KvLayer& kv, const ReqMaps& maps, const int32_t* probe_off,
                        const int32_t* sk_idx, const int32_t* sv_idx, const void* k_fresh, const void* v_fresh, int M,
-                       int n_kv, int hd, const float2* table, float* mu_k, float* mu_v, cudaStream_t st) {
+                       int N, int n_probe_cap, int n_kv, int hd, const float2* table, float* mu_k, float* mu_v,
+                       int32_t* status, cudaStream_t st) {
   if (M == 0) return AKVS_OK;
   AKVS_TRY(check_kv_shape(dtype, kv, hd));
-  if (hd > 256) return AKVS_ERR_UNSUPPORTED;      // a lane keeps at most 4 rotation pairs
+  const int V = dtype == AKVS_F32 ? 4 : 8;
+  const int ch = hd / 2 / V;
+  if (ch > OFF_THREADS) return AKVS_ERR_UNSUPPORTED;
   const dim3 grid(M, n_kv, 2);
-  const size_t smem = (size_t)OFF_WARPS * hd * sizeof(float);
+  const size_t smem = (size_t)(OFF_THREADS / ch) * hd * sizeof(float);
+  if (smem > 48 * 1024) return AKVS_ERR_UNSUPPORTED;
   ProfScope prof(5, kv.fmt, 0.0, st);
   return dispatch_dtype(dtype, [&](auto tag) -> int32_t {
     using T = decltype(tag);
     return dispatch_fmt(kv.fmt, [&](auto f) -> int32_t {
-      AKVS_CUDA(launch_pdl(offsets_kernel<T, T, decltype(f)::value>, grid, dim3(OFF_WARPS * 32), smem, st, kv, maps,
-                           probe_off, sk_idx, sv_idx, (const T*)k_fresh, (const T*)v_fresh, n_kv, hd, table, mu_k, mu_v));
+      AKVS_CUDA(launch_pdl(offsets_kernel<T, T, decltype(f)::value>, grid, dim3(OFF_THREADS), smem, st, kv, maps,
+                           probe_off, sk_idx, sv_idx, (const T*)k_fresh, (const T*)v_fresh, N, n_probe_cap, n_kv, hd,
+                           table, mu_k, mu_v, status));
       AKVS_LAUNCHED();
       return AKVS_OK;
     });
@@ -469,13 +481,45 @@ int32_t launch_offsets(int dtype, const KvLayer& kv, const ReqMaps& maps, const 
 //   context token j of unit u, not in S^K:  K_out = Rot(off_u) deq(K_cached) + w_K[j] mu_K[u]
 //                              in S^K:      K_out = fresh K of its recomputed row
 //   V likewise with S^V (no rotation);  query token i: fresh K/V of row P + i.
-// One thread owns one pair chunk (16 B of the lower half of a head + its RoPE partner in the
-// upper half) of COR_TOK consecutive tokens: it first issues all of their 16-byte loads
-// (4 per token: K lo/hi, V lo/hi), then decodes, rotates, corrects and stores.  The unit's
-// rotation row and offsets are fetched once per run of tokens of the same unit, so that the
-// L1 traffic per token is little more than the data itself.
+//
+// Work split: a token's K row and V row are two "role rows"; a thread owns ONE pair chunk (16
+// bytes of the lower half of a head + its RoPE partner 16 bytes in the upper half) of one role
+// for the whole launch, so its rotation entries and the unit's offsets sit in registers and are
+// refetched only when the token's unit changes (units are runs of >= a hundred tokens).  The
+// threads of a role row read and write its heads as whole 128-byte lines.  A CTA takes a
+// contiguous slice of tokens, `tl` tokens side by side, COR_U tokens per thread and batch: the
+// thread first reads the batch's per-token records (one 16-byte load each, weight included),
+// then issues all 2 COR_U data loads, then decodes / rotates / adds w mu on packed float pairs
+// (fma.rn.f32x2: half the floating-point issue slots) and stores.  Fresh rows (probes, query)
+// are copied as the 16 bytes they are.  The grid is one wave: slices are sized so that every
+// CTA slot of the device gets one slice of the same length.
 // ---------------------------------------------------------------------------------------
-constexpr int COR_TOK = 2;
+#ifndef AKVS_COR_U
+#define AKVS_COR_U 4
+#endif
+#ifndef AKVS_COR_CTAS
+#define AKVS_COR_CTAS 2
+#endif
+constexpr int COR_THREADS = 256, COR_U = AKVS_COR_U, COR_CTAS_PER_SM = AKVS_COR_CTAS;
+
+__device__ __forceinline__ uint64_t pk2(float lo, float hi) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ void upk2(uint64_t v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t r;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+  return r;
+}
+__device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b) {
+  uint64_t r;
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
 
 template <typename TW, int FMT> struct RawChunk;
 template <typename TW> struct RawChunk<TW, AKVS_KV_NATIVE> { uint4 v; };
@@ -500,23 +544,18 @@ __device__ __forceinline__ void unpack16(const uint4& r, float (&o)[8], const f1
   }
 }
 
-// Issues the load of one 16-byte-equivalent chunk: either from the fresh rows (T) or from
-// the cache in its own format.  A native cache of the same element type shares the register
-// with the fresh row (one pointer select, one load).
+// Issues the load of one chunk of the cache in its own format (V elements from element `e0` of
+// store row `src`): 16 bytes for a native cache, V bytes for FP8, V * bits / 8 bytes of codes and
+// the group's (scale, min) record for the group-quantised formats.
 template <typename T, typename TW, int FMT>
-__device__ __forceinline__ void issue_chunk(bool from_fresh, const T* fresh_p, const void* base, const void* meta,
-                                            int64_t src, int n_kv, int hd, int h, int dim0, uint4& fresh_raw,
-                                            RawChunk<TW, FMT>& raw) {
+__device__ __forceinline__ void issue_cached(const void* base, const void* meta, int64_t src, int row_elems, int hd,
+                                             int e0, RawChunk<TW, FMT>& raw) {
   constexpr int V = VecOf<T>::N;
-  if constexpr (FMT == AKVS_KV_NATIVE && std::is_same<T, TW>::value) {
-    const T* cp = reinterpret_cast<const T*>(base) + ((size_t)(from_fresh ? 0 : src) * n_kv + h) * hd + dim0;
-    fresh_raw = *reinterpret_cast<const uint4*>(from_fresh ? fresh_p : cp);
-  } else if (from_fresh) {
-    fresh_raw = *reinterpret_cast<const uint4*>(fresh_p);
-  } else if constexpr (FMT == AKVS_KV_NATIVE) {
-    raw.v = *reinterpret_cast<const uint4*>(reinterpret_cast<const TW*>(base) + ((size_t)src * n_kv + h) * hd + dim0);
+  const size_t e = (size_t)src * row_elems + e0;
+  if constexpr (FMT == AKVS_KV_NATIVE) {
+    raw.v = *reinterpret_cast<const uint4*>(reinterpret_cast<const TW*>(base) + e);
   } else if constexpr (FMT == AKVS_KV_FP8) {
-    const uint8_t* cp = reinterpret_cast<const uint8_t*>(base) + ((size_t)src * n_kv + h) * hd + dim0;
+    const uint8_t* cp = reinterpret_cast<const uint8_t*>(base) + e;
     if constexpr (V == 8) {
       const uint2 t = *reinterpret_cast<const uint2*>(cp);
       raw.w[0] = t.x; raw.w[1] = t.y;
@@ -525,19 +564,14 @@ __device__ __forceinline__ void issue_chunk(bool from_fresh, const T* fresh_p, c
     }
   } else {
     constexpr int BYTES = V * FMT / 8;
-    raw.packed = ld_codes<BYTES>(reinterpret_cast<const uint8_t*>(base) + (((size_t)src * n_kv + h) * hd + dim0) * FMT / 8);
-    raw.sm = reinterpret_cast<const __half2*>(meta)[((size_t)src * n_kv + h) * (hd / 64) + dim0 / 64];
+    raw.packed = ld_codes<BYTES>(reinterpret_cast<const uint8_t*>(base) + e * FMT / 8);
+    raw.sm = reinterpret_cast<const __half2*>(meta)[e / 64];          // hd is a multiple of 64: groups do not straddle heads
   }
 }
 template <typename T, typename TW, int FMT>
-__device__ __forceinline__ void decode_chunk(bool from_fresh, const uint4& fresh_raw, const RawChunk<TW, FMT>& raw,
-                                             float (&out)[VecOf<T>::N]) {
+__device__ __forceinline__ void decode_cached(const RawChunk<TW, FMT>& raw, float (&out)[VecOf<T>::N]) {
   constexpr int V = VecOf<T>::N;
-  if constexpr (FMT == AKVS_KV_NATIVE && std::is_same<T, TW>::value) {
-    unpack16(fresh_raw, out, (const T*)nullptr);
-  } else if (from_fresh) {
-    unpack16(fresh_raw, out, (const T*)nullptr);
-  } else if constexpr (FMT == AKVS_KV_NATIVE) {
+  if constexpr (FMT == AKVS_KV_NATIVE) {
     unpack16(raw.v, out, (const TW*)nullptr);
   } else if constexpr (FMT == AKVS_KV_FP8) {
 #pragma unroll
@@ -553,131 +587,154 @@ __device__ __forceinline__ void decode_chunk(bool from_fresh, const uint4& fresh
   }
 }
 
-// V consecutive floats / float2 as 16-byte loads (the addresses are 16-byte aligned by layout)
-template <int V>
-__device__ __forceinline__ void ld_f(const float* p, float (&o)[V]) {
-#pragma unroll
-  for (int i = 0; i < V; i += 4) {
-    const float4 t = *reinterpret_cast<const float4*>(p + i);
-    o[i] = t.x; o[i + 1] = t.y; o[i + 2] = t.z; o[i + 3] = t.w;
-  }
-}
-template <int V>
-__device__ __forceinline__ void ld_f2(const float2* p, float2 (&o)[V]) {
-#pragma unroll
-  for (int i = 0; i < V; i += 2) {
-    const float4 t = *reinterpret_cast<const float4*>(p + i);
-    o[i] = make_float2(t.x, t.y); o[i + 1] = make_float2(t.z, t.w);
-  }
-}
-
 template <typename T, typename TW, int FMT>
-__global__ void __launch_bounds__(256, 2)
-correct_kernel(KvLayer kv, ReqMaps maps, const T* __restrict__ k_fresh, const T* __restrict__ v_fresh,
-               const float* __restrict__ w_k, const float* __restrict__ w_v, const float* __restrict__ mu_k,
-               const float* __restrict__ mu_v, int N, int T_tok, int n_probe_rows, int n_kv, int hd,
+__global__ void __launch_bounds__(COR_THREADS, COR_CTAS_PER_SM)
+correct_kernel(KvLayer kv, const int4* __restrict__ tok_meta, const int32_t* __restrict__ unit_pos,
+               const T* __restrict__ k_fresh, const T* __restrict__ v_fresh, const float* __restrict__ mu_k,
+               const float* __restrict__ mu_v, int T_tok, int n_kv, int hd, int ipt, int tl, int slice, int weighted,
                const float2* __restrict__ table, T* __restrict__ out_k, T* __restrict__ out_v) {
+  // ipt = pair chunks of the kv heads this CTA column (blockIdx.y) covers: heads_per_cta * chunks per head
   constexpr int V = VecOf<T>::N;
   pdl_trigger();
   pdl_wait();
+  const int tpt = 2 * ipt;                              // threads per token: K items, then V items
+  const int lane_tok = threadIdx.x / tpt;
+  if (lane_tok >= tl) return;
+  const int rem = threadIdx.x - lane_tok * tpt;
+  const int role = rem / ipt;                           // 0: K, 1: V
+  const int item = rem - role * ipt;
   const int half = hd / 2, ch = half / V;
-  const int groups = (T_tok + COR_TOK - 1) / COR_TOK;
-  const int total = groups * n_kv * ch;                 // < 2^31: checked by the launcher
-  const bool weighted = w_k != nullptr;
-  for (int idx = blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += gridDim.x * blockDim.x) {
-    const int c = idx % ch;
-    const int h = (idx / ch) % n_kv;
-    const int j0 = (idx / (ch * n_kv)) * COR_TOK;
-    int4 meta[COR_TOK];
-    float wk[COR_TOK], wv[COR_TOK];
+  const int h = blockIdx.y * (ipt / ch) + item / ch, c = item % ch;
+  if (h >= n_kv) return;                                // the last head group may be short
+  const int row_elems = n_kv * hd;
+  const int col = h * hd + c * V;                       // element of the lower chunk within a role row
+  const int4* __restrict__ meta = tok_meta + (size_t)role * T_tok;
+  const T* __restrict__ fresh = role ? v_fresh : k_fresh;
+  const void* cbase = role ? kv.v : kv.k;
+  const void* cmeta = role ? kv.v_meta : kv.k_meta;
+  const float* __restrict__ mu = role ? mu_v : mu_k;
+  T* __restrict__ out = role ? out_v : out_k;
+  const int t_end = min(T_tok, (blockIdx.x + 1) * slice);
+
+  uint64_t C2[V / 2], S2[V / 2], ML2[V / 2], MH2[V / 2];   // (cos, cos), (sin, sin), offsets of the lower / upper chunk
+  int cur_unit = -1;
+  for (int b0 = blockIdx.x * slice + lane_tok; b0 < t_end; b0 += tl * COR_U) {
+    int4 mt[COR_U];
 #pragma unroll
-    for (int t = 0; t < COR_TOK; ++t) {
-      const int j = j0 + t;
-      meta[t] = j < T_tok ? maps.tok_meta[j] : make_int4(-1, -1, -1, -1);
-      const bool ctx = j < N && weighted;
-      wk[t] = ctx ? w_k[j] : 0.f;
-      wv[t] = ctx ? w_v[j] : 0.f;
+    for (int u = 0; u < COR_U; ++u) {
+      const int j = b0 + u * tl;
+      mt[u] = j < t_end ? meta[j] : make_int4(-1, -1, 0, 0);
     }
-    // ---- all loads first
-    uint4 fk_lo[COR_TOK], fk_hi[COR_TOK], fv_lo[COR_TOK], fv_hi[COR_TOK];
-    RawChunk<TW, FMT> ck_lo[COR_TOK], ck_hi[COR_TOK], cv_lo[COR_TOK], cv_hi[COR_TOK];
+    // ---- all data loads of the batch (a native cache of the model's type shares the registers
+    // of the fresh rows: one pointer select, one pair of loads)
+    constexpr bool kShared = FMT == AKVS_KV_NATIVE && std::is_same<T, TW>::value;
+    uint4 f_lo[COR_U], f_hi[COR_U];
+    RawChunk<TW, FMT> c_lo[kShared ? 1 : COR_U], c_hi[kShared ? 1 : COR_U];
 #pragma unroll
-    for (int t = 0; t < COR_TOK; ++t) {
-      if (j0 + t >= T_tok) continue;
-      const bool kf = meta[t].y >= 0, vf = meta[t].z >= 0;
-      const T* fkp = k_fresh + ((size_t)(kf ? meta[t].y : 0) * n_kv + h) * hd + c * V;
-      const T* fvp = v_fresh + ((size_t)(vf ? meta[t].z : 0) * n_kv + h) * hd + c * V;
-      issue_chunk<T, TW, FMT>(kf, fkp, kv.k, kv.k_meta, meta[t].x, n_kv, hd, h, c * V, fk_lo[t], ck_lo[t]);
-      issue_chunk<T, TW, FMT>(kf, fkp + half, kv.k, kv.k_meta, meta[t].x, n_kv, hd, h, half + c * V, fk_hi[t], ck_hi[t]);
-      issue_chunk<T, TW, FMT>(vf, fvp, kv.v, kv.v_meta, meta[t].x, n_kv, hd, h, c * V, fv_lo[t], cv_lo[t]);
-      issue_chunk<T, TW, FMT>(vf, fvp + half, kv.v, kv.v_meta, meta[t].x, n_kv, hd, h, half + c * V, fv_hi[t], cv_hi[t]);
+    for (int u = 0; u < COR_U; ++u) {
+      if (b0 + u * tl >= t_end) continue;
+      if (kShared || mt[u].y >= 0) {
+        const T* fp = mt[u].y >= 0 ? fresh + (size_t)mt[u].y * row_elems + col
+                                   : reinterpret_cast<const T*>(cbase) + (size_t)mt[u].x * row_elems + col;
+        f_lo[u] = *reinterpret_cast<const uint4*>(fp);
+        f_hi[u] = *reinterpret_cast<const uint4*>(fp + half);
+      } else {
+        issue_cached<T, TW, FMT>(cbase, cmeta, mt[u].x, row_elems, hd, col, c_lo[kShared ? 0 : u]);
+        issue_cached<T, TW, FMT>(cbase, cmeta, mt[u].x, row_elems, hd, col + half, c_hi[kShared ? 0 : u]);
+      }
     }
     // ---- decode, re-align, correct, store
-    float2 rot[V];
-    float muk_lo[V], muk_hi[V], muv_lo[V], muv_hi[V];
-    int cur_unit = -1;
 #pragma unroll
-    for (int t = 0; t < COR_TOK; ++t) {
-      const int j = j0 + t;
-      if (j >= T_tok) continue;
-      const bool kf = meta[t].y >= 0, vf = meta[t].z >= 0;
-      const int u = meta[t].w;
-      if ((!kf || !vf) && u != cur_unit) {
-        cur_unit = u;
-        ld_f2<V>(table + (size_t)maps.unit_pos[u] * half + c * V, rot);
+    for (int u = 0; u < COR_U; ++u) {
+      const int j = b0 + u * tl;
+      if (j >= t_end) continue;
+      T* op = out + (size_t)j * row_elems + col;
+      if (mt[u].y >= 0) {                               // a fresh row: the bytes as they are
+        *reinterpret_cast<uint4*>(op) = f_lo[u];
+        *reinterpret_cast<uint4*>(op + half) = f_hi[u];
+        continue;
+      }
+      if (mt[u].z != cur_unit) {
+        cur_unit = mt[u].z;
+        if (role == 0) {
+          float2 rot[V];
+          ld_f2<V>(table + (size_t)unit_pos[cur_unit] * half + c * V, rot);
+#pragma unroll
+          for (int i = 0; i < V / 2; ++i) {
+            C2[i] = pk2(rot[2 * i].x, rot[2 * i + 1].x);
+            S2[i] = pk2(rot[2 * i].y, rot[2 * i + 1].y);
+          }
+        }
         if (weighted) {
-          const float* mk = mu_k + ((size_t)u * n_kv + h) * hd + c * V;
-          const float* mv = mu_v + ((size_t)u * n_kv + h) * hd + c * V;
-          ld_f<V>(mk, muk_lo);
-          ld_f<V>(mk + half, muk_hi);
-          ld_f<V>(mv, muv_lo);
-          ld_f<V>(mv + half, muv_hi);
+          float ml[V], mh[V];
+          const float* mp = mu + (size_t)cur_unit * row_elems + col;
+          ld_f<V>(mp, ml);
+          ld_f<V>(mp + half, mh);
+#pragma unroll
+          for (int i = 0; i < V / 2; ++i) { ML2[i] = pk2(ml[2 * i], ml[2 * i + 1]); MH2[i] = pk2(mh[2 * i], mh[2 * i + 1]); }
         } else {
 #pragma unroll
-          for (int i = 0; i < V; ++i) muk_lo[i] = muk_hi[i] = muv_lo[i] = muv_hi[i] = 0.f;
+          for (int i = 0; i < V / 2; ++i) ML2[i] = MH2[i] = 0ull;
         }
       }
-      const size_t o = ((size_t)j * n_kv + h) * hd + c * V;
       float lo[V], hi[V];
-      decode_chunk<T, TW, FMT>(kf, fk_lo[t], ck_lo[t], lo);
-      decode_chunk<T, TW, FMT>(kf, fk_hi[t], ck_hi[t], hi);
-      if (!kf) {
-#pragma unroll
-        for (int i = 0; i < V; ++i) {
-          const float a = lo[i], b = hi[i];
-          lo[i] = fmaf(wk[t], muk_lo[i], a * rot[i].x - b * rot[i].y);
-          hi[i] = fmaf(wk[t], muk_hi[i], b * rot[i].x + a * rot[i].y);
-        }
+      if constexpr (kShared) {
+        unpack16(f_lo[u], lo, (const T*)nullptr);
+        unpack16(f_hi[u], hi, (const T*)nullptr);
+      } else {
+        decode_cached<T, TW, FMT>(c_lo[u], lo);
+        decode_cached<T, TW, FMT>(c_hi[u], hi);
       }
-      st16(out_k + o, lo);
-      st16(out_k + o + half, hi);
-      decode_chunk<T, TW, FMT>(vf, fv_lo[t], cv_lo[t], lo);
-      decode_chunk<T, TW, FMT>(vf, fv_hi[t], cv_hi[t], hi);
-      if (!vf) {
+      const float w = __int_as_float(mt[u].w);
+      const uint64_t W2 = pk2(w, w);
 #pragma unroll
-        for (int i = 0; i < V; ++i) {
-          lo[i] = fmaf(wv[t], muv_lo[i], lo[i]);
-          hi[i] = fmaf(wv[t], muv_hi[i], hi[i]);
+      for (int i = 0; i < V / 2; ++i) {
+        const uint64_t A2 = pk2(lo[2 * i], lo[2 * i + 1]), B2 = pk2(hi[2 * i], hi[2 * i + 1]);
+        uint64_t rl, rh;
+        if (role == 0) {
+          // lo' = a cos - b sin + w mu_lo,  hi' = b cos + a sin + w mu_hi
+          const uint64_t nb = B2 ^ 0x8000000080000000ull;               // (-b, -b): sign bits
+          rl = fma2(nb, S2[i], fma2(W2, ML2[i], mul2(A2, C2[i])));
+          rh = fma2(A2, S2[i], fma2(W2, MH2[i], mul2(B2, C2[i])));
+        } else {
+          rl = fma2(W2, ML2[i], A2);
+          rh = fma2(W2, MH2[i], B2);
         }
+        upk2(rl, lo[2 * i], lo[2 * i + 1]);
+        upk2(rh, hi[2 * i], hi[2 * i + 1]);
       }
-      st16(out_v + o, lo);
-      st16(out_v + o + half, hi);
+      st16(op, lo);
+      st16(op + half, hi);
     }
   }
 }
 
+int g_cor_slots = 0;                 // CTA slots of the device for the correction kernel (SMs x CTAs per SM)
+
 int32_t launch_correct(int dtype, const KvLayer& kv, const ReqMaps& maps, const void* k_fresh, const void* v_fresh,
-                       const float* w_k, const float* w_v, const float* mu_k, const float* mu_v, int N, int n_query,
-                       int n_probe_rows, int n_kv, int hd, const float2* table, void* out_k, void* out_v,
-                       cudaStream_t st) {
+                       bool weighted, const float* mu_k, const float* mu_v, int N, int n_query, int n_kv, int hd,
+                       const float2* table, void* out_k, void* out_v, cudaStream_t st) {
   const int T_tok = N + n_query;
   if (T_tok == 0) return AKVS_OK;
   AKVS_TRY(check_kv_shape(dtype, kv, hd));
   const int V = dtype == AKVS_F32 ? 4 : 8;
-  const int64_t total = (int64_t)((T_tok + COR_TOK - 1) / COR_TOK) * n_kv * (hd / 2 / V);
-  if (total >= (1ll << 31) - (1 << 20)) return AKVS_ERR_SHAPE;
-  int64_t want = (total + 255) / 256;
-  const int grid = (int)(want < 148 * 4 ? want : 148 * 4);   // grid-stride; two resident CTAs of 256 threads per SM
+  const int ch = hd / 2 / V;                            // pair chunks of one head
+  if (2 * ch > COR_THREADS) return AKVS_ERR_UNSUPPORTED;
+  const int heads_per_cta = n_kv < COR_THREADS / (2 * ch) ? n_kv : COR_THREADS / (2 * ch);
+  const int head_groups = (n_kv + heads_per_cta - 1) / heads_per_cta;
+  const int ipt = heads_per_cta * ch;                   // pair chunks of one role row within a head group
+  if ((int64_t)T_tok * n_kv * hd >= (1ll << 31)) return AKVS_ERR_SHAPE;     // 32-bit element offsets inside a layer
+  if (!g_cor_slots) {
+    int dev = 0, sms = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    g_cor_slots = (sms > 0 ? sms : 148) * COR_CTAS_PER_SM;
+  }
+  const int tl = COR_THREADS / (2 * ipt);               // tokens side by side in a CTA
+  const int slots = g_cor_slots / head_groups > 0 ? g_cor_slots / head_groups : 1;
+  int slice = (T_tok + slots - 1) / slots;              // one wave of equal slices
+  slice = (slice + tl - 1) / tl * tl;
+  const int grid = (T_tok + slice - 1) / slice;
   // algorithmic bytes: every context K and V element read once in its cache format and
   // written once; fresh rows and query rows copied; 8 bytes of weights per context token
   const double in_b = kv.fmt == AKVS_KV_NATIVE ? (double)dtype_size(dtype)
@@ -688,9 +745,9 @@ int32_t launch_correct(int dtype, const KvLayer& kv, const ReqMaps& maps, const 
   return dispatch_dtype(dtype, [&](auto tag) -> int32_t {
     using T = decltype(tag);
     return dispatch_fmt(kv.fmt, [&](auto f) -> int32_t {
-      AKVS_CUDA(launch_pdl(correct_kernel<T, T, decltype(f)::value>, dim3(grid), dim3(256), 0, st, kv, maps,
-                           (const T*)k_fresh, (const T*)v_fresh, w_k, w_v, mu_k, mu_v, N, T_tok, n_probe_rows, n_kv, hd,
-                           table, (T*)out_k, (T*)out_v));
+      AKVS_CUDA(launch_pdl(correct_kernel<T, T, decltype(f)::value>, dim3(grid, head_groups), dim3(COR_THREADS), 0, st, kv,
+                           maps.tok_meta, maps.unit_pos, (const T*)k_fresh, (const T*)v_fresh, mu_k, mu_v, T_tok, n_kv,
+                           hd, ipt, tl, slice, weighted ? 1 : 0, table, (T*)out_k, (T*)out_v));
       AKVS_LAUNCHED();
       return AKVS_OK;
     });

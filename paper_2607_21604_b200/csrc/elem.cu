@@ -7,17 +7,27 @@
 // ---------------------------------------------------------------------------------------
 // h[r][:] = float(tok_emb[ids[gather ? gather[r] : r]][:])
 // ---------------------------------------------------------------------------------------
+// A token id outside [0, vocab) (ids are caller data) raises AKVS_ERR_INVALID_ARG in the status
+// word and the row is written as zeros: the table is never read out of range.
 template <typename T>
 __global__ void embed_kernel(const T* __restrict__ emb, const int32_t* __restrict__ ids,
-                             const int32_t* __restrict__ gather, int n, int d, float* __restrict__ h) {
+                             const int32_t* __restrict__ gather, int n, int d, int vocab, int32_t* status,
+                             float* __restrict__ h) {
   constexpr int V = VecOf<T>::N;
   const int r = blockIdx.x;
   const int id = ids[gather ? gather[r] : r];
-  const T* src = emb + (size_t)id * d;
+  const bool ok = id >= 0 && id < vocab;
+  if (!ok && threadIdx.x == 0) set_status(status, AKVS_ERR_INVALID_ARG);
+  const T* src = emb + (size_t)(ok ? id : 0) * d;
   float* dst = h + (size_t)r * d;
   for (int c = threadIdx.x * V; c < d; c += blockDim.x * V) {
     float v[V];
-    ld16(src + c, v);
+    if (ok) {
+      ld16(src + c, v);
+    } else {
+#pragma unroll
+      for (int i = 0; i < V; ++i) v[i] = 0.f;
+    }
 #pragma unroll
     for (int i = 0; i < V; i += 4) {
       float t[4] = {v[i], v[i + 1], v[i + 2], v[i + 3]};
@@ -27,27 +37,33 @@ __global__ void embed_kernel(const T* __restrict__ emb, const int32_t* __restric
 }
 
 int32_t launch_embed(int dtype, const void* tok_emb, const int32_t* ids, const int32_t* gather, int n, int d,
-                     float* h, cudaStream_t st) {
+                     int vocab, int32_t* status, float* h, cudaStream_t st) {
   if (n == 0) return AKVS_OK;
   return dispatch_dtype(dtype, [&](auto tag) -> int32_t {
     using T = decltype(tag);
-    embed_kernel<T><<<n, 128, 0, st>>>((const T*)tok_emb, ids, gather, n, d, h);
+    embed_kernel<T><<<n, 128, 0, st>>>((const T*)tok_emb, ids, gather, n, d, vocab, status, h);
     AKVS_LAUNCHED();
     return AKVS_OK;
   });
 }
 
-__global__ void gather_rows_kernel(const float* __restrict__ src, const int32_t* __restrict__ rows, int d,
-                                   float* __restrict__ dst) {
+// rows[] may have been written by the caller (akvs_probes.rows): an entry outside [0, n_src)
+// raises AKVS_ERR_INVALID_ARG and yields a row of zeros instead of an out-of-range read.
+__global__ void gather_rows_kernel(const float* __restrict__ src, const int32_t* __restrict__ rows, int d, int n_src,
+                                   int32_t* status, float* __restrict__ dst) {
   const int r = blockIdx.x;
-  const float4* s = reinterpret_cast<const float4*>(src + (size_t)rows[r] * d);
+  const int j = rows[r];
+  const bool ok = j >= 0 && j < n_src;
+  if (!ok && threadIdx.x == 0) set_status(status, AKVS_ERR_INVALID_ARG);
+  const float4* s = reinterpret_cast<const float4*>(src + (size_t)(ok ? j : 0) * d);
   float4* t = reinterpret_cast<float4*>(dst + (size_t)r * d);
-  for (int c = threadIdx.x; c < d / 4; c += blockDim.x) t[c] = s[c];
+  for (int c = threadIdx.x; c < d / 4; c += blockDim.x) t[c] = ok ? s[c] : make_float4(0.f, 0.f, 0.f, 0.f);
 }
 
-int32_t launch_gather_rows(const float* src, const int32_t* rows, int n, int d, float* dst, cudaStream_t st) {
+int32_t launch_gather_rows(const float* src, const int32_t* rows, int n, int d, int n_src, int32_t* status, float* dst,
+                           cudaStream_t st) {
   if (n == 0) return AKVS_OK;
-  gather_rows_kernel<<<n, 256, 0, st>>>(src, rows, d, dst);
+  gather_rows_kernel<<<n, 256, 0, st>>>(src, rows, d, n_src, status, dst);
   AKVS_LAUNCHED();
   return AKVS_OK;
 }
@@ -156,7 +172,7 @@ int32_t launch_rope_table(float base, int hd, int n_pos, float2* table, cudaStre
 // the lower half; it also owns the partner chunk in the upper half.
 template <typename T>
 __global__ void rope_kernel(T* __restrict__ x, const int32_t* __restrict__ pos, int n, int n_heads, int hd, int ld,
-                            const float2* __restrict__ table, double base) {
+                            const float2* __restrict__ table, int n_pos, int32_t* status, double base) {
   constexpr int V = VecOf<T>::N;
   pdl_trigger();
   pdl_wait();
@@ -166,7 +182,11 @@ __global__ void rope_kernel(T* __restrict__ x, const int32_t* __restrict__ pos, 
   const int c = (int)(idx % ch);
   const int hh = (int)((idx / ch) % n_heads);
   const int r = (int)(idx / ((int64_t)ch * n_heads));
-  const int p = pos[r];
+  int p = pos[r];
+  if (table && (p < 0 || p >= n_pos)) {           // positions may be caller data: never index past the table
+    set_status(status, AKVS_ERR_INVALID_ARG);
+    p = 0;
+  }
   T* lo_p = x + (size_t)r * ld + (size_t)hh * hd + c * V;
   T* hi_p = lo_p + half;
   float lo[V], hi[V], olo[V], ohi[V];
@@ -194,7 +214,7 @@ __global__ void rope_kernel(T* __restrict__ x, const int32_t* __restrict__ pos, 
 }
 
 int32_t launch_rope(int dtype, void* x, const int32_t* pos, int n, int n_heads, int hd, int ld,
-                    const float2* table, float base, cudaStream_t st) {
+                    const float2* table, int n_pos, int32_t* status, float base, cudaStream_t st) {
   if (n == 0) return AKVS_OK;
   const int V = dtype == AKVS_F32 ? 4 : 8;
   if (hd % (2 * V) != 0) return AKVS_ERR_UNSUPPORTED;
@@ -202,7 +222,8 @@ int32_t launch_rope(int dtype, void* x, const int32_t* pos, int n, int n_heads, 
   const int blocks = akvs_cdiv(total, 256);
   return dispatch_dtype(dtype, [&](auto tag) -> int32_t {
     using T = decltype(tag);
-    AKVS_CUDA(launch_pdl(rope_kernel<T>, dim3(blocks), dim3(256), 0, st, (T*)x, pos, n, n_heads, hd, ld, table, (double)base));
+    AKVS_CUDA(launch_pdl(rope_kernel<T>, dim3(blocks), dim3(256), 0, st, (T*)x, pos, n, n_heads, hd, ld, table, n_pos, status,
+                         (double)base));
     AKVS_LAUNCHED();
     return AKVS_OK;
   });

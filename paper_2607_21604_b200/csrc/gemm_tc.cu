@@ -48,6 +48,8 @@ struct GemmParams {
   const float2* rope;     // [positions][64] (cos, sin)
   const int32_t* pos;     // [M]
   int rope_mask;
+  int n_pos;              // rows of the rope table: a position outside [0, n_pos) (positions may be caller
+                          // data) raises AKVS_ERR_INVALID_ARG and is rotated as position 0
 };
 
 // Which weight matrix and which of its rows the 128-row block `block` of the concatenated
@@ -118,7 +120,12 @@ __device__ __forceinline__ void epilogue_warp(const GemmParams& p, uint32_t t_ad
     const int ldc = p.seg_ldc[seg];
     if (EPI == EPI_STORE && ((p.rope_mask >> seg) & 1)) {
       // this 128-column block is one head: rotate the pairs (i, i + 64) in registers
-      const float2* rt = p.rope + (size_t)(row < p.M ? p.pos[row] : 0) * 64;
+      int ps = row < p.M ? p.pos[row] : 0;
+      if ((unsigned)ps >= (unsigned)p.n_pos) {
+        set_status(p.status, AKVS_ERR_INVALID_ARG);
+        ps = 0;
+      }
+      const float2* rt = p.rope + (size_t)ps * 64;
       T* out = reinterpret_cast<T*>(p.seg_out[seg]);
 #pragma unroll 1
       for (int c = 0; c < 2; ++c) {
@@ -664,7 +671,7 @@ int32_t encode_tmap_3d_16bit(CUtensorMap* map, const void* base, uint64_t d0, ui
 //   epi 2: out[0] = silu(x w[0]^T) * (x w[1]^T) (16-bit), n[0] == n[1].
 int32_t launch_linear_tc(int dtype, int epi, const void* x, int M, int K, int n_seg, const void* const* w, const int* n,
                          void* const* out, const int* ldc, int32_t* status, cudaStream_t st, const float2* rope,
-                         const int32_t* pos, int rope_mask, int tiling) {
+                         const int32_t* pos, int rope_mask, int tiling, int n_pos) {
   if (M == 0) return AKVS_OK;
   if (K % 8 != 0 || n_seg < 1 || n_seg > 3) return AKVS_ERR_SHAPE;
   if (dtype != AKVS_BF16 && dtype != AKVS_F16) return AKVS_ERR_UNSUPPORTED;
@@ -691,7 +698,8 @@ int32_t launch_linear_tc(int dtype, int epi, const void* x, int M, int K, int n_
   p.status = status;
   p.rope = rope;
   p.pos = pos;
-  p.rope_mask = (epi == EPI_STORE && rope && pos) ? rope_mask : 0;
+  p.rope_mask = (epi == EPI_STORE && rope && pos && n_pos > 0) ? rope_mask : 0;
+  p.n_pos = n_pos;
   const uint32_t fmt = dtype == AKVS_F16 ? tc::kF16 : tc::kBF16;
   CUtensorMap tmA, tmB[3];
   AKVS_TRY(encode_tmap_2d_16bit(&tmA, x, M, K, K, BM));
@@ -735,7 +743,7 @@ int32_t launch_linear_tc(int dtype, int epi, const void* x, int M, int K, int n_
     const int r_pair = (t_pair + pairs - 1) / pairs, r_single = (t_single + sm_count() - 1) / sm_count();
     if (tiling == 2 || r_pair <= r_single) {
       p.tiles_m = tiles_m2;
-      p.idesc = tc::idesc_f16(fmt, fmt, 2 * BM, 2 * BNH, 0);
+      p.idesc = tc::idesc_f16(fmt, 2 * BM, 2 * BNH, 0);
       const int n_pairs = t_pair < pairs ? t_pair : pairs;
 #define AKVS_GEMM_LAUNCH(E, T) \
   AKVS_CUDA(launch_pdl_pair(gemm_tc_pair_kernel<E, T>, dim3(2 * n_pairs), dim3(THREADS), SMEM2_BYTES, st, tmA, tmB[0], tmB[1], tmB[2], p))
@@ -753,7 +761,7 @@ int32_t launch_linear_tc(int dtype, int epi, const void* x, int M, int K, int n_
       return AKVS_OK;
     }
   }
-  p.idesc = tc::idesc_f16(fmt, fmt, BM, p.nh * BNH, 0);
+  p.idesc = tc::idesc_f16(fmt, BM, p.nh * BNH, 0);
   const int n_tiles = p.tiles_m * p.tiles_n;
   const int grid = n_tiles < sm_count() ? n_tiles : sm_count();
 #define AKVS_GEMM_LAUNCH(E, T) \

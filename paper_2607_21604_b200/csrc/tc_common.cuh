@@ -43,14 +43,15 @@ __device__ __forceinline__ bool mbar_test(uint64_t* bar, uint32_t parity) {
 // Bounded wait.  Returns false when the limit ran out: the caller records AKVS_ERR_TIMEOUT,
 // stops its role and falls through to the common teardown.  No trap, no endless spin.
 constexpr long long kWaitCycles = 4000000000ll;   // about two seconds of SM clock
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
+                                          long long limit_cycles = kWaitCycles) {
   for (int it = 0; it < 128; ++it)
     if (mbar_test(bar, parity)) return true;
   const long long t0 = clock64();
   for (uint32_t it = 0;; ++it) {
     if (mbar_test(bar, parity)) return true;
     __nanosleep(32);
-    if ((it & 255) == 255 && (*abort_flag || clock64() - t0 > kWaitCycles)) return false;
+    if ((it & 255) == 255 && (*abort_flag || clock64() - t0 > limit_cycles)) return false;
   }
 }
 
@@ -110,13 +111,15 @@ __device__ __forceinline__ uint64_t smem_desc_mn_sw128(uint32_t saddr, uint32_t 
   d |= (uint64_t)2 << 61;
   return d;
 }
-// Instruction descriptor for kind::f16 (16-bit inputs, float accumulation).  A and B carry
-// their own format fields, so float16 activations can meet bfloat16 weights.
-//   bits 4-5 D format (1 = f32), 7-9 A format (0 = f16, 1 = bf16), 10-12 B format,
+// Instruction descriptor for kind::f16 (16-bit inputs, float accumulation).  BOTH operands
+// must have the SAME 16-bit format: the descriptor has a format field for A and one for B, but
+// an MMA issued with float16 in one and bfloat16 in the other raised "illegal instruction" on
+// the B200, so one `fmt` fills both fields and nothing here can build the mixed form.
+//   bits 4-5 D format (1 = f32), 7-9 A format (0 = f16, 1 = bf16), 10-12 B format (= A's),
 //   bit 15 A major (0 = K), bit 16 B major (0 = K, 1 = MN), 17-22 N >> 3, 24-28 M >> 4.
 constexpr uint32_t kF16 = 0, kBF16 = 1;
-__host__ __device__ constexpr uint32_t idesc_f16(uint32_t a_fmt, uint32_t b_fmt, int M, int N, int b_mn_major) {
-  return (1u << 4) | (a_fmt << 7) | (b_fmt << 10) | ((uint32_t)b_mn_major << 16) | ((uint32_t)(N >> 3) << 17) |
+__host__ __device__ constexpr uint32_t idesc_f16(uint32_t fmt, int M, int N, int b_mn_major) {
+  return (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)b_mn_major << 16) | ((uint32_t)(N >> 3) << 17) |
          ((uint32_t)(M >> 4) << 24);
 }
 

@@ -1,6 +1,7 @@
 """Plumbing shared by the GPU parity tests: the same seeded inputs go to the oracle (numpy,
 float64) and to the CUDA library (through the C ABI binding)."""
 import ctypes as C
+import dataclasses
 
 import numpy as np
 import torch
@@ -19,20 +20,24 @@ def t2n(t):
 class Case:
     """A workload instantiated on both sides."""
 
-    def __init__(self, w, std_scale=1.0, kv_format=0, order=None):
+    def __init__(self, w, std_scale=1.0, kv_format=0, order=None, omodel=None, gpu_dtype=None):
+        """`omodel`: an oracle model built elsewhere (shared between cases); `gpu_dtype`: storage
+        type of the library's model when it differs from the workload's (the weight VALUES must
+        then be representable in both, which holds for bf16 values rounded to float16)."""
         import paper_2607_21604_b200 as akvs
         self.akvs = akvs
         self.w, self.cfg = w, w.model
-        self.omodel = oracle_model(w.model, std_scale=std_scale)
+        self.omodel = oracle_model(w.model, std_scale=std_scale) if omodel is None else omodel
         self.lens, self.ctx_store, self.qry, self.units_ids = make_inputs(w)
         self.order = list(range(len(self.lens))) if order is None else list(order)
         self.ctx = np.concatenate([self.units_ids[u] for u in self.order]) if len(self.order) else np.zeros(0, np.int32)
         self.N, self.nq, self.M = len(self.ctx), len(self.qry), len(self.order)
-        self.gmodel = akvs.Model.from_numpy(w.model, self.omodel.tok_emb, self.omodel.layers)
+        gcfg = w.model if gpu_dtype is None else dataclasses.replace(w.model, dtype=gpu_dtype)
+        self.gmodel = akvs.Model.from_numpy(gcfg, self.omodel.tok_emb, self.omodel.layers)
         self.kv_format = kv_format
         self.store = akvs.UnitStore(self.gmodel, self.lens, self.ctx_store, kv_format)
         self.req = akvs.Request(self.order, self.qry)
-        self.tol = TOL[w.model.dtype]
+        self.tol = TOL[gcfg.dtype]
 
     def workspace(self, check_layer=1, n_ctx=None):
         n_ctx = max(self.N, self.store.n_tokens) if n_ctx is None else n_ctx

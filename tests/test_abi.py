@@ -11,7 +11,10 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 @pytest.fixture(scope="module")
 def lib():
-    from paper_2607_21604_b200 import build
+    import importlib.util
+    spec = importlib.util.spec_from_file_location("akvs_build", os.path.join(ROOT, "paper_2607_21604_b200", "build.py"))
+    build = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(build)                  # by path: importing the package needs the library built
     return C.CDLL(build.build())
 
 

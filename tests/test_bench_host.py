@@ -62,3 +62,21 @@ def test_max_over_ranks_with_two_gloo_processes():
         assert p.exitcode == 0
     assert ms == 20.0                       # the slowest rank decides
     assert rate == pytest.approx(2 * 1000 / 0.020)
+
+
+def test_oracle_sample_is_the_oracles_corrected_reuse_when_nothing_is_skipped():
+    """On the tiny configuration the bounded sample skips no row and no layer, so the steps it
+    strings together must reproduce the oracle's corrected reuse."""
+    import numpy as np
+    import bench
+    import testgen
+    from oracle import akvs_oracle as orc
+    w = testgen.workload("c1")
+    smp = bench.OracleSample(w)
+    smp.step()
+    assert smp.last["rows_sampled"] == smp.last["rows_recomputed"] and smp.last["dense_rows_sampled"] == smp.T
+    ctx = np.concatenate([np.asarray(testgen.token_ids(w, bench.SEED_IDS, testgen.unit_lengths(w, bench.SEED_LEN))[0])])
+    qry = testgen.token_ids(w, bench.SEED_IDS, testgen.unit_lengths(w, bench.SEED_LEN))[1]
+    ref = orc.corrected_reuse(smp.model, smp.units, smp.order, ctx, qry, smp.bp, bench.CHECK_LAYER)
+    assert np.allclose(smp.last_hidden, ref["hidden"], rtol=0, atol=1e-12)
+    assert smp.last["extrapolated_s"] > 0

@@ -1,0 +1,64 @@
+"""The sweep tool and the device-side timeout, on the GPU.
+
+* `paper_2607_21604_b200.sweep.run` on a small 2-layer model for two refresh ratios: the error
+  columns it prints (library against the library's own full recompute) must agree with the
+  same quantities computed by the oracle alone (Section 4.4 reports throughput against refresh
+  ratio; the error against full recompute is this build's quality proxy).
+* a bounded device wait that runs out: the status word reports AKVS_ERR_TIMEOUT, the context
+  stays usable and the next ordinary call succeeds."""
+import numpy as np
+import pytest
+import torch
+
+import testgen
+from oracle import akvs_oracle as orc
+from helpers import oracle_model, make_inputs
+
+pytestmark = pytest.mark.gpu
+
+
+def test_sweep_error_columns_agree_with_the_oracle():
+    from paper_2607_21604_b200 import sweep
+    cfg = testgen.ModelCfg("toy", 2, 256, 4, 2, 128, 768, 512, "f16")
+    w = testgen.Workload("toy", cfg, 4, 40, 90, 16, (2500,))
+    scale = 4.0
+    lines = []
+    rows = sweep.run(w, [1000, 4000], batches=(1,), check_layer=2, emit=lines.append, std_scale=scale)
+    assert len(rows) == 2 and sum(l.startswith("| ") for l in lines) == 3       # header + two data rows
+    om = oracle_model(cfg, std_scale=scale)
+    lens, ctx, qry, units_ids = make_inputs(w)
+    units = orc.encode_units(om, units_ids)
+    order = list(range(len(lens)))
+    full = orc.full_recompute(om, ctx, qry)[0]
+    naive = orc.naive_reuse(om, units, order, qry)[0]
+    e_naive = orc.rel_l2(naive, full)
+    for row in rows:
+        bp = row["refresh_bp"]
+        ref = orc.corrected_reuse(om, units, order, ctx, qry, bp, 2)
+        stale = orc.corrected_reuse(om, units, order, ctx, qry, bp, 2, zero_weights=True)
+        e_corr, e_sel = orc.rel_l2(ref["hidden"], full), orc.rel_l2(stale["hidden"], full)
+        print(f"refresh {bp}: sweep naive/no-offset/corrected {row['err_naive']:.4f} {row['err_no_offset']:.4f} "
+              f"{row['err_corrected']:.4f}; oracle {e_naive:.4f} {e_sel:.4f} {e_corr:.4f}")
+        assert row["rows"] == len(ref["rows"])
+        assert row["err_naive"] == pytest.approx(e_naive, rel=0.05)
+        assert row["err_no_offset"] == pytest.approx(e_sel, rel=0.05)
+        assert row["err_corrected"] == pytest.approx(e_corr, rel=0.05)
+        assert row["corrected_ms"] > 0 and row["full_ms"] > 0
+    assert rows[1]["err_corrected"] < rows[0]["err_corrected"] < e_naive * 1.05
+
+
+def test_bounded_device_wait_runs_out_and_reports_timeout():
+    import paper_2607_21604_b200 as akvs
+    ws = akvs.alloc_workspace(4096)
+    ws.zero_()
+    assert akvs.check(ws) == 0
+    akvs.debug_wait_timeout(ws, 2_000_000)          # about a millisecond of SM clock, nothing ever arrives
+    assert akvs.check(ws) == -6                     # AKVS_ERR_TIMEOUT; check() clears the word
+    assert akvs.check(ws) == 0
+    # the context is intact: an ordinary tensor-core call right after it
+    x = torch.randn(200, 256, device="cuda").half()
+    wt = torch.randn(384, 256, device="cuda").half()
+    y = akvs.op_linear(x, wt)
+    torch.cuda.synchronize()
+    ref = x.double() @ wt.double().T
+    assert float((y.double() - ref).norm() / ref.norm()) < 2e-3

@@ -236,3 +236,17 @@ def test_quantised_cache_path(setup, bits):
     # check layer 1 with a quantised cache: scores are the quantisation error, non-zero
     r = orc.corrected_reuse(model, quant, range(len(quant)), ctx, qry, 2500, 1)
     assert r["d_k"].min() > 0
+
+
+def test_threads_over_heads_change_nothing():
+    """ATTENTION_WORKERS only spreads the heads of one attention call over threads."""
+    g = np.random.default_rng(5)
+    q, k, v = g.standard_normal((9, 6, 8)), g.standard_normal((23, 2, 8)), g.standard_normal((23, 2, 8))
+    qpos = np.sort(g.choice(23, 9, replace=False))
+    a = orc.attention(q, k, v, qpos, np.arange(23))
+    orc.ATTENTION_WORKERS = 4
+    try:
+        b = orc.attention(q, k, v, qpos, np.arange(23))
+    finally:
+        orc.ATTENTION_WORKERS = 1
+    assert np.array_equal(a, b)
