@@ -468,6 +468,34 @@ def main():
             akvs.debug_correct_repeat(gmodel, store, req, probes, out_k, out_v, ps.ctx, ws)
         b2b_ms = timed(corr_only, 5, 2) / n_rep
         by = R_.other["correct_kernel"]["bytes_per_launch"]
+        # calibration: a plain device-to-device copy moving the same number of bytes (half read,
+        # half written), timed both ways over buffers cycled beyond the L2
+        n_el = int(by // 4)
+        srcs = [torch.empty(n_el, dtype=torch.float16, device="cuda").normal_() for _ in range(8)]
+        dsts = [torch.empty_like(t) for t in srcs]
+        for a_, b_ in zip(srcs, dsts):
+            b_.copy_(a_)
+        torch.cuda.synchronize()
+        singles = []
+        for rep in range(3):
+            for a_, b_ in zip(srcs, dsts):
+                x0, x1 = ev(), ev()
+                x0.record(); b_.copy_(a_); x1.record()
+                torch.cuda.synchronize()
+                singles.append(x0.elapsed_time(x1))
+        x0, x1 = ev(), ev()
+        x0.record()
+        for rep in range(3):
+            for a_, b_ in zip(srcs, dsts):
+                b_.copy_(a_)
+        x1.record()
+        torch.cuda.synchronize()
+        copy_b2b = x0.elapsed_time(x1) / 24
+        del srcs, dsts
+        R_.other["correct_kernel"]["copy_of_the_same_bytes"] = {
+            "what": "torch device-to-device copy of bytes_per_launch / 2, same two ways of timing",
+            "single_launch_us": 1e3 * float(np.median(singles)), "single_launch_frac": by / (float(np.median(singles)) * 1e-3) / 1e9 / pk["hbm"],
+            "back_to_back_us": 1e3 * copy_b2b, "back_to_back_frac": by / (copy_b2b * 1e-3) / 1e9 / pk["hbm"]}
         R_.other["correct_kernel"]["back_to_back"] = {
             "how": f"{n_rep} launches in a row over the layers' own cache and output buffers ({n_rep * by / 1e9:.2f} GB, "
                    "beyond the L2), one pair of events around them",

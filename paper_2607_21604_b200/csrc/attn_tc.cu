@@ -74,26 +74,9 @@ __device__ __forceinline__ float ex2(float x) {
   return y;
 }
 
-// Packed float pairs (one instruction for two lanes of arithmetic) and the 3-input maximum:
-// the softmax loop is bound by issue slots shared between two warps of a scheduler.
-__device__ __forceinline__ uint64_t pack_f32x2(float lo, float hi) {
-  uint64_t r;
-  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
-  return r;
-}
-__device__ __forceinline__ void unpack_f32x2(uint64_t v, float& lo, float& hi) {
-  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
-}
-__device__ __forceinline__ uint64_t fma_f32x2(uint64_t a, uint64_t b, uint64_t c) {
-  uint64_t r;
-  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
-  return r;
-}
-__device__ __forceinline__ uint64_t add_f32x2(uint64_t a, uint64_t b) {
-  uint64_t r;
-  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
-  return r;
-}
+// Packed float pairs (one instruction for two lanes of arithmetic, the sm_100 float2 builtins:
+// a pair stays in an aligned register pair, no moves around the instruction) and the 3-input
+// maximum: the softmax loop is bound by issue slots shared between two warps of a scheduler.
 __device__ __forceinline__ float max3(float a, float b, float c) {
   float r;
   asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
@@ -367,20 +350,16 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
           tc::tmem_st32(lane_addr + COL_O + c * 32, ob);
         }
       }
-      const uint64_t scale2 = pack_f32x2(p.scale_log2, p.scale_log2), shift2 = pack_f32x2(-m_new, -m_new);
-      uint64_t sum2[2] = {0ull, 0ull};                          // two packed pairs of partial sums
+      const float2 scale2 = make_float2(p.scale_log2, p.scale_log2), shift2 = make_float2(-m_new, -m_new);
+      float2 sum2[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};      // two packed pairs of partial sums
 #pragma unroll
       for (int i = 0; i < BN; i += 2) {
-        float x0, x1;
-        unpack_f32x2(fma_f32x2(pack_f32x2(t[i], t[i + 1]), scale2, shift2), x0, x1);
-        t[i] = ex2(x0);                                         // exp2(-inf) = 0 for masked keys
-        t[i + 1] = ex2(x1);
-        sum2[(i >> 1) & 1] = add_f32x2(sum2[(i >> 1) & 1], pack_f32x2(t[i], t[i + 1]));
+        const float2 x = __ffma2_rn(make_float2(t[i], t[i + 1]), scale2, shift2);
+        t[i] = ex2(x.x);                                        // exp2(-inf) = 0 for masked keys
+        t[i + 1] = ex2(x.y);
+        sum2[(i >> 1) & 1] = __fadd2_rn(sum2[(i >> 1) & 1], make_float2(t[i], t[i + 1]));
       }
-      float s0, s1, s2, s3;
-      unpack_f32x2(sum2[0], s0, s1);
-      unpack_f32x2(sum2[1], s2, s3);
-      l_mine += (s0 + s1) + (s2 + s3);
+      l_mine += (sum2[0].x + sum2[0].y) + (sum2[1].x + sum2[1].y);
       // two 16-bit probabilities per 32-bit column, packed before the wait below: only the two
       // stores stay on the chain P(j-1) ready -> P(j-1) V(j-1) -> P(j) stored
       uint32_t pk[64];

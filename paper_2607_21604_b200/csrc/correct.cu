@@ -392,7 +392,6 @@ offsets_kernel(KvLayer kv, ReqMaps maps, const int32_t* __restrict__ probe_off, 
   constexpr int V = VecOf<T>::N;
   extern __shared__ float part[];                 // [slots][hd]
   pdl_trigger();
-  pdl_wait();
   const int u = blockIdx.x, h = blockIdx.y, is_v = blockIdx.z;
   const int half = hd / 2, ch = half / V;
   const int slots = OFF_THREADS / ch;
@@ -410,21 +409,21 @@ offsets_kernel(KvLayer kv, ReqMaps maps, const int32_t* __restrict__ probe_off, 
   float acc_lo[V], acc_hi[V];
 #pragma unroll
   for (int i = 0; i < V; ++i) acc_lo[i] = acc_hi[i] = 0.f;
+  // First the reused half, -sum Rot(off_u) K_cached: the probe lists, the index maps, the
+  // rotation table and the unit cache are inputs no kernel of the layer writes, so this part
+  // runs while the projection GEMM before this kernel is still busy.  Then, once that GEMM has
+  // completed (griddepcontrol.wait), + sum of the fresh rows.
   if (slot < slots) {
     float2 rot[V];
     if (!is_v) ld_f2<V>(table + (size_t)maps.unit_pos[u] * half + c * V, rot);
     for (int i = slot; i < b; i += slots) {
       const int j = S[i];
       if (j < 0 || j >= N) { set_status(status, AKVS_ERR_INVALID_ARG); continue; }
-      const int row = maps.row_of_pos[j];
+      if (maps.row_of_pos[j] < 0) continue;         // inconsistent caller-supplied sets: skip
       const int64_t src = maps.tok_src[j];
-      if (row < 0) continue;                        // inconsistent caller-supplied sets: skip
-      float lo[V], hi[V], flo[V], fhi[V];
+      float lo[V], hi[V];
       load_cached_chunk<TW, FMT>(cbase, cmeta, src, n_kv, hd, h, c * V, lo);
       load_cached_chunk<TW, FMT>(cbase, cmeta, src, n_kv, hd, h, half + c * V, hi);
-      const T* fp = fresh + ((size_t)row * n_kv + h) * hd + c * V;
-      ld16(fp, flo);
-      ld16(fp + half, fhi);
 #pragma unroll
       for (int e = 0; e < V; ++e) {
         float rl = lo[e], rh = hi[e];
@@ -432,8 +431,26 @@ offsets_kernel(KvLayer kv, ReqMaps maps, const int32_t* __restrict__ probe_off, 
           rl = lo[e] * rot[e].x - hi[e] * rot[e].y;
           rh = hi[e] * rot[e].x + lo[e] * rot[e].y;
         }
-        acc_lo[e] += flo[e] - rl;
-        acc_hi[e] += fhi[e] - rh;
+        acc_lo[e] -= rl;
+        acc_hi[e] -= rh;
+      }
+    }
+  }
+  pdl_wait();
+  if (slot < slots) {
+    for (int i = slot; i < b; i += slots) {
+      const int j = S[i];
+      if (j < 0 || j >= N) continue;
+      const int row = maps.row_of_pos[j];
+      if (row < 0) continue;
+      float flo[V], fhi[V];
+      const T* fp = fresh + ((size_t)row * n_kv + h) * hd + c * V;
+      ld16(fp, flo);
+      ld16(fp + half, fhi);
+#pragma unroll
+      for (int e = 0; e < V; ++e) {
+        acc_lo[e] += flo[e];
+        acc_hi[e] += fhi[e];
       }
     }
 #pragma unroll
@@ -482,230 +499,301 @@ int32_t launch_offsets(int dtype, const KvLayer& kv, const ReqMaps& maps, const 
 //                              in S^K:      K_out = fresh K of its recomputed row
 //   V likewise with S^V (no rotation);  query token i: fresh K/V of row P + i.
 //
-// Work split: a token's K row and V row are two "role rows"; a thread owns ONE pair chunk (16
+// Work split.  A token's K row and V row are two "role rows".  A thread owns ONE pair chunk (16
 // bytes of the lower half of a head + its RoPE partner 16 bytes in the upper half) of one role
 // for the whole launch, so its rotation entries and the unit's offsets sit in registers and are
-// refetched only when the token's unit changes (units are runs of >= a hundred tokens).  The
-// threads of a role row read and write its heads as whole 128-byte lines.  A CTA takes a
-// contiguous slice of tokens, `tl` tokens side by side, COR_U tokens per thread and batch: the
-// thread first reads the batch's per-token records (one 16-byte load each, weight included),
-// then issues all 2 COR_U data loads, then decodes / rotates / adds w mu on packed float pairs
-// (fma.rn.f32x2: half the floating-point issue slots) and stores.  Fresh rows (probes, query)
-// are copied as the 16 bytes they are.  The grid is one wave: slices are sized so that every
-// CTA slot of the device gets one slice of the same length.
+// refetched only when the token's unit changes (units are runs of a hundred tokens and more).
+// A CTA takes a contiguous slice of tokens, `tl` of them side by side; the grid is one wave of
+// equal slices.
+//
+// Data movement.  The input is streamed through shared memory with per-thread asynchronous
+// copies (cp.async), COR_DEPTH tokens ahead, so the bytes in flight do not cost registers: the
+// `ch` threads that own a head's chunks (always lanes of one warp) copy that head's bytes of the
+// token's row - cached codes (+ the group records) or a fresh row - 16 bytes per thread and
+// copy, into their slot of the ring; cp.async.wait_group + __syncwarp hands the slot to its
+// owners, who decode, rotate and add w mu on packed float pairs (fma.rn.f32x2) and store 16-byte
+// vectors that neighbouring threads complete to whole 128-byte lines.  Fresh rows are copied as
+// the bytes they are.
+//
+// Overlap with the kernel before it.  The per-token records, the rotation table and the unit
+// cache are inputs that no kernel of the layer writes, so the slice's records and the first
+// COR_DEPTH tokens' CACHE bytes are requested BEFORE griddepcontrol.wait, while the offset kernel
+// (and the projection GEMM before it) still run; only the fresh rows and the offsets wait.
 // ---------------------------------------------------------------------------------------
-#ifndef AKVS_COR_U
-#define AKVS_COR_U 4
+#ifndef AKVS_COR_DEPTH
+#define AKVS_COR_DEPTH 4
 #endif
 #ifndef AKVS_COR_CTAS
-#define AKVS_COR_CTAS 2
+#define AKVS_COR_CTAS 3
 #endif
-constexpr int COR_THREADS = 256, COR_U = AKVS_COR_U, COR_CTAS_PER_SM = AKVS_COR_CTAS;
+constexpr int COR_THREADS = 256, COR_DEPTH = AKVS_COR_DEPTH, COR_CTAS_PER_SM = AKVS_COR_CTAS;
 
-__device__ __forceinline__ uint64_t pk2(float lo, float hi) {
-  uint64_t r;
-  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
-  return r;
-}
-__device__ __forceinline__ void upk2(uint64_t v, float& lo, float& hi) {
-  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
-}
-__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
-  uint64_t r;
-  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
-  return r;
-}
-__device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b) {
-  uint64_t r;
-  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
-  return r;
-}
+// Packed float pairs: the sm_100 float2 builtins (one FFMA2 / FMUL2 / FADD2 per two lanes of
+// arithmetic) keep a pair in an aligned register pair from the conversion to the pack, with no
+// moves in between.
+__device__ __forceinline__ float2 fma2(float2 a, float2 b, float2 c) { return __ffma2_rn(a, b, c); }
+__device__ __forceinline__ float2 mul2(float2 a, float2 b) { return __fmul2_rn(a, b); }
+__device__ __forceinline__ float2 add2(float2 a, float2 b) { return __fadd2_rn(a, b); }
+__device__ __forceinline__ uint32_t tc_smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
-template <typename TW, int FMT> struct RawChunk;
-template <typename TW> struct RawChunk<TW, AKVS_KV_NATIVE> { uint4 v; };
-template <typename TW> struct RawChunk<TW, AKVS_KV_Q4> { uint32_t packed; __half2 sm; };
-template <typename TW> struct RawChunk<TW, AKVS_KV_Q2> { uint32_t packed; __half2 sm; };
-template <typename TW> struct RawChunk<TW, AKVS_KV_FP8> { uint32_t w[2]; };
-
-__device__ __forceinline__ void unpack16(const uint4& r, float (&o)[4], const float*) {
-  o[0] = __uint_as_float(r.x); o[1] = __uint_as_float(r.y); o[2] = __uint_as_float(r.z); o[3] = __uint_as_float(r.w);
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gsrc) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gsrc)
+               : "memory");
 }
-__device__ __forceinline__ void unpack16(const uint4& r, float (&o)[8], const bf16*) {
+__device__ __forceinline__ void cp_async4(void* smem_dst, const void* gsrc) {
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gsrc)
+               : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+__device__ __forceinline__ void unpack16(const uint4& r, float2 (&o)[2], const float*) {
+  o[0] = make_float2(__uint_as_float(r.x), __uint_as_float(r.y));
+  o[1] = make_float2(__uint_as_float(r.z), __uint_as_float(r.w));
+}
+__device__ __forceinline__ void unpack16(const uint4& r, float2 (&o)[4], const bf16*) {
   const uint32_t w[4] = {r.x, r.y, r.z, r.w};
 #pragma unroll
-  for (int i = 0; i < 4; ++i) { o[2 * i] = __uint_as_float(w[i] << 16); o[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u); }
+  for (int i = 0; i < 4; ++i) o[i] = make_float2(__uint_as_float(w[i] << 16), __uint_as_float(w[i] & 0xFFFF0000u));
 }
-__device__ __forceinline__ void unpack16(const uint4& r, float (&o)[8], const f16*) {
+__device__ __forceinline__ void unpack16(const uint4& r, float2 (&o)[4], const f16*) {
   const uint32_t w[4] = {r.x, r.y, r.z, r.w};
 #pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&w[i]));
-    o[2 * i] = f.x; o[2 * i + 1] = f.y;
-  }
+  for (int i = 0; i < 4; ++i) o[i] = __half22float2(*reinterpret_cast<const __half2*>(&w[i]));
+}
+__device__ __forceinline__ uint4 pack16(const float2 (&o)[2], const float*) {
+  return make_uint4(__float_as_uint(o[0].x), __float_as_uint(o[0].y), __float_as_uint(o[1].x), __float_as_uint(o[1].y));
+}
+__device__ __forceinline__ uint4 pack16(const float2 (&o)[4], const bf16*) {
+  return make_uint4(pack_bf16x2(o[0].x, o[0].y), pack_bf16x2(o[1].x, o[1].y), pack_bf16x2(o[2].x, o[2].y),
+                    pack_bf16x2(o[3].x, o[3].y));
+}
+__device__ __forceinline__ uint4 pack16(const float2 (&o)[4], const f16*) {
+  return make_uint4(pack_f16x2(o[0].x, o[0].y), pack_f16x2(o[1].x, o[1].y), pack_f16x2(o[2].x, o[2].y),
+                    pack_f16x2(o[3].x, o[3].y));
 }
 
-// Issues the load of one chunk of the cache in its own format (V elements from element `e0` of
-// store row `src`): 16 bytes for a native cache, V bytes for FP8, V * bits / 8 bytes of codes and
-// the group's (scale, min) record for the group-quantised formats.
-template <typename T, typename TW, int FMT>
-__device__ __forceinline__ void issue_cached(const void* base, const void* meta, int64_t src, int row_elems, int hd,
-                                             int e0, RawChunk<TW, FMT>& raw) {
+__device__ __forceinline__ uint4 lds128(uint32_t a) {
+  uint4 v;
+  asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(a));
+  return v;
+}
+__device__ __forceinline__ uint2 lds64(uint32_t a) {
+  uint2 v;
+  asm volatile("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(a));
+  return v;
+}
+__device__ __forceinline__ uint32_t lds32(uint32_t a) {
+  uint32_t v;
+  asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(a));
+  return v;
+}
+__device__ __forceinline__ void cp_async16s(uint32_t dst, const void* gsrc) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(gsrc) : "memory");
+}
+__device__ __forceinline__ void cp_async4s(uint32_t dst, const void* gsrc) {
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst), "l"(gsrc) : "memory");
+}
+
+// V cached elements starting at element `e` of one head, from that head's bytes in shared memory
+// (shared-memory addresses; `codes`: the head's values or codes as they lie in the store; `recs`:
+// its (scale, min) records).
+template <typename T, int FMT>
+__device__ __forceinline__ void decode_head_chunk(uint32_t codes, uint32_t recs, int e, float2 (&out)[VecOf<T>::N / 2]) {
   constexpr int V = VecOf<T>::N;
-  const size_t e = (size_t)src * row_elems + e0;
   if constexpr (FMT == AKVS_KV_NATIVE) {
-    raw.v = *reinterpret_cast<const uint4*>(reinterpret_cast<const TW*>(base) + e);
+    unpack16(lds128(codes + e * (int)sizeof(T)), out, (const T*)nullptr);
   } else if constexpr (FMT == AKVS_KV_FP8) {
-    const uint8_t* cp = reinterpret_cast<const uint8_t*>(base) + e;
+    uint32_t w[2];
     if constexpr (V == 8) {
-      const uint2 t = *reinterpret_cast<const uint2*>(cp);
-      raw.w[0] = t.x; raw.w[1] = t.y;
+      const uint2 t = lds64(codes + e);
+      w[0] = t.x; w[1] = t.y;
     } else {
-      raw.w[0] = *reinterpret_cast<const uint32_t*>(cp);
+      w[0] = lds32(codes + e);
     }
-  } else {
-    constexpr int BYTES = V * FMT / 8;
-    raw.packed = ld_codes<BYTES>(reinterpret_cast<const uint8_t*>(base) + e * FMT / 8);
-    raw.sm = reinterpret_cast<const __half2*>(meta)[e / 64];          // hd is a multiple of 64: groups do not straddle heads
-  }
-}
-template <typename T, typename TW, int FMT>
-__device__ __forceinline__ void decode_cached(const RawChunk<TW, FMT>& raw, float (&out)[VecOf<T>::N]) {
-  constexpr int V = VecOf<T>::N;
-  if constexpr (FMT == AKVS_KV_NATIVE) {
-    unpack16(raw.v, out, (const TW*)nullptr);
-  } else if constexpr (FMT == AKVS_KV_FP8) {
 #pragma unroll
     for (int i = 0; i < V / 2; ++i) {
-      const __half2_raw h = __nv_cvt_fp8x2_to_halfraw2((__nv_fp8x2_storage_t)((raw.w[i >> 1] >> (16 * (i & 1))) & 0xFFFFu), __NV_E4M3);
-      const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&h));
-      out[2 * i] = f.x; out[2 * i + 1] = f.y;
+      const __half2_raw h = __nv_cvt_fp8x2_to_halfraw2((__nv_fp8x2_storage_t)((w[i >> 1] >> (16 * (i & 1))) & 0xFFFFu), __NV_E4M3);
+      out[i] = __half22float2(*reinterpret_cast<const __half2*>(&h));
     }
   } else {
-    const float s = __low2float(raw.sm), mn = __high2float(raw.sm);
+    constexpr int BYTES = V * FMT / 8;                   // 4, 2 or 1 bytes of codes
+    const int byte0 = e * FMT / 8;
+    const uint32_t word = lds32(codes + (byte0 & ~3));
+    const uint32_t packed = BYTES == 4 ? word : (word >> (8 * (byte0 & 3))) & ((1u << (8 * BYTES)) - 1u);
+    const uint32_t rec = lds32(recs + (e / 64) * 4);
+    const __half2 sm = *reinterpret_cast<const __half2*>(&rec);
+    const float s = __low2float(sm), mn = __high2float(sm);
 #pragma unroll
-    for (int i = 0; i < V; ++i) out[i] = __fmaf_rn((float)((raw.packed >> (FMT * i)) & ((1u << FMT) - 1u)), s, mn);
+    for (int i = 0; i < V / 2; ++i)
+      out[i] = make_float2(__fmaf_rn((float)((packed >> (FMT * 2 * i)) & ((1u << FMT) - 1u)), s, mn),
+                           __fmaf_rn((float)((packed >> (FMT * (2 * i + 1))) & ((1u << FMT) - 1u)), s, mn));
   }
 }
 
-template <typename T, typename TW, int FMT>
+template <typename T, int FMT>
 __global__ void __launch_bounds__(COR_THREADS, COR_CTAS_PER_SM)
 correct_kernel(KvLayer kv, const int4* __restrict__ tok_meta, const int32_t* __restrict__ unit_pos,
                const T* __restrict__ k_fresh, const T* __restrict__ v_fresh, const float* __restrict__ mu_k,
-               const float* __restrict__ mu_v, int T_tok, int n_kv, int hd, int ipt, int tl, int slice, int weighted,
-               const float2* __restrict__ table, T* __restrict__ out_k, T* __restrict__ out_v) {
-  // ipt = pair chunks of the kv heads this CTA column (blockIdx.y) covers: heads_per_cta * chunks per head
+               const float* __restrict__ mu_v, int T_tok, int n_kv, int hd, int ipt, int tl, int slice, int slot_bytes,
+               int weighted, const float2* __restrict__ table, T* __restrict__ out_k, T* __restrict__ out_v) {
+  // ipt = pair chunks of the kv heads this CTA column (blockIdx.y) covers: heads per CTA x chunks per head
   constexpr int V = VecOf<T>::N;
+  constexpr int ES = (int)sizeof(T);
+  constexpr int CODE_BITS = FMT == AKVS_KV_NATIVE ? 8 * ES : FMT;      // bits per cached element
+  extern __shared__ __align__(16) uint8_t cor_smem[];
+  int4* meta_s = reinterpret_cast<int4*>(cor_smem);                    // [2][slice] the slice's records
   pdl_trigger();
-  pdl_wait();
+  const int t0 = blockIdx.x * slice;
+  const int n_slice = min(T_tok, t0 + slice) - t0;
+  for (int i = threadIdx.x; i < 2 * n_slice; i += COR_THREADS) {
+    const int r = i >= n_slice, jl = i - r * n_slice;
+    meta_s[r * slice + jl] = tok_meta[(size_t)r * T_tok + t0 + jl];
+  }
+  __syncthreads();
+
+  const int half = hd / 2, ch = half / V;
   const int tpt = 2 * ipt;                              // threads per token: K items, then V items
   const int lane_tok = threadIdx.x / tpt;
-  if (lane_tok >= tl) return;
   const int rem = threadIdx.x - lane_tok * tpt;
   const int role = rem / ipt;                           // 0: K, 1: V
   const int item = rem - role * ipt;
-  const int half = hd / 2, ch = half / V;
   const int h = blockIdx.y * (ipt / ch) + item / ch, c = item % ch;
-  if (h >= n_kv) return;                                // the last head group may be short
-  const int row_elems = n_kv * hd;
-  const int col = h * hd + c * V;                       // element of the lower chunk within a role row
-  const int4* __restrict__ meta = tok_meta + (size_t)role * T_tok;
-  const T* __restrict__ fresh = role ? v_fresh : k_fresh;
-  const void* cbase = role ? kv.v : kv.k;
-  const void* cmeta = role ? kv.v_meta : kv.k_meta;
-  const float* __restrict__ mu = role ? mu_v : mu_k;
-  T* __restrict__ out = role ? out_v : out_k;
-  const int t_end = min(T_tok, (blockIdx.x + 1) * slice);
+  const bool active = lane_tok < tl && h < n_kv;        // idle lanes still take part in the warp syncs
+  const int n_q = (n_slice + tl - 1) / tl;              // steps of the CTA (the same for every thread)
+  const int n_mine = active ? (n_slice - lane_tok + tl - 1) / tl : 0;   // tokens of this thread
+  // shared-memory addresses: this role's records; the slot of this thread's head in ring stage 0
+  const uint32_t meta_a = tc_smem_u32(meta_s) + (uint32_t)(role * slice + lane_tok) * 16u;
+  const uint32_t meta_step = (uint32_t)tl * 16u;
+  const uint32_t ring0 = tc_smem_u32(cor_smem) + (uint32_t)(2 * slice) * 16u + (uint32_t)(threadIdx.x / ch) * slot_bytes;
+  const uint32_t ring_stride = (uint32_t)(COR_THREADS / ch) * slot_bytes;
+  const uint32_t ring_end = ring0 + COR_DEPTH * ring_stride;
+  // global bases of this thread's pieces
+  const int head_code_bytes = hd * CODE_BITS / 8;
+  const size_t cache_row_bytes = (size_t)n_kv * head_code_bytes;
+  const size_t fresh_row_bytes = (size_t)n_kv * hd * ES;
+  const uint8_t* cache_p = reinterpret_cast<const uint8_t*>(role ? kv.v : kv.k) + (size_t)h * head_code_bytes + c * 16;
+  const uint8_t* rec_p = reinterpret_cast<const uint8_t*>(role ? kv.v_meta : kv.k_meta) + (size_t)h * (hd / 64) * 4 + c * 4;
+  const size_t rec_row_bytes = (size_t)n_kv * (hd / 64) * 4;
+  const uint8_t* fresh_p = reinterpret_cast<const uint8_t*>(role ? v_fresh : k_fresh) + (size_t)h * hd * ES + c * 16;
+  uint8_t* out_p = reinterpret_cast<uint8_t*>(role ? out_v : out_k) + ((size_t)(t0 + lane_tok) * n_kv + h) * hd * ES + c * 16;
+  const size_t out_step = (size_t)tl * fresh_row_bytes;
+  const float* __restrict__ mu = (role ? mu_v : mu_k) + (size_t)h * hd + c * V;
+  const uint32_t hi_off = (uint32_t)ch * 16u;           // byte distance of the upper chunk (fresh rows, native cache)
+  const bool copy_codes = c * 16 < head_code_bytes;      // quantised formats: fewer 16-byte pieces than lanes
+  const bool copy_rec = c < hd / 64;
 
-  uint64_t C2[V / 2], S2[V / 2], ML2[V / 2], MH2[V / 2];   // (cos, cos), (sin, sin), offsets of the lower / upper chunk
-  int cur_unit = -1;
-  for (int b0 = blockIdx.x * slice + lane_tok; b0 < t_end; b0 += tl * COR_U) {
-    int4 mt[COR_U];
-#pragma unroll
-    for (int u = 0; u < COR_U; ++u) {
-      const int j = b0 + u * tl;
-      mt[u] = j < t_end ? meta[j] : make_int4(-1, -1, 0, 0);
-    }
-    // ---- all data loads of the batch (a native cache of the model's type shares the registers
-    // of the fresh rows: one pointer select, one pair of loads)
-    constexpr bool kShared = FMT == AKVS_KV_NATIVE && std::is_same<T, TW>::value;
-    uint4 f_lo[COR_U], f_hi[COR_U];
-    RawChunk<TW, FMT> c_lo[kShared ? 1 : COR_U], c_hi[kShared ? 1 : COR_U];
-#pragma unroll
-    for (int u = 0; u < COR_U; ++u) {
-      if (b0 + u * tl >= t_end) continue;
-      if (kShared || mt[u].y >= 0) {
-        const T* fp = mt[u].y >= 0 ? fresh + (size_t)mt[u].y * row_elems + col
-                                   : reinterpret_cast<const T*>(cbase) + (size_t)mt[u].x * row_elems + col;
-        f_lo[u] = *reinterpret_cast<const uint4*>(fp);
-        f_hi[u] = *reinterpret_cast<const uint4*>(fp + half);
+  // Requests the bytes of local token q into ring stage `dst` (WHICH: 1 = cached rows only,
+  // 2 = fresh rows only, 3 = either).  No-op past the slice.
+  auto issue = [&](int q, uint32_t dst, auto which) {
+    constexpr int WHICH = decltype(which)::value;
+    if (q >= n_mine) return;
+    const uint4 m = lds128(meta_a + (uint32_t)q * meta_step);
+    if ((int)m.y >= 0) {
+      if (WHICH & 2) {
+        const uint8_t* src = fresh_p + (size_t)m.y * fresh_row_bytes;
+        cp_async16s(dst + c * 16, src);
+        cp_async16s(dst + c * 16 + hi_off, src + hi_off);
+      }
+    } else if (WHICH & 1) {
+      if constexpr (FMT == AKVS_KV_NATIVE) {
+        const uint8_t* src = cache_p + (size_t)m.x * cache_row_bytes;
+        cp_async16s(dst + c * 16, src);
+        cp_async16s(dst + c * 16 + hi_off, src + hi_off);
       } else {
-        issue_cached<T, TW, FMT>(cbase, cmeta, mt[u].x, row_elems, hd, col, c_lo[kShared ? 0 : u]);
-        issue_cached<T, TW, FMT>(cbase, cmeta, mt[u].x, row_elems, hd, col + half, c_hi[kShared ? 0 : u]);
+        if (copy_codes) cp_async16s(dst + c * 16, cache_p + (size_t)m.x * cache_row_bytes);
+        if constexpr (FMT == AKVS_KV_Q4 || FMT == AKVS_KV_Q2)
+          if (copy_rec) cp_async4s(dst + head_code_bytes + c * 4, rec_p + (size_t)m.x * rec_row_bytes);
       }
     }
-    // ---- decode, re-align, correct, store
+  };
+  using W1 = std::integral_constant<int, 1>;
+  using W2_ = std::integral_constant<int, 2>;
+  using W3 = std::integral_constant<int, 3>;
+
 #pragma unroll
-    for (int u = 0; u < COR_U; ++u) {
-      const int j = b0 + u * tl;
-      if (j >= t_end) continue;
-      T* op = out + (size_t)j * row_elems + col;
-      if (mt[u].y >= 0) {                               // a fresh row: the bytes as they are
-        *reinterpret_cast<uint4*>(op) = f_lo[u];
-        *reinterpret_cast<uint4*>(op + half) = f_hi[u];
-        continue;
-      }
-      if (mt[u].z != cur_unit) {
-        cur_unit = mt[u].z;
-        if (role == 0) {
-          float2 rot[V];
-          ld_f2<V>(table + (size_t)unit_pos[cur_unit] * half + c * V, rot);
+  for (int q = 0; q < COR_DEPTH; ++q) {
+    issue(q, ring0 + q * ring_stride, W1{});
+    cp_async_commit();
+  }
+  pdl_wait();                                           // fresh rows and offsets are other kernels' outputs
 #pragma unroll
-          for (int i = 0; i < V / 2; ++i) {
-            C2[i] = pk2(rot[2 * i].x, rot[2 * i + 1].x);
-            S2[i] = pk2(rot[2 * i].y, rot[2 * i + 1].y);
+  for (int q = 0; q < COR_DEPTH; ++q) {
+    issue(q, ring0 + q * ring_stride, W2_{});
+    cp_async_commit();
+  }
+
+  float2 C2[V / 2], NS2[V / 2], ML2[V / 2], MH2[V / 2];   // (cos, cos), (-sin, -sin), offsets of the lower / upper chunk
+  int cur_unit = -1;
+  uint32_t slot = ring0;
+  for (int q = 0; q < n_q; ++q) {
+    cp_async_wait<COR_DEPTH - 1>();                     // everything up to this token's copies has landed
+    __syncwarp();                                       // ... for every lane of the head's group
+    if (q < n_mine) {
+      const uint4 m = lds128(meta_a + (uint32_t)q * meta_step);
+      if ((int)m.y >= 0) {                              // a fresh row: the bytes as they are
+        *reinterpret_cast<uint4*>(out_p) = lds128(slot + c * 16);
+        *reinterpret_cast<uint4*>(out_p + hi_off) = lds128(slot + c * 16 + hi_off);
+      } else {
+        if ((int)m.z != cur_unit) {
+          cur_unit = (int)m.z;
+          if (role == 0) {
+            float2 rot[V];
+            ld_f2<V>(table + (size_t)unit_pos[cur_unit] * half + c * V, rot);
+#pragma unroll
+            for (int i = 0; i < V / 2; ++i) {
+              C2[i] = make_float2(rot[2 * i].x, rot[2 * i + 1].x);
+              NS2[i] = make_float2(-rot[2 * i].y, -rot[2 * i + 1].y);
+            }
+          }
+          if (weighted) {
+            float ml[V], mh[V];
+            const float* mp = mu + (size_t)cur_unit * n_kv * hd;
+            ld_f<V>(mp, ml);
+            ld_f<V>(mp + half, mh);
+#pragma unroll
+            for (int i = 0; i < V / 2; ++i) {
+              ML2[i] = make_float2(ml[2 * i], ml[2 * i + 1]);
+              MH2[i] = make_float2(mh[2 * i], mh[2 * i + 1]);
+            }
+          } else {
+#pragma unroll
+            for (int i = 0; i < V / 2; ++i) ML2[i] = MH2[i] = make_float2(0.f, 0.f);
           }
         }
-        if (weighted) {
-          float ml[V], mh[V];
-          const float* mp = mu + (size_t)cur_unit * row_elems + col;
-          ld_f<V>(mp, ml);
-          ld_f<V>(mp + half, mh);
-#pragma unroll
-          for (int i = 0; i < V / 2; ++i) { ML2[i] = pk2(ml[2 * i], ml[2 * i + 1]); MH2[i] = pk2(mh[2 * i], mh[2 * i + 1]); }
-        } else {
-#pragma unroll
-          for (int i = 0; i < V / 2; ++i) ML2[i] = MH2[i] = 0ull;
-        }
-      }
-      float lo[V], hi[V];
-      if constexpr (kShared) {
-        unpack16(f_lo[u], lo, (const T*)nullptr);
-        unpack16(f_hi[u], hi, (const T*)nullptr);
-      } else {
-        decode_cached<T, TW, FMT>(c_lo[u], lo);
-        decode_cached<T, TW, FMT>(c_hi[u], hi);
-      }
-      const float w = __int_as_float(mt[u].w);
-      const uint64_t W2 = pk2(w, w);
-#pragma unroll
-      for (int i = 0; i < V / 2; ++i) {
-        const uint64_t A2 = pk2(lo[2 * i], lo[2 * i + 1]), B2 = pk2(hi[2 * i], hi[2 * i + 1]);
-        uint64_t rl, rh;
+        float2 lo[V / 2], hi[V / 2];
+        decode_head_chunk<T, FMT>(slot, slot + head_code_bytes, c * V, lo);
+        decode_head_chunk<T, FMT>(slot, slot + head_code_bytes, half + c * V, hi);
+        const float w = __uint_as_float(m.w);
+        const float2 W2 = make_float2(w, w);
         if (role == 0) {
-          // lo' = a cos - b sin + w mu_lo,  hi' = b cos + a sin + w mu_hi
-          const uint64_t nb = B2 ^ 0x8000000080000000ull;               // (-b, -b): sign bits
-          rl = fma2(nb, S2[i], fma2(W2, ML2[i], mul2(A2, C2[i])));
-          rh = fma2(A2, S2[i], fma2(W2, MH2[i], mul2(B2, C2[i])));
+          // lo' = a cos - b sin + w mu_lo,  hi' = b cos + a sin + w mu_hi   (NS2 = -sin)
+#pragma unroll
+          for (int i = 0; i < V / 2; ++i) {
+            const float2 a2 = lo[i], b2 = hi[i];
+            lo[i] = fma2(b2, NS2[i], fma2(W2, ML2[i], mul2(a2, C2[i])));
+            const float2 t = fma2(W2, MH2[i], mul2(b2, C2[i]));
+            const float2 u = mul2(a2, NS2[i]);
+            hi[i] = add2(t, make_float2(-u.x, -u.y));
+          }
         } else {
-          rl = fma2(W2, ML2[i], A2);
-          rh = fma2(W2, MH2[i], B2);
+#pragma unroll
+          for (int i = 0; i < V / 2; ++i) {
+            lo[i] = fma2(W2, ML2[i], lo[i]);
+            hi[i] = fma2(W2, MH2[i], hi[i]);
+          }
         }
-        upk2(rl, lo[2 * i], lo[2 * i + 1]);
-        upk2(rh, hi[2 * i], hi[2 * i + 1]);
+        *reinterpret_cast<uint4*>(out_p) = pack16(lo, (const T*)nullptr);
+        *reinterpret_cast<uint4*>(out_p + hi_off) = pack16(hi, (const T*)nullptr);
       }
-      st16(op, lo);
-      st16(op + half, hi);
     }
+    out_p += out_step;
+    __syncwarp();                                       // the group is done with the stage before it is refilled
+    if (q + COR_DEPTH < n_mine) issue(q + COR_DEPTH, slot, W3{});
+    cp_async_commit();                                  // one group per step keeps the wait count constant
+    slot += ring_stride;
+    if (slot == ring_end) slot = ring0;
   }
 }
 
@@ -718,12 +806,13 @@ int32_t launch_correct(int dtype, const KvLayer& kv, const ReqMaps& maps, const 
   if (T_tok == 0) return AKVS_OK;
   AKVS_TRY(check_kv_shape(dtype, kv, hd));
   const int V = dtype == AKVS_F32 ? 4 : 8;
+  const int es = (int)dtype_size(dtype);
   const int ch = hd / 2 / V;                            // pair chunks of one head
-  if (2 * ch > COR_THREADS) return AKVS_ERR_UNSUPPORTED;
+  if (ch > 32 || (ch & (ch - 1)) != 0) return AKVS_ERR_UNSUPPORTED;   // a head's chunk owners are lanes of one warp
   const int heads_per_cta = n_kv < COR_THREADS / (2 * ch) ? n_kv : COR_THREADS / (2 * ch);
   const int head_groups = (n_kv + heads_per_cta - 1) / heads_per_cta;
   const int ipt = heads_per_cta * ch;                   // pair chunks of one role row within a head group
-  if ((int64_t)T_tok * n_kv * hd >= (1ll << 31)) return AKVS_ERR_SHAPE;     // 32-bit element offsets inside a layer
+  if ((int64_t)T_tok * n_kv * hd >= (1ll << 31)) return AKVS_ERR_SHAPE;
   if (!g_cor_slots) {
     int dev = 0, sms = 0;
     cudaGetDevice(&dev);
@@ -735,19 +824,31 @@ int32_t launch_correct(int dtype, const KvLayer& kv, const ReqMaps& maps, const 
   int slice = (T_tok + slots - 1) / slots;              // one wave of equal slices
   slice = (slice + tl - 1) / tl * tl;
   const int grid = (T_tok + slice - 1) / slice;
+  // bytes of one head in the ring: a fresh row's head, or the cached head and its records
+  const int code_bits = kv.fmt == AKVS_KV_NATIVE ? 8 * es : kv.fmt;
+  int slot_bytes = hd * code_bits / 8 + ((kv.fmt == AKVS_KV_Q4 || kv.fmt == AKVS_KV_Q2) ? (hd / 64) * 4 : 0);
+  if (slot_bytes < hd * es) slot_bytes = hd * es;
+  slot_bytes = (slot_bytes + 15) / 16 * 16;
+  const size_t smem = (size_t)2 * slice * sizeof(int4) + (size_t)COR_DEPTH * (COR_THREADS / ch) * slot_bytes;
+  if (smem > 200 * 1024) return AKVS_ERR_TOO_LARGE;
   // algorithmic bytes: every context K and V element read once in its cache format and
   // written once; fresh rows and query rows copied; 8 bytes of weights per context token
-  const double in_b = kv.fmt == AKVS_KV_NATIVE ? (double)dtype_size(dtype)
-                      : kv.fmt == AKVS_KV_FP8  ? 1.0 : kv.fmt / 8.0 + 4.0 / 64.0;
-  const double out_b = (double)dtype_size(dtype);
+  const double in_b = kv.fmt == AKVS_KV_NATIVE ? (double)es : kv.fmt == AKVS_KV_FP8 ? 1.0 : kv.fmt / 8.0 + 4.0 / 64.0;
+  const double out_b = (double)es;
   const double bytes = 2.0 * n_kv * hd * ((double)N * (in_b + out_b) + (double)n_query * 2 * out_b) + 8.0 * N;
   ProfScope prof(2, kv.fmt, bytes, st);
   return dispatch_dtype(dtype, [&](auto tag) -> int32_t {
     using T = decltype(tag);
     return dispatch_fmt(kv.fmt, [&](auto f) -> int32_t {
-      AKVS_CUDA(launch_pdl(correct_kernel<T, T, decltype(f)::value>, dim3(grid, head_groups), dim3(COR_THREADS), 0, st, kv,
-                           maps.tok_meta, maps.unit_pos, (const T*)k_fresh, (const T*)v_fresh, mu_k, mu_v, T_tok, n_kv,
-                           hd, ipt, tl, slice, weighted ? 1 : 0, table, (T*)out_k, (T*)out_v));
+      auto kern = correct_kernel<T, decltype(f)::value>;
+      static size_t smem_allowed = 48 * 1024;          // per instantiation: raised when a launch needs more
+      if (smem > smem_allowed) {
+        AKVS_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        smem_allowed = smem;
+      }
+      AKVS_CUDA(launch_pdl(kern, dim3(grid, head_groups), dim3(COR_THREADS), smem, st, kv, maps.tok_meta, maps.unit_pos,
+                           (const T*)k_fresh, (const T*)v_fresh, mu_k, mu_v, T_tok, n_kv, hd, ipt, tl, slice, slot_bytes,
+                           weighted ? 1 : 0, table, (T*)out_k, (T*)out_v));
       AKVS_LAUNCHED();
       return AKVS_OK;
     });

@@ -18,6 +18,8 @@
 // (one B block per tile, `nh` = 1); every other launch of more than 128 rows runs on CTA pairs
 // with 256x256 tiles (gemm_tc_pair_kernel below, tcgen05.mma.cta_group::2).  The kernels are launched as
 // programmatic dependents: set-up and the first weight tiles overlap the tail of the kernel before.
+#include <unordered_map>
+
 #include "tc_common.cuh"
 
 namespace {
@@ -635,11 +637,39 @@ int pair_count() {
 
 }  // namespace
 
+// A tensor map is a pure function of (base, rows, cols, ld, box): the maps of the weights and of
+// the workspace's activation buffers recur on every layer call of every step, so they are
+// encoded once per process and looked up afterwards (a few hundred driver calls per step
+// otherwise).  Process-wide and, like the rest of the library's host state, not thread-safe.
+namespace {
+struct TmapKey {
+  const void* base; uint64_t rows, cols, ld; uint32_t box;
+  bool operator==(const TmapKey& o) const { return base == o.base && rows == o.rows && cols == o.cols && ld == o.ld && box == o.box; }
+};
+struct TmapKeyHash {
+  size_t operator()(const TmapKey& k) const {
+    uint64_t h = reinterpret_cast<uintptr_t>(k.base) * 0x9E3779B97F4A7C15ull;
+    h ^= (k.rows + 0x9E3779B97F4A7C15ull + (h << 6) + (h >> 2));
+    h ^= (k.cols * 0xC2B2AE3D27D4EB4Full + (h << 6) + (h >> 2));
+    h ^= (k.ld * 31 + k.box + (h << 6) + (h >> 2));
+    return (size_t)h;
+  }
+};
+std::unordered_map<TmapKey, CUtensorMap, TmapKeyHash> g_tmap_cache;
+constexpr size_t kTmapCacheMax = 16384;
+}  // namespace
+
 int32_t encode_tmap_2d_16bit(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, uint64_t ld,
                             uint32_t box_rows) {
   EncodeFn enc = get_encoder();
   if (!enc) return AKVS_ERR_CUDA;
   if ((reinterpret_cast<uintptr_t>(base) & 15) || (ld * 2) % 16 != 0) return AKVS_ERR_SHAPE;
+  const TmapKey key{base, rows, cols, ld, box_rows};
+  auto it = g_tmap_cache.find(key);
+  if (it != g_tmap_cache.end()) {
+    *map = it->second;
+    return AKVS_OK;
+  }
   const cuuint64_t dims[2] = {cols, rows};
   const cuuint64_t strides[1] = {ld * 2};
   const cuuint32_t box[2] = {64, box_rows};
@@ -647,7 +677,10 @@ int32_t encode_tmap_2d_16bit(CUtensorMap* map, const void* base, uint64_t rows, 
   const CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_UINT16, 2, const_cast<void*>(base), dims, strides, box, estr,
                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  return r == CUDA_SUCCESS ? AKVS_OK : AKVS_ERR_CUDA;
+  if (r != CUDA_SUCCESS) return AKVS_ERR_CUDA;
+  if (g_tmap_cache.size() >= kTmapCacheMax) g_tmap_cache.clear();
+  g_tmap_cache.emplace(key, *map);
+  return AKVS_OK;
 }
 
 int32_t encode_tmap_3d_16bit(CUtensorMap* map, const void* base, uint64_t d0, uint64_t d1, uint64_t d2, uint64_t ld1,
