@@ -625,10 +625,15 @@ __device__ __forceinline__ void decode_head_chunk(uint32_t codes, uint32_t recs,
     const uint32_t rec = lds32(recs + (e / 64) * 4);
     const __half2 sm = *reinterpret_cast<const __half2*>(&rec);
     const float s = __low2float(sm), mn = __high2float(sm);
+    const float2 s2 = make_float2(s, s), mn2 = make_float2(mn, mn), bias2 = make_float2(-8388608.f, -8388608.f);
+    // code -> float without the integer-to-float unit: 2^23 + code as a bit pattern, minus 2^23
+    // (exact), then the same single-rounding fma(code, scale, min) as everywhere else
 #pragma unroll
-    for (int i = 0; i < V / 2; ++i)
-      out[i] = make_float2(__fmaf_rn((float)((packed >> (FMT * 2 * i)) & ((1u << FMT) - 1u)), s, mn),
-                           __fmaf_rn((float)((packed >> (FMT * (2 * i + 1))) & ((1u << FMT) - 1u)), s, mn));
+    for (int i = 0; i < V / 2; ++i) {
+      const uint32_t u0 = ((packed >> (FMT * 2 * i)) & ((1u << FMT) - 1u)) | 0x4B000000u;
+      const uint32_t u1 = ((packed >> (FMT * (2 * i + 1))) & ((1u << FMT) - 1u)) | 0x4B000000u;
+      out[i] = __ffma2_rn(__fadd2_rn(make_float2(__uint_as_float(u0), __uint_as_float(u1)), bias2), s2, mn2);
+    }
   }
 }
 
