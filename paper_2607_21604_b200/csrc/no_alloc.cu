@@ -22,6 +22,10 @@ constexpr size_t kScratchBytes = kStatusBytes + kKeysBytes + kFlagsBytes;
 // calls; the device address is obtained with cudaGetSymbolAddress, per device.
 static __device__ __align__(256) unsigned char g_select_scratch[kScratchBytes];
 
+// One resolved address per device ordinal.  Written without synchronisation: like the rest of
+// the library's host state it relies on the convention that one host thread drives one device
+// per process.  An address stays valid for the life of the process's context on that device;
+// after a cudaDeviceReset the library must not be used any further (its module state is gone).
 constexpr int kMaxDevices = 64;
 void* g_scratch_ptr[kMaxDevices] = {};
 
