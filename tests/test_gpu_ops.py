@@ -340,6 +340,15 @@ def test_correct_layer_small_ragged(akvs, dtype_t, kv_format, hd):
     _correct_case(akvs, dtype_t, kv_format, 2, 20, 30, 2, hd, 3, 10000, seed=2)   # everything is a probe
 
 
+@pytest.mark.parametrize("dtype_t,kv_format,hd,nkv", [(torch.float16, 0, 128, 20), (torch.float32, 0, 128, 9),
+                                                      (torch.bfloat16, 4, 64, 35), (torch.float16, 8, 128, 17),
+                                                      (torch.float16, 2, 128, 3)])
+def test_correct_layer_many_kv_heads(akvs, dtype_t, kv_format, hd, nkv):
+    """More kv heads than one CTA row of the correction kernel covers (16 heads of 128 in a 16-bit
+    type): the heads are split over blockIdx.y and the last group is short; odd head counts."""
+    _correct_case(akvs, dtype_t, kv_format, 4, 5, 23, nkv, hd, 5, 3000, seed=5)
+
+
 @pytest.mark.parametrize("kv_format", [0, 4, 2, 8])
 def test_correct_layer_full_size(akvs, kv_format):
     """One layer at the 8B-class shapes (8 kv heads x 128, ~8k / ~12k context tokens)."""
