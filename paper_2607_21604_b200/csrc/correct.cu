@@ -676,14 +676,14 @@ correct_kernel(KvLayer kv, const int4* __restrict__ tok_meta, const int32_t* __r
   const uint32_t ring_end = ring0 + COR_DEPTH * ring_stride;
   // global bases of this thread's pieces
   const int head_code_bytes = hd * CODE_BITS / 8;
-  const size_t cache_row_bytes = (size_t)n_kv * head_code_bytes;
-  const size_t fresh_row_bytes = (size_t)n_kv * hd * ES;
+  const uint32_t cache_row_bytes = (uint32_t)(n_kv * head_code_bytes);   // 32-bit sizes: one widening multiply per address
+  const uint32_t fresh_row_bytes = (uint32_t)(n_kv * hd * ES);
   const uint8_t* cache_p = reinterpret_cast<const uint8_t*>(role ? kv.v : kv.k) + (size_t)h * head_code_bytes + c * 16;
   const uint8_t* rec_p = reinterpret_cast<const uint8_t*>(role ? kv.v_meta : kv.k_meta) + (size_t)h * (hd / 64) * 4 + c * 4;
-  const size_t rec_row_bytes = (size_t)n_kv * (hd / 64) * 4;
+  const uint32_t rec_row_bytes = (uint32_t)(n_kv * (hd / 64) * 4);
   const uint8_t* fresh_p = reinterpret_cast<const uint8_t*>(role ? v_fresh : k_fresh) + (size_t)h * hd * ES + c * 16;
   uint8_t* out_p = reinterpret_cast<uint8_t*>(role ? out_v : out_k) + ((size_t)(t0 + lane_tok) * n_kv + h) * hd * ES + c * 16;
-  const size_t out_step = (size_t)tl * fresh_row_bytes;
+  const uint32_t out_step = (uint32_t)tl * fresh_row_bytes;
   const float* __restrict__ mu = (role ? mu_v : mu_k) + (size_t)h * hd + c * V;
   const uint32_t hi_off = (uint32_t)ch * 16u;           // byte distance of the upper chunk (fresh rows, native cache)
   const bool copy_codes = c * 16 < head_code_bytes;      // quantised formats: fewer 16-byte pieces than lanes
@@ -697,19 +697,19 @@ correct_kernel(KvLayer kv, const int4* __restrict__ tok_meta, const int32_t* __r
     const uint4 m = lds128(meta_a + (uint32_t)q * meta_step);
     if ((int)m.y >= 0) {
       if (WHICH & 2) {
-        const uint8_t* src = fresh_p + (size_t)m.y * fresh_row_bytes;
+        const uint8_t* src = fresh_p + (uint64_t)m.y * fresh_row_bytes;
         cp_async16s(dst + c * 16, src);
         cp_async16s(dst + c * 16 + hi_off, src + hi_off);
       }
     } else if (WHICH & 1) {
       if constexpr (FMT == AKVS_KV_NATIVE) {
-        const uint8_t* src = cache_p + (size_t)m.x * cache_row_bytes;
+        const uint8_t* src = cache_p + (uint64_t)m.x * cache_row_bytes;
         cp_async16s(dst + c * 16, src);
         cp_async16s(dst + c * 16 + hi_off, src + hi_off);
       } else {
-        if (copy_codes) cp_async16s(dst + c * 16, cache_p + (size_t)m.x * cache_row_bytes);
+        if (copy_codes) cp_async16s(dst + c * 16, cache_p + (uint64_t)m.x * cache_row_bytes);
         if constexpr (FMT == AKVS_KV_Q4 || FMT == AKVS_KV_Q2)
-          if (copy_rec) cp_async4s(dst + head_code_bytes + c * 4, rec_p + (size_t)m.x * rec_row_bytes);
+          if (copy_rec) cp_async4s(dst + head_code_bytes + c * 4, rec_p + (uint64_t)m.x * rec_row_bytes);
       }
     }
   };
@@ -729,14 +729,14 @@ correct_kernel(KvLayer kv, const int4* __restrict__ tok_meta, const int32_t* __r
     cp_async_commit();
   }
 
-  float2 C2[V / 2], NS2[V / 2], ML2[V / 2], MH2[V / 2];   // (cos, cos), (-sin, -sin), offsets of the lower / upper chunk
+  float2 C2[V / 2], S2[V / 2], NS2[V / 2], ML2[V / 2], MH2[V / 2];   // (cos, cos), (sin, sin), (-sin, -sin), offsets of the lower / upper chunk
   int cur_unit = -1;
-  uint32_t slot = ring0;
-  for (int q = 0; q < n_q; ++q) {
+  uint32_t slot = ring0, meta_q = meta_a;
+  for (int q = 0; q < n_q; ++q, meta_q += meta_step) {
     cp_async_wait<COR_DEPTH - 1>();                     // everything up to this token's copies has landed
     __syncwarp();                                       // ... for every lane of the head's group
     if (q < n_mine) {
-      const uint4 m = lds128(meta_a + (uint32_t)q * meta_step);
+      const uint4 m = lds128(meta_q);
       if ((int)m.y >= 0) {                              // a fresh row: the bytes as they are
         *reinterpret_cast<uint4*>(out_p) = lds128(slot + c * 16);
         *reinterpret_cast<uint4*>(out_p + hi_off) = lds128(slot + c * 16 + hi_off);
@@ -749,6 +749,7 @@ correct_kernel(KvLayer kv, const int4* __restrict__ tok_meta, const int32_t* __r
 #pragma unroll
             for (int i = 0; i < V / 2; ++i) {
               C2[i] = make_float2(rot[2 * i].x, rot[2 * i + 1].x);
+              S2[i] = make_float2(rot[2 * i].y, rot[2 * i + 1].y);
               NS2[i] = make_float2(-rot[2 * i].y, -rot[2 * i + 1].y);
             }
           }
@@ -773,14 +774,12 @@ correct_kernel(KvLayer kv, const int4* __restrict__ tok_meta, const int32_t* __r
         const float w = __uint_as_float(m.w);
         const float2 W2 = make_float2(w, w);
         if (role == 0) {
-          // lo' = a cos - b sin + w mu_lo,  hi' = b cos + a sin + w mu_hi   (NS2 = -sin)
+          // lo' = a cos - b sin + w mu_lo,  hi' = b cos + a sin + w mu_hi
 #pragma unroll
           for (int i = 0; i < V / 2; ++i) {
             const float2 a2 = lo[i], b2 = hi[i];
             lo[i] = fma2(b2, NS2[i], fma2(W2, ML2[i], mul2(a2, C2[i])));
-            const float2 t = fma2(W2, MH2[i], mul2(b2, C2[i]));
-            const float2 u = mul2(a2, NS2[i]);
-            hi[i] = add2(t, make_float2(-u.x, -u.y));
+            hi[i] = fma2(a2, S2[i], fma2(W2, MH2[i], mul2(b2, C2[i])));
           }
         } else {
 #pragma unroll
