@@ -387,6 +387,9 @@ def main():
         ps.ms_step = timed(step, args.steps, 0)
         ps.ms_median, ps.ms_best = float(np.median(step_times)), float(min(step_times))
         ps.launches = akvs.launch_count() - launches0 + graph_launches * args.steps
+        # the per-kernel events are recorded at launch time, so this pass launches eagerly even when
+        # the timed steps replayed a graph
+        g_timed, ps.graph = ps.graph, None
         akvs.prof_enable((1 << 1) | (1 << 2) | (1 << 3) | (1 << 4) | (1 << 5), 8192)
         step()
         barrier()
@@ -395,6 +398,7 @@ def main():
         ps.clocks = sampler.stop()
         recs = akvs.prof_read()
         akvs.prof_enable(0)
+        ps.graph = g_timed
         assert akvs.check(ps.ws) == 0
         ps.P = ps.probes.n_probe_rows
 

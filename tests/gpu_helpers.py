@@ -17,6 +17,14 @@ def t2n(t):
     return t.detach().float().cpu().numpy().astype(np.float64)
 
 
+def both_16bit(x):
+    """Values representable in bfloat16 AND in float16: round to bf16, then to float16 (which
+    only touches magnitudes under 2^-17 and keeps them bf16-representable).  Inputs rounded this
+    way can be given unchanged to a model in either 16-bit storage type."""
+    r = testgen.bf16_round(np.asarray(x, np.float32))
+    return r.astype(np.float16).astype(np.float64)
+
+
 class Case:
     """A workload instantiated on both sides."""
 

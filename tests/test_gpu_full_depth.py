@@ -38,7 +38,7 @@ import torch
 
 import testgen
 from oracle import akvs_oracle as orc
-from gpu_helpers import Case, t2n
+from gpu_helpers import Case, t2n, both_16bit
 from helpers import SEED_W, make_inputs
 
 pytestmark = pytest.mark.gpu
@@ -59,13 +59,6 @@ def _workload(name):
     base, n_layers, n_units, _ = FULL[name]
     # "f16" weight values: the configuration's bf16 values, representable in both 16-bit types
     return testgen.reduced(testgen.workload(base), n_layers=n_layers, n_units=n_units, dtype="f16")
-
-
-def _both_16bit(x):
-    """Values representable in bfloat16 and in float16: round to bf16, then to float16 (which
-    only touches magnitudes under 2^-17 and keeps them bf16-representable)."""
-    r = testgen.bf16_round(np.asarray(x, np.float32))
-    return r.astype(np.float16).astype(np.float64)
 
 
 @functools.lru_cache(maxsize=1)
@@ -90,7 +83,7 @@ def _golden(name):
     if fmt == 0:
         # keep the unrounded encoding for the check of the library's own encoder
         fresh_units = [{"K": u["K"], "V": u["V"]} for u in units]
-        units = [{"K": _both_16bit(u["K"]), "V": _both_16bit(u["V"])} for u in units]
+        units = [{"K": both_16bit(u["K"]), "V": both_16bit(u["V"])} for u in units]
     t2 = time.time()
     ctx = np.concatenate(units_ids)
     ref = orc.corrected_reuse(omodel, units, list(range(len(units))), ctx, qry, w.refresh_bp[0], CHECK_LAYER)

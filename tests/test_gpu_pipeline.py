@@ -13,7 +13,7 @@ import torch
 
 import testgen
 from oracle import akvs_oracle as orc
-from gpu_helpers import Case, t2n, max_layer_err
+from gpu_helpers import Case, t2n, max_layer_err, both_16bit
 
 pytestmark = pytest.mark.gpu
 
@@ -111,6 +111,34 @@ def test_small16_all_modes(dtype, scale):
     case = Case(small16(dtype), std_scale=scale)
     units = _check_encode(case, case.tol)
     _run_all_modes(case, 2500, 2, units)
+
+
+def test_small16_bf16_storage_at_weight_scale_4_tracks_float16_by_the_roundoff_ratio():
+    """The case bfloat16 storage does NOT pass at 1e-2 (sharp softmax at 4x weight scale): instead
+    of leaving it out, both storage types run on identical inputs (bf16-valued weights and cache)
+    and the bfloat16 error is held to the first-order bound 12 x the float16 error of the same
+    tensor (unit roundoff 2^-8 against 2^-11 = 8x, times 1.5 for the spread of the rounding noise)
+    and to 5e-2 absolutely; float16 meets the benchmark spec's 1e-2."""
+    w = small16("f16")
+    errs = {}
+    ref = None
+    for dtype in ("f16", "bf16"):
+        case = Case(w, std_scale=4.0, gpu_dtype=dtype)
+        if ref is None:
+            units = [{"K": both_16bit(u["K"]), "V": both_16bit(u["V"])} for u in case.oracle_units()]
+            ref = orc.corrected_reuse(case.omodel, units, list(case.order), case.ctx, case.qry, 2500, 2)
+        case.load_oracle_cache(units)
+        probes, ctx, ws = case.gpu_select(2500, 2)
+        case.set_probes(probes, ref["probes"])
+        hid, k, v = case.gpu_prefill(case.akvs.MODE_CORRECTED, ws, probes, ctx, 2)
+        case.akvs.free(ctx)
+        errs[dtype] = (orc.rel_l2(hid, ref["hidden"]), max_layer_err(k, ref["K"]), max_layer_err(v, ref["V"]))
+    print("rel L2 (hidden, K, V): f16", errs["f16"], "bf16", errs["bf16"],
+          "ratio", [b / a for a, b in zip(errs["f16"], errs["bf16"])])
+    assert max(errs["f16"]) < 1e-2
+    assert max(errs["bf16"]) < 5e-2
+    for a, b in zip(errs["f16"], errs["bf16"]):
+        assert b < 12.0 * max(a, 2e-4)
 
 
 @pytest.mark.parametrize("dtype,scale", SMALL16)
