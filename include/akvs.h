@@ -212,6 +212,21 @@ int32_t akvs_check(void* workspace, void* stream);
 int32_t akvs_op_linear(int32_t dtype, const void* x, const void* w, void* y,
                        int32_t M, int32_t N, int32_t K, int32_t algo, void* stream);
 
+/* h[M][N] (float, read and written) += x[M][K] * w[N][K]^T: the residual form of the linear
+ * layers after attention and after the MLP (the decoder layer of the models the paper serves;
+ * the paper itself only says the probes are "recomputed", Algorithm 1).  algo as above.
+ * splits (tensor-core kernel only): the k range is cut into that many work items per output
+ * tile, each adding its partial sum into h with a vector reduction at the L2 - 0 lets the
+ * library choose (it splits launches that would leave SMs idle), 1..4 force the count
+ * (AKVS_ERR_SHAPE when K holds fewer 64-wide slabs than that).  With more than one split the
+ * order in which partial sums reach an element is not fixed, so results may differ in the last
+ * bit from run to run.  Errors: AKVS_ERR_INVALID_ARG (null pointer, bad size, splits outside
+ * 0..4), AKVS_ERR_SHAPE (16-bit: N not a multiple of 128, K not of 8), AKVS_ERR_UNSUPPORTED
+ * (dtype; splits > 1 on the CUDA-core kernel). */
+int32_t akvs_op_linear_residual(int32_t dtype, const void* x, const void* w, float* h,
+                                int32_t M, int32_t N, int32_t K, int32_t algo, int32_t splits,
+                                void* stream);
+
 /* Rotate-half RoPE in place on x[n][n_heads][head_dim] at positions pos[n] (device). */
 int32_t akvs_op_rope(int32_t dtype, void* x, const int32_t* pos, int32_t n, int32_t n_heads,
                      int32_t head_dim, float rope_base, void* stream);
@@ -308,8 +323,9 @@ int32_t akvs_op_quantize(int32_t dtype, const void* x, int32_t n, int32_t n_kv_h
 /* Cross-check switch for the tests: bit 0 set routes the 16-bit linear layers, bit 1 set the
  * 16-bit attention, to the CUDA-core kernels instead of the tcgen05 ones (default 0: tensor
  * cores for both).  Bits 2-3: tiling of the tcgen05 linear layers - 0 picked by shape
- * (default), 1 single CTAs, 2 CTA pairs wherever M > 128.  Process-wide; not part of the
- * serving surface. */
+ * (default), 1 single CTAs, 2 CTA pairs wherever M > 128.  Bits 4-6: split-K of the residual
+ * linear layers - 0 by the library's cost model (default), 1..4 that many splits.
+ * Process-wide; not part of the serving surface. */
 int32_t akvs_debug_set_linear_algo(int32_t algo);
 
 /* Number of kernels this library has launched in this process so far. */

@@ -24,7 +24,7 @@ MODE_CORRECTED, MODE_NAIVE, MODE_FULL = 0, 1, 2
 
 EXPORTS = ["akvs_workspace_bytes", "akvs_debug_set_linear_algo", "akvs_launch_count", "akvs_prof_enable",
            "akvs_prof_reset", "akvs_prof_read", "akvs_encode_units", "akvs_select_probes", "akvs_prefill_corrected",
-           "akvs_free", "akvs_check", "akvs_op_linear", "akvs_op_rope", "akvs_op_attention",
+           "akvs_free", "akvs_check", "akvs_op_linear", "akvs_op_linear_residual", "akvs_op_rope", "akvs_op_attention",
            "akvs_op_scratch_bytes", "akvs_op_select", "akvs_op_select_static", "akvs_op_correct_layer",
            "akvs_op_quantize", "akvs_op_residual_stats", "akvs_debug_correct_repeat", "akvs_debug_wait_timeout"]
 STATIC_MAX_CTX, STATIC_MAX_UNITS = 16384, 1024
@@ -357,6 +357,17 @@ def op_linear(x, w, algo=0):
     y = torch.empty((M, N), dtype=x.dtype, device=x.device)
     _chk(lib.akvs_op_linear(dtype, _ptr(x), _ptr(w), _ptr(y), M, N, K, algo, _stream()), "akvs_op_linear")
     return y
+
+
+def op_linear_residual(x, w, h, algo=0, splits=0):
+    """h (float32 [M][N], in place) += x w^T."""
+    dtype = _dt(x)
+    M, K = x.shape
+    N = w.shape[0]
+    assert h.dtype == torch.float32 and tuple(h.shape) == (M, N) and h.is_contiguous()
+    _chk(lib.akvs_op_linear_residual(dtype, _ptr(x), _ptr(w), _ptr(h), M, N, K, algo, splits, _stream()),
+         "akvs_op_linear_residual")
+    return h
 
 
 def op_rope(x, pos, base):

@@ -165,6 +165,7 @@ struct Ctx {                   // host object that carries a request from select
 // ----------------------------------------------------------------------------- linear layers
 int g_bf16_linear_algo = 0;    // 16-bit models: 0 = tcgen05; 1 = CUDA cores (kept for cross-checking)
 int g_linear_tiling = 0;       // tcgen05 linear layers: 0 = by shape; 1 = single CTAs; 2 = CTA pairs (cross-checking)
+int g_linear_splits = 0;       // residual linear layers: 0 = split-K by the cost model; 1..4 = forced (comparisons)
 
 // Projections that share the input x.  Segments whose bit is set in rope_mask are [M][heads][hd]
 // tensors that get RoPE at pos[row]: fused into the tensor-core epilogue when hd == 128,
@@ -189,11 +190,16 @@ int32_t linear_multi(const Dims& D, const void* x, int M, int K, int n_seg, cons
         AKVS_TRY(launch_rope(D.dtype, out[i], pos, M, n[i] / D.hd, D.hd, ldc[i], rope, n_pos, status, rope_base, st));
   return AKVS_OK;
 }
+// split_ok: the k range may be cut into ordered partial sums where that fills the device.  Off
+// for the unit encoder and the dense front, whose K/V of a unit at offset 0 are then the same
+// bits (one accumulation chain per element whatever the launch shape), so that such a unit scores
+// exactly zero at the check layer, as in exact arithmetic.
 int32_t linear_resid(const Dims& D, const void* x, int M, int K, const void* w, int n, float* h, int32_t* status,
-                     cudaStream_t st) {
+                     cudaStream_t st, bool split_ok) {
   if (D.dtype != AKVS_F32 && g_bf16_linear_algo == 0 && K % 8 == 0 && n % 128 == 0) {
     void* out = h;
-    return launch_linear_tc(D.dtype, 1, x, M, K, 1, &w, &n, &out, &n, status, st, nullptr, nullptr, 0, g_linear_tiling);
+    return launch_linear_tc(D.dtype, 1, x, M, K, 1, &w, &n, &out, &n, status, st, nullptr, nullptr, 0, g_linear_tiling, 0,
+                            split_ok ? g_linear_splits : 1);
   }
   return launch_linear_simt(D.dtype, x, w, nullptr, nullptr, h, M, n, K, n, st);
 }
@@ -234,7 +240,7 @@ int32_t attention(const Dims& D, const void* q, const void* k, const void* v, vo
 
 int32_t run_layer(const akvs_model_desc* m, const Dims& D, int l, const Workspace& ws, int n, const RowGeom& g,
                   void* k_dst, void* v_dst, const void* attn_k, const void* attn_v, int n_keys,
-                  const std::function<int32_t()>& between, cudaStream_t st) {
+                  const std::function<int32_t()>& between, cudaStream_t st, bool split_ok = false) {
   if (n == 0) return between ? between() : AKVS_OK;
   AKVS_TRY(launch_rmsnorm(D.dtype, ws.h, m->attn_norm[l], m->rms_eps, n, D.d, ws.x, st));
   {
@@ -246,10 +252,10 @@ int32_t run_layer(const akvs_model_desc* m, const Dims& D, int l, const Workspac
   }
   if (between) AKVS_TRY(between());
   AKVS_TRY(attention(D, ws.q, attn_k, attn_v, ws.ao, g, n, n_keys, ws.status, st));
-  AKVS_TRY(linear_resid(D, ws.ao, n, D.dq, m->wo[l], D.d, ws.h, ws.status, st));
+  AKVS_TRY(linear_resid(D, ws.ao, n, D.dq, m->wo[l], D.d, ws.h, ws.status, st, split_ok));
   AKVS_TRY(launch_rmsnorm(D.dtype, ws.h, m->mlp_norm[l], m->rms_eps, n, D.d, ws.x, st));
   AKVS_TRY(linear_swiglu(D, ws.x, n, D.d, m->w_gate[l], m->w_up[l], D.f, ws.act, ws.status, st));
-  AKVS_TRY(linear_resid(D, ws.act, n, D.f, m->w_down[l], D.d, ws.h, ws.status, st));
+  AKVS_TRY(linear_resid(D, ws.act, n, D.f, m->w_down[l], D.d, ws.h, ws.status, st, split_ok));
   return AKVS_OK;
 }
 
@@ -462,6 +468,8 @@ int32_t akvs_debug_set_linear_algo(int32_t algo) {
   g_attention_algo = (algo >> 1) & 1;
   g_linear_tiling = (algo >> 2) & 3;
   if (g_linear_tiling == 3) g_linear_tiling = 0;
+  g_linear_splits = (algo >> 4) & 7;
+  if (g_linear_splits > 4) g_linear_splits = 0;
   return AKVS_OK;
 }
 
@@ -727,7 +735,8 @@ int32_t akvs_prefill_corrected(const akvs_model_desc* model, const akvs_cache* c
       return launch_correct(D.dtype, kv, maps, ws.k, ws.v, corrected, ws.mu_k, ws.mu_v, N, nq, D.nkv, D.hd, ws.rope,
                             ok + l * kv_l, ov + l * kv_l, st);
     };
-    AKVS_TRY(run_layer(model, D, l, ws, R, geom, ws.k, ws.v, ok + l * kv_l, ov + l * kv_l, T, assemble, st));
+    AKVS_TRY(run_layer(model, D, l, ws, R, geom, ws.k, ws.v, ok + l * kv_l, ov + l * kv_l, T, assemble, st,
+                       /*split_ok=*/true));
   }
   return launch_rmsnorm(AKVS_F32, ws.h + (size_t)P * D.d, model->final_norm, model->rms_eps, nq, D.d, out_hidden, st);
 }
@@ -793,6 +802,22 @@ int32_t akvs_op_linear(int32_t dtype, const void* x, const void* w, void* y, int
                             algo == 0 ? 0 : algo - 1);
   }
   return launch_linear_simt(dtype, x, w, nullptr, y, nullptr, M, N, K, N, st);
+}
+
+int32_t akvs_op_linear_residual(int32_t dtype, const void* x, const void* w, float* h, int32_t M, int32_t N, int32_t K,
+                                int32_t algo, int32_t splits, void* stream) {
+  if (!x || !w || !h || M < 0 || N <= 0 || K <= 0 || splits < 0 || splits > 4) return AKVS_ERR_INVALID_ARG;
+  if (dtype != AKVS_F32 && dtype != AKVS_BF16 && dtype != AKVS_F16) return AKVS_ERR_UNSUPPORTED;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  if (algo < 0 || algo > 3) return AKVS_ERR_INVALID_ARG;
+  if (dtype != AKVS_F32 && algo != 1) {
+    if (N % 128 != 0 || K % 8 != 0) return AKVS_ERR_SHAPE;
+    void* out = h;
+    return launch_linear_tc(dtype, 1, x, M, K, 1, &w, &N, &out, &N, nullptr, st, nullptr, nullptr, 0,
+                            algo == 0 ? 0 : algo - 1, 0, splits);
+  }
+  if (splits > 1) return AKVS_ERR_UNSUPPORTED;
+  return launch_linear_simt(dtype, x, w, nullptr, nullptr, h, M, N, K, N, st);
 }
 
 int32_t akvs_op_rope(int32_t dtype, void* x, const int32_t* pos, int32_t n, int32_t n_heads, int32_t head_dim,

@@ -240,10 +240,12 @@ int32_t launch_linear_simt(int dtype, const void* x, const void* w, const void* 
 // rope[pos[row]] in the epilogue (rope: [n_pos][64] (cos, sin); null = no rotation; a position
 // outside [0, n_pos) raises AKVS_ERR_INVALID_ARG in the status word and rotates by position 0).
 // tiling 0: single CTAs or CTA pairs, whichever the shape favours; 1: single CTAs; 2: pairs (M > 128).
+// splits_force (epi 1): 0 = the k range is split over work items where a cost model favours it
+// (launches that would leave SMs idle); 1..4 = exactly that many splits.
 int32_t launch_linear_tc(int dtype, int epi, const void* x, int M, int K, int n_seg, const void* const* w, const int* n,
                          void* const* out, const int* ldc, int32_t* status, cudaStream_t st,
                          const float2* rope = nullptr, const int32_t* pos = nullptr, int rope_mask = 0, int tiling = 0,
-                         int n_pos = 0);
+                         int n_pos = 0, int splits_force = 0);
 
 // tcgen05 attention (attn_tc.cu): 16-bit types, head_dim 128.
 int32_t launch_attention_tc(int dtype, const void* q, const void* k, const void* v, void* out, const int32_t* k_lo,

@@ -52,7 +52,67 @@ struct GemmParams {
   int rope_mask;
   int n_pos;              // rows of the rope table: a position outside [0, n_pos) (positions may be caller
                           // data) raises AKVS_ERR_INVALID_ARG and is rotated as position 0
+  // split-K (EPI_RESID only: its epilogue adds into h at the L2, so partial sums over k ranges
+  // need no second pass): work item i = (split i / n_tiles, tile i % n_tiles); a split covers
+  // k slabs [split * kb_split, min(KB, (split + 1) * kb_split)), never empty
+  int splits, kb_split;
+  // Ordered partial sums: the epilogue warps of split s of a tile start adding only when all
+  // split_warps epilogue warps of every earlier split of that tile have added theirs (a counter
+  // per tile, back at zero when the launch ends), so every element receives its partial sums in
+  // the same order on every run.
+  unsigned int* split_count;
+  int split_warps;
 };
+
+constexpr int SPLITK_MAX_TILES = 8192;
+#ifndef AKVS_SPLIT_MIN_KB
+#define AKVS_SPLIT_MIN_KB 32
+#endif
+// One counter per output tile of the split launch in flight.  File-scope device memory, so a
+// single-step call needs no workspace; like the rest of the library's process-wide state it
+// assumes one stream of launches per device at a time.
+__device__ unsigned int g_splitk_count[SPLITK_MAX_TILES];
+
+// Bounded wait until *c >= target.  False when the limit ran out or the CTA is aborting.
+__device__ __forceinline__ bool wait_count(const unsigned int* c, unsigned int target, volatile int* abort_flag) {
+  const long long t0 = clock64();
+  for (uint32_t it = 0;; ++it) {
+    unsigned int v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(c) : "memory");
+    if (v >= target) return true;
+    __nanosleep(64);
+    if ((it & 63) == 63 && (*abort_flag || clock64() - t0 > tc::kWaitCycles)) return false;
+  }
+}
+
+// Before the epilogue of a split work item: wait for the tile's earlier splits.
+__device__ __forceinline__ bool split_turn(const GemmParams& p, int item, int n_tiles, int lane, volatile int* abort_flag) {
+  const int split = item / n_tiles;
+  if (split == 0) return true;
+  int got = 1;
+  if (lane == 0) got = wait_count(p.split_count + (item - split * n_tiles), (unsigned)(split * p.split_warps), abort_flag);
+  return __shfl_sync(0xffffffffu, got, 0) != 0;
+}
+// After it: this warp's reductions are performed, then the tile's count moves; the launch's last
+// arrival puts it back to zero.
+__device__ __forceinline__ void split_done(const GemmParams& p, int tile, int lane) {
+  __threadfence();
+  __syncwarp();
+  if (lane == 0) {
+    unsigned int* c = p.split_count + tile;
+    const unsigned int old = atomicAdd(c, 1u);
+    if (old + 1u == (unsigned)(p.splits * p.split_warps)) atomicExch(c, 0u);
+  }
+}
+
+// Tile and k-slab range of work item `item`.
+__device__ __forceinline__ void item_range(const GemmParams& p, int item, int n_tiles, int KB, int& tile, int& kb0,
+                                           int& kb1) {
+  const int split = item / n_tiles;
+  tile = item - split * n_tiles;
+  kb0 = split * p.kb_split;
+  kb1 = kb0 + p.kb_split < KB ? kb0 + p.kb_split : KB;
+}
 
 // Which weight matrix and which of its rows the 128-row block `block` of the concatenated
 // output columns comes from.  Past the last matrix the row lies beyond its extent and the
@@ -237,6 +297,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int KB = (p.K + BK - 1) / BK;
   const int n_tiles = p.tiles_m * p.tiles_n;
+  const int n_items = n_tiles * p.splits;
   pdl_trigger();
 
   if (threadIdx.x == 0) {
@@ -279,31 +340,35 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       // weight tiles of the first stages (every stage is free at the start: no wait), then the
       // dependency on the earlier kernels, then the activation tiles of the same stages
       const uint32_t stage_tx = A_BYTES + p.nh * BH_BYTES;
-      const int pre = blockIdx.x < n_tiles ? (KB < STAGES ? KB : STAGES) : 0;
+      int tile0 = 0, kbf0 = 0, kbf1 = 0;                  // the CTA's first work item
+      if (blockIdx.x < n_items) item_range(p, blockIdx.x, n_tiles, KB, tile0, kbf0, kbf1);
+      const int pre = kbf1 - kbf0 < STAGES ? kbf1 - kbf0 : STAGES;
       if (pre > 0) {
         const CUtensorMap *m0, *m1;
         int row0, row1;
-        b_tiles(blockIdx.x, m0, m1, row0, row1);
+        b_tiles(tile0, m0, m1, row0, row1);
         for (int kb = 0; kb < pre; ++kb) {
           uint8_t* st = smem + kb * STAGE_BYTES;
           tc::mbar_expect_tx(&full[kb], stage_tx);
-          tc::tma_load_2d(st + A_BYTES, m0, kb * BK, row0, &full[kb]);
-          if (p.nh == 2) tc::tma_load_2d(st + A_BYTES + BH_BYTES, m1, kb * BK, row1, &full[kb]);
+          tc::tma_load_2d(st + A_BYTES, m0, (kbf0 + kb) * BK, row0, &full[kb]);
+          if (p.nh == 2) tc::tma_load_2d(st + A_BYTES + BH_BYTES, m1, (kbf0 + kb) * BK, row1, &full[kb]);
         }
       }
       pdl_wait();
       for (int kb = 0; kb < pre; ++kb)
-        tc::tma_load_2d(smem + kb * STAGE_BYTES, &tmA, kb * BK, (blockIdx.x % p.tiles_m) * BM, &full[kb]);
+        tc::tma_load_2d(smem + kb * STAGE_BYTES, &tmA, (kbf0 + kb) * BK, (tile0 % p.tiles_m) * BM, &full[kb]);
       int s = pre % STAGES;
       uint32_t ph = pre == STAGES ? 1u : 0u;
       int kb_start = pre;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+      for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
+        int tile, kb0, kb1;
+        item_range(p, item, n_tiles, KB, tile, kb0, kb1);
         const int tm = tile % p.tiles_m;
         const CUtensorMap *m0, *m1;
         int row0, row1;
         b_tiles(tile, m0, m1, row0, row1);
-        for (int kb = kb_start; kb < KB; ++kb) {
+        for (int kb = kb0 + kb_start; kb < kb1; ++kb) {
           if (!tc::mbar_wait(&empty[s], ph ^ 1, abort_flag)) { ok = false; break; }
           uint8_t* st = smem + s * STAGE_BYTES;
           tc::mbar_expect_tx(&full[s], stage_tx);
@@ -324,12 +389,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       uint32_t ph = 0;
       bool ok = true;
       int it = 0;
-      for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++it) {
+      for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++it) {
+        int tile, kb0, kb1;
+        item_range(p, item, n_tiles, KB, tile, kb0, kb1);
         const int acc = it & 1;
         if (!tc::mbar_wait(&acc_empty[acc], ((it >> 1) & 1) ^ 1, abort_flag)) { ok = false; break; }
         tc::fence_after_sync();
         const uint32_t d_tmem = tmem_base + acc * (2 * BNH);
-        for (int kb = 0; kb < KB; ++kb) {
+        for (int kb = kb0; kb < kb1; ++kb) {
           if (!tc::mbar_wait(&full[s], ph, abort_flag)) { ok = false; break; }
           tc::fence_after_sync();
           const uint32_t a_addr = tc::smem_u32(smem + s * STAGE_BYTES);
@@ -338,7 +405,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           for (int k = 0; k < BK / 16; ++k) {
             const uint64_t da = tc::smem_desc_k_sw128(a_addr + k * 32);
             const uint64_t db = tc::smem_desc_k_sw128(b_addr + k * 32);
-            tc::mma_f16(d_tmem, da, db, idesc, (kb | k) != 0);
+            tc::mma_f16(d_tmem, da, db, idesc, kb > kb0 || k != 0);
           }
           tc::mma_commit(&empty[s]);            // frees the stage once these MMAs retire
           if (++s == STAGES) { s = 0; ph ^= 1; }
@@ -353,17 +420,20 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     pdl_wait();                                // outputs, residual and positions are other kernels' memory
     bool ok = true;
     int it = 0;
-    for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++it) {
+    for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++it) {
+      const int tile = item % n_tiles;
       const int acc = it & 1;
       const int tn = tile / p.tiles_m, tm = tile % p.tiles_m;
       if (!tc::mbar_wait(&acc_full[acc], (it >> 1) & 1, abort_flag)) { ok = false; break; }
       tc::fence_after_sync();
+      if (EPI == EPI_RESID && p.splits > 1 && !split_turn(p, item, n_tiles, lane, abort_flag)) { ok = false; break; }
       const uint32_t t_addr = tmem_base + acc * (2 * BNH) + ((uint32_t)(quad * 32) << 16);
       if (EPI == EPI_SWIGLU)
         epilogue_swiglu_row<T>(p, t_addr, tm * BM + quad * 32 + lane, tn);
       else
         epilogue_warp<EPI, T>(p, t_addr, tm * BM + quad * 32, lane, tn, p.nh,
                               smem + STAGES * STAGE_BYTES + 256 + (warp - 2) * EPI_STAGE_BYTES);
+      if (EPI == EPI_RESID && p.splits > 1) split_done(p, tile, lane);
       tc::fence_before_sync();
       __syncwarp();
       if (lane == 0) tc::mbar_arrive(&acc_empty[acc]);
@@ -422,6 +492,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
   const int KB = (p.K + BK - 1) / BK;
   const int n_tiles = p.tiles_m * p.tiles_n;            // tiles_m counts 256-row tiles here
+  const int n_items = n_tiles * p.splits;
   pdl_trigger();
 
   if (threadIdx.x == 0) {
@@ -459,29 +530,34 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       };
       uint32_t full0[STAGES2];                // rank 0's full barriers as shared::cluster addresses
       for (int i = 0; i < STAGES2; ++i) full0[i] = tc::map_to_rank(tc::smem_u32(&full[i]), 0);
-      const int pre = pair < n_tiles ? (KB < STAGES2 ? KB : STAGES2) : 0;
+      int tile0 = 0, kbf0 = 0, kbf1 = 0;                  // the pair's first work item
+      if (pair < n_items) item_range(p, pair, n_tiles, KB, tile0, kbf0, kbf1);
+      const int pre = kbf1 - kbf0 < STAGES2 ? kbf1 - kbf0 : STAGES2;
       if (pre > 0) {
         const CUtensorMap* m;
         int row;
-        b_half(pair, m, row);
+        b_half(tile0, m, row);
         for (int kb = 0; kb < pre; ++kb) {
           if (rank == 0) tc::mbar_expect_tx(&full[kb], 2 * STAGE2_BYTES);
-          tc::tma_load_2d_pair(smem + kb * STAGE2_BYTES + A_BYTES, m, kb * BK, row, full0[kb]);
+          tc::tma_load_2d_pair(smem + kb * STAGE2_BYTES + A_BYTES, m, (kbf0 + kb) * BK, row, full0[kb]);
         }
       }
       pdl_wait();
       for (int kb = 0; kb < pre; ++kb)
-        tc::tma_load_2d_pair(smem + kb * STAGE2_BYTES, &tmA, kb * BK, ((pair % p.tiles_m) * 2 + (int)rank) * BM, full0[kb]);
+        tc::tma_load_2d_pair(smem + kb * STAGE2_BYTES, &tmA, (kbf0 + kb) * BK, ((tile0 % p.tiles_m) * 2 + (int)rank) * BM,
+                             full0[kb]);
       int s = pre % STAGES2;
       uint32_t ph = pre == STAGES2 ? 1u : 0u;
       int kb_start = pre;
       bool ok = true;
-      for (int tile = pair; tile < n_tiles && ok; tile += n_pairs) {
+      for (int item = pair; item < n_items && ok; item += n_pairs) {
+        int tile, kb0, kb1;
+        item_range(p, item, n_tiles, KB, tile, kb0, kb1);
         const int tm = tile % p.tiles_m;
         const CUtensorMap* m;
         int row;
         b_half(tile, m, row);
-        for (int kb = kb_start; kb < KB; ++kb) {
+        for (int kb = kb0 + kb_start; kb < kb1; ++kb) {
           if (!tc::mbar_wait(&empty[s], ph ^ 1, abort_flag)) { ok = false; break; }
           uint8_t* st = smem + s * STAGE2_BYTES;
           if (rank == 0) tc::mbar_expect_tx(&full[s], 2 * STAGE2_BYTES);
@@ -501,12 +577,14 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       uint32_t ph = 0;
       bool ok = true;
       int it = 0;
-      for (int tile = pair; tile < n_tiles && ok; tile += n_pairs, ++it) {
+      for (int item = pair; item < n_items && ok; item += n_pairs, ++it) {
+        int tile, kb0, kb1;
+        item_range(p, item, n_tiles, KB, tile, kb0, kb1);
         const int acc = it & 1;
         if (!tc::mbar_wait(&acc_empty[acc], ((it >> 1) & 1) ^ 1, abort_flag)) { ok = false; break; }
         tc::fence_after_sync();
         const uint32_t d_tmem = tmem_base + acc * (2 * BNH);
-        for (int kb = 0; kb < KB; ++kb) {
+        for (int kb = kb0; kb < kb1; ++kb) {
           if (!tc::mbar_wait(&full[s], ph, abort_flag)) { ok = false; break; }
           tc::fence_after_sync();
           const uint32_t a_addr = tc::smem_u32(smem + s * STAGE2_BYTES);
@@ -515,7 +593,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           for (int k = 0; k < BK / 16; ++k) {
             const uint64_t da = tc::smem_desc_k_sw128(a_addr + k * 32);
             const uint64_t db = tc::smem_desc_k_sw128(b_addr + k * 32);
-            tc::mma_f16_pair(d_tmem, da, db, idesc, (kb | k) != 0);
+            tc::mma_f16_pair(d_tmem, da, db, idesc, kb > kb0 || k != 0);
           }
           tc::mma_commit_pair(&empty[s], 3);            // frees the stage in both CTAs
           if (++s == STAGES2) { s = 0; ph ^= 1; }
@@ -532,11 +610,13 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     pdl_wait();
     bool ok = true;
     int it = 0;
-    for (int tile = pair; tile < n_tiles && ok; tile += n_pairs, ++it) {
+    for (int item = pair; item < n_items && ok; item += n_pairs, ++it) {
+      const int tile = item % n_tiles;
       const int acc = it & 1;
       const int tn = tile / p.tiles_m, tm = tile % p.tiles_m;
       if (!tc::mbar_wait(&acc_full[acc], (it >> 1) & 1, abort_flag)) { ok = false; break; }
       tc::fence_after_sync();
+      if (EPI == EPI_RESID && p.splits > 1 && !split_turn(p, item, n_tiles, lane, abort_flag)) { ok = false; break; }
       const uint32_t t_addr = tmem_base + acc * (2 * BNH) + ((uint32_t)(quad * 32) << 16);
       const int row0 = (tm * 2 + (int)rank) * BM + quad * 32;
       if (EPI == EPI_SWIGLU)
@@ -544,6 +624,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       else
         epilogue_warp<EPI, T>(p, t_addr, row0, lane, tn, 2,
                               smem + STAGES2 * STAGE2_BYTES + 256 + (warp - 2) * EPI_STAGE_BYTES);
+      if (EPI == EPI_RESID && p.splits > 1) split_done(p, tile, lane);
       tc::fence_before_sync();
       __syncwarp();
       if (lane == 0) tc::mbar_arrive_cluster(acc_empty0[acc]);
@@ -702,9 +783,10 @@ int32_t encode_tmap_3d_16bit(CUtensorMap* map, const void* base, uint64_t d0, ui
 // outputs go to out[i] with row stride ldc[i].
 //   epi 0: out[i] = x w[i]^T (16-bit);   epi 1: out[0] (float) += x w[0]^T;
 //   epi 2: out[0] = silu(x w[0]^T) * (x w[1]^T) (16-bit), n[0] == n[1].
+// splits_force (epi 1 only): 0 = the k range is split by the cost model; 1..4 = that many splits.
 int32_t launch_linear_tc(int dtype, int epi, const void* x, int M, int K, int n_seg, const void* const* w, const int* n,
                          void* const* out, const int* ldc, int32_t* status, cudaStream_t st, const float2* rope,
-                         const int32_t* pos, int rope_mask, int tiling, int n_pos) {
+                         const int32_t* pos, int rope_mask, int tiling, int n_pos, int splits_force) {
   if (M == 0) return AKVS_OK;
   if (K % 8 != 0 || n_seg < 1 || n_seg > 3) return AKVS_ERR_SHAPE;
   if (dtype != AKVS_BF16 && dtype != AKVS_F16) return AKVS_ERR_UNSUPPORTED;
@@ -748,55 +830,117 @@ int32_t launch_linear_tc(int dtype, int epi, const void* x, int M, int K, int n_
   }
   p.tiles_m = (M + BM - 1) / BM;
   p.nh = 2;
+  p.splits = 1;
+  p.split_count = nullptr;
+  p.split_warps = 4;
+  const int KB = (K + BK - 1) / BK;
+  p.kb_split = KB;
+  const int sms = sm_count();
+  // CTA pairs on 256x256 tiles: a tile takes the same number of MMA cycles as two 128x256 tiles
+  // of single CTAs, and the pair moves a third less operand data per SM (measured on the 8B
+  // shapes: main loop ~8 % faster under the power cap).  tiling 1 / 2 force single CTAs / pairs
+  // (tests, comparisons).
+  const int pairs = (tiling == 1 || M <= BM) ? 0 : pair_count();
+  bool use_pair = false;
   if (epi == EPI_SWIGLU) {
     if (n_seg != 2 || n[0] != n[1]) return AKVS_ERR_SHAPE;
     p.tiles_n = n[0] / BNH;
+  } else if (epi == EPI_RESID) {
+    // The residual epilogue adds into h at the L2, so the k range may be split over several work
+    // items at no extra pass.  Cost model in units of one 128x256x64 slab on one SM: rounds x
+    // (slabs per item x cost of a slab on that tiling + a per-item constant); a 128x128 tile's slab
+    // costs 0.62 (it reads as many shared-memory bytes per flop again), a pair's 0.92 per SM.
+    // A split keeps at least 32 slabs per item, so that an item's epilogue still fits under the
+    // next item's main loop; more splits must win by 3 % each.
+    double best = 1e30;
+    for (int pr = 0; pr < 2; ++pr) {
+      if (pr == 1 && pairs == 0) continue;
+      if (pr == 0 && tiling == 2 && pairs > 0) continue;
+      for (int nh = 1; nh <= 2; ++nh) {
+        if (pr == 1 && nh == 1) continue;
+        const int tiles = (pr ? (M + 2 * BM - 1) / (2 * BM) : p.tiles_m) * ((blocks + nh - 1) / nh);
+        const int cap = pr ? pairs : sms;
+        const double slab = pr ? 0.92 : (nh == 2 ? 1.0 : 0.62);
+        for (int sp = 1; sp <= 4; ++sp) {
+          if (splits_force > 0 && sp != splits_force) continue;
+          const int kbs = (KB + sp - 1) / sp;
+          if ((kbs + 0) * (sp - 1) >= KB && sp > 1) continue;      // the last split would be empty
+          if (splits_force == 0 && sp > 1 && kbs < AKVS_SPLIT_MIN_KB) continue;
+          const int rounds = (tiles * sp + cap - 1) / cap;
+          const double cost = rounds * (kbs * slab + 4.0) * (1.0 + 0.03 * (sp - 1));
+          if (cost < best) {
+            best = cost;
+            use_pair = pr == 1;
+            p.nh = nh;
+            p.splits = sp;
+            p.kb_split = kbs;
+          }
+        }
+      }
+    }
+    if (best >= 1e30) return AKVS_ERR_SHAPE;                     // a forced split count the k range cannot carry
+    p.tiles_n = (blocks + p.nh - 1) / p.nh;
+    if (p.splits > 1) {
+      const int tiles = (use_pair ? (M + 2 * BM - 1) / (2 * BM) : p.tiles_m) * p.tiles_n;
+      static unsigned int* counters[64] = {};
+      int dev = 0;
+      AKVS_CUDA(cudaGetDevice(&dev));
+      if (tiles > SPLITK_MAX_TILES || dev < 0 || dev >= 64) {
+        if (splits_force > 1) return AKVS_ERR_TOO_LARGE;
+        p.splits = 1;                                           // (only reachable with the tiling the model chose for 1 split
+        p.kb_split = KB;                                        //  being worse than another: correct, just not the fastest)
+      } else {
+        if (!counters[dev]) AKVS_CUDA(cudaGetSymbolAddress(reinterpret_cast<void**>(&counters[dev]), g_splitk_count));
+        p.split_count = counters[dev];
+        p.split_warps = use_pair ? 8 : 4;
+      }
+    }
   } else {
     // 128x128 tiles when that shortens the launch: a tile of half the width takes ~0.62 of the
-    // time (its MMAs read as many shared-memory bytes per flop again), rounds = tiles / SMs
-    const int sms = sm_count();
+    // time, rounds = tiles / SMs
     const int t2 = p.tiles_m * ((blocks + 1) / 2), t1 = p.tiles_m * blocks;
     const double cost2 = (double)((t2 + sms - 1) / sms), cost1 = 0.62 * ((t1 + sms - 1) / sms);
     if (cost1 < 0.9 * cost2) p.nh = 1;
     p.tiles_n = (blocks + p.nh - 1) / p.nh;
   }
+  if (epi != EPI_RESID && (p.nh == 2 || tiling == 2) && pairs > 0) {
+    // pairs when that takes no more rounds than single CTAs on 128x256 tiles
+    const int tiles_n2 = (blocks + 1) / 2;
+    const int tn = epi == EPI_SWIGLU ? p.tiles_n : tiles_n2;
+    const int t_pair = ((M + 2 * BM - 1) / (2 * BM)) * tn, t_single = p.tiles_m * tn;
+    const int r_pair = (t_pair + pairs - 1) / pairs, r_single = (t_single + sms - 1) / sms;
+    if (tiling == 2 || r_pair <= r_single) {
+      use_pair = true;
+      if (p.nh == 1) { p.nh = 2; p.tiles_n = tiles_n2; }
+    }
+  }
   double flops = 0;
   for (int i = 0; i < n_seg; ++i) flops += 2.0 * M * (double)n[i] * K;
   ProfScope prof(1, epi, flops, st);
   if (epi < 0 || epi > 2) return AKVS_ERR_INVALID_ARG;
-  // CTA pairs on 256x256 tiles when that takes no more rounds than single CTAs on 128x256 tiles:
-  // a tile takes the same number of MMA cycles either way, and the pair moves a third less
-  // operand data per SM (measured on the 8B shapes: main loop ~8 % faster under the power cap).
-  // tiling 1 / 2 force single CTAs / pairs (tests, comparisons).
-  const int pairs = tiling == 1 ? 0 : pair_count();
-  if ((p.nh == 2 || tiling == 2) && pairs > 0 && M > BM) {
-    if (p.nh == 1) { p.nh = 2; p.tiles_n = (blocks + 1) / 2; }
-    const int tiles_m2 = (M + 2 * BM - 1) / (2 * BM);
-    const int t_pair = tiles_m2 * p.tiles_n, t_single = p.tiles_m * p.tiles_n;
-    const int r_pair = (t_pair + pairs - 1) / pairs, r_single = (t_single + sm_count() - 1) / sm_count();
-    if (tiling == 2 || r_pair <= r_single) {
-      p.tiles_m = tiles_m2;
-      p.idesc = tc::idesc_f16(fmt, 2 * BM, 2 * BNH, 0);
-      const int n_pairs = t_pair < pairs ? t_pair : pairs;
+  if (use_pair) {
+    p.tiles_m = (M + 2 * BM - 1) / (2 * BM);
+    p.idesc = tc::idesc_f16(fmt, 2 * BM, 2 * BNH, 0);
+    const int items = p.tiles_m * p.tiles_n * p.splits;
+    const int n_pairs = items < pairs ? items : pairs;
 #define AKVS_GEMM_LAUNCH(E, T) \
   AKVS_CUDA(launch_pdl_pair(gemm_tc_pair_kernel<E, T>, dim3(2 * n_pairs), dim3(THREADS), SMEM2_BYTES, st, tmA, tmB[0], tmB[1], tmB[2], p))
-      if (dtype == AKVS_BF16) {
-        if (epi == EPI_STORE) AKVS_GEMM_LAUNCH(EPI_STORE, bf16);
-        else if (epi == EPI_RESID) AKVS_GEMM_LAUNCH(EPI_RESID, bf16);
-        else AKVS_GEMM_LAUNCH(EPI_SWIGLU, bf16);
-      } else {
-        if (epi == EPI_STORE) AKVS_GEMM_LAUNCH(EPI_STORE, f16);
-        else if (epi == EPI_RESID) AKVS_GEMM_LAUNCH(EPI_RESID, f16);
-        else AKVS_GEMM_LAUNCH(EPI_SWIGLU, f16);
-      }
-#undef AKVS_GEMM_LAUNCH
-      AKVS_LAUNCHED();
-      return AKVS_OK;
+    if (dtype == AKVS_BF16) {
+      if (epi == EPI_STORE) AKVS_GEMM_LAUNCH(EPI_STORE, bf16);
+      else if (epi == EPI_RESID) AKVS_GEMM_LAUNCH(EPI_RESID, bf16);
+      else AKVS_GEMM_LAUNCH(EPI_SWIGLU, bf16);
+    } else {
+      if (epi == EPI_STORE) AKVS_GEMM_LAUNCH(EPI_STORE, f16);
+      else if (epi == EPI_RESID) AKVS_GEMM_LAUNCH(EPI_RESID, f16);
+      else AKVS_GEMM_LAUNCH(EPI_SWIGLU, f16);
     }
+#undef AKVS_GEMM_LAUNCH
+    AKVS_LAUNCHED();
+    return AKVS_OK;
   }
   p.idesc = tc::idesc_f16(fmt, BM, p.nh * BNH, 0);
-  const int n_tiles = p.tiles_m * p.tiles_n;
-  const int grid = n_tiles < sm_count() ? n_tiles : sm_count();
+  const int n_items = p.tiles_m * p.tiles_n * p.splits;
+  const int grid = n_items < sm_count() ? n_items : sm_count();
 #define AKVS_GEMM_LAUNCH(E, T) \
   AKVS_CUDA(launch_pdl(gemm_tc_kernel<E, T>, dim3(grid), dim3(THREADS), SMEM_BYTES, st, tmA, tmB[0], tmB[1], tmB[2], p))
   if (dtype == AKVS_BF16) {

@@ -45,6 +45,33 @@ def test_linear_16bit(akvs, M, N, K, algo, dtype):
     assert np.abs(n64(y) - ref).max() <= ulp * np.abs(ref).max() + 1e-5
 
 
+@pytest.mark.parametrize("M,N,K", [(300, 256, 4096), (958, 2048, 11008), (130, 384, 2120), (77, 128, 136)])
+@pytest.mark.parametrize("algo", [0, 2, 3])         # by shape, single CTAs, CTA pairs
+@pytest.mark.parametrize("splits", [0, 1, 2, 3, 4])  # split-K: by the cost model, or forced
+@pytest.mark.parametrize("dtype", H16)
+def test_linear_residual_split_k(akvs, M, N, K, algo, splits, dtype):
+    """h += x W^T with the k range cut into work items that add into h at the L2: every split
+    count gives the plain sum (float accumulation; the ragged last 64-wide slab and a last split
+    shorter than the others included)."""
+    g = np.random.default_rng(M + N + K)
+    x = dev(g.standard_normal((M, K)).astype(np.float32), dtype)
+    w = dev((g.standard_normal((N, K)) * 0.05).astype(np.float32), dtype)
+    h0 = g.standard_normal((M, N)).astype(np.float32)
+    h = dev(h0)
+    slabs = (K + 63) // 64
+    if splits > 1 and (slabs + splits - 1) // splits * (splits - 1) >= slabs:
+        with pytest.raises(akvs.AkvsError):
+            akvs.op_linear_residual(x, w, h, algo, splits)
+        return
+    akvs.op_linear_residual(x, w, h, algo, splits)
+    again = dev(h0)
+    akvs.op_linear_residual(x, w, again, algo, splits)
+    torch.cuda.synchronize()
+    assert torch.equal(h, again)                     # partial sums arrive in a fixed order
+    ref = h0.astype(np.float64) + n64(x) @ n64(w).T
+    assert np.abs(n64(h) - ref).max() <= 1e-5 * np.abs(ref).max() * max(1.0, np.sqrt(K / 1024))
+
+
 @pytest.mark.parametrize("M,N,K", [(1, 1, 1), (65, 130, 33), (200, 688, 256)])
 def test_linear_f32(akvs, M, N, K):
     g = np.random.default_rng(M)
