@@ -241,6 +241,9 @@ def main():
     ap.add_argument("--dtype", default="f16", choices=["f16", "bf16"],
                     help="16-bit storage type of weights, cache and activations (weight VALUES are bf16 either way)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--kernel-switches", type=int, default=0,
+                    help="comparisons: the library's cross-check switch word (bits 2-3: tiling of the linear layers; "
+                         "bits 4-6: forced split-K count); recorded in config, 0 for any reported result")
     ap.add_argument("--no-variants", action="store_true", help="skip the pass with the other 16-bit storage type")
     ap.add_argument("--graph", action="store_true",
                     help="replay the corrected prefill from a CUDA graph captured once (selection stays eager)")
@@ -278,6 +281,8 @@ def main():
     import torch
     import torch.distributed as dist
     import paper_2607_21604_b200 as akvs
+    if args.kernel_switches:
+        akvs.lib.akvs_debug_set_linear_algo(int(args.kernel_switches))
 
     torch.cuda.set_device(local)
     if world > 1:
@@ -594,7 +599,7 @@ def main():
         "config": {"workload": f"{w.name}: {m.name}-class decoder L{m.n_layers} d{m.d_model} {m.n_q_heads}q/{m.n_kv_heads}kv "
                                f"hd{m.head_dim} ff{m.d_ff}; {M // B} units {w.len_lo}-{w.len_hi} tok (N={N // B}) + {nq // B} query"
                                + (f", batch of {B} requests per call" if B > 1 else ""),
-                   "batch": B, "cuda_graph": bool(args.graph),
+                   "batch": B, "cuda_graph": bool(args.graph), "kernel_switches": int(args.kernel_switches),
                    "refresh_bp": bp, "check_layer": CHECK_LAYER, "probe_rows": P, "rows_recomputed": P + nq,
                    "effective_refresh": P / max(1, N), "kv_format": w.kv_format, "parallelism": f"replicas x{world}",
                    "l2": f"inputs larger than L2: each step streams all layer weights ({weight_gb:.1f} GB)",

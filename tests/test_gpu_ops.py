@@ -82,6 +82,19 @@ def test_linear_f32(akvs, M, N, K):
     assert orc.rel_l2(n64(y), n64(x) @ n64(w).T) < 1e-6
 
 
+@pytest.mark.parametrize("M,N,K", [(1, 1, 1), (65, 130, 33), (200, 688, 256)])
+def test_linear_residual_f32(akvs, M, N, K):
+    g = np.random.default_rng(M + 1)
+    x = dev(g.standard_normal((M, K)).astype(np.float32))
+    w = dev(g.standard_normal((N, K)).astype(np.float32))
+    h0 = g.standard_normal((M, N)).astype(np.float32)
+    h = akvs.op_linear_residual(x, w, dev(h0))
+    torch.cuda.synchronize()
+    assert orc.rel_l2(n64(h), h0.astype(np.float64) + n64(x) @ n64(w).T) < 1e-6
+    with pytest.raises(akvs.AkvsError):
+        akvs.op_linear_residual(x, w, dev(h0), 0, 2)     # no split-K on the CUDA-core kernel
+
+
 @pytest.mark.parametrize("algo", [2, 3])
 @pytest.mark.parametrize("dtype", H16)
 def test_linear_16bit_full_size_sampled(akvs, dtype, algo):

@@ -155,6 +155,26 @@ def test_small16_all_modes_linear_layers_on_cta_pairs(dtype, scale):
         case.akvs.lib.akvs_debug_set_linear_algo(0)
 
 
+def wide16(dtype):
+    return testgen.Workload("wide16-" + dtype, testgen.ModelCfg("wide16", 4, 512, 4, 2, 128, 896, 512, dtype),
+                            5, 40, 90, 24, (2500,))
+
+
+@pytest.mark.parametrize("dtype,scale", SMALL16)
+@pytest.mark.parametrize("switches", [0, 2 << 2, (2 << 2) | (2 << 4), 3 << 4])
+def test_wide16_all_modes_tilings_and_split_k(dtype, scale, switches):
+    """A four-layer model of width 512 (d_ff 896 = 14 slabs of 64): every mode against the oracle
+    with the linear layers by shape, on CTA pairs, and with the residual layers' k range forced
+    into 2 (on pairs) and 3 ordered partial sums."""
+    case = Case(wide16(dtype), std_scale=scale)
+    case.akvs.lib.akvs_debug_set_linear_algo(switches)
+    try:
+        units = _check_encode(case, case.tol)
+        _run_all_modes(case, 2500, 2, units)
+    finally:
+        case.akvs.lib.akvs_debug_set_linear_algo(0)
+
+
 @pytest.mark.parametrize("kv_format", [4, 2])
 @pytest.mark.parametrize("dtype,scale", SMALL16)
 def test_small16_quantised_cache(kv_format, dtype, scale):
