@@ -580,6 +580,9 @@ def main():
             "correct_kernel_frac": p2.other["correct_kernel"]["frac"], "clocks": p2.clocks,
             "dtype": f"{other_dt} storage (weights, cache, activations, K/V outputs), f32 accumulate"}}
 
+    if world > 1:
+        dist.barrier()                     # every rank is past its last collective before any of them leaves
+        dist.destroy_process_group()
     if rank != 0:
         return
     cpu = None
