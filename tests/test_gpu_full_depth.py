@@ -1,6 +1,9 @@
 """Parity at the configurations as they are specified: full depth, full context, both 16-bit
 storage types.
 
+* config 2 (3B-class): all 36 layers, all 20 units (5219 context + 64 query tokens), 10 % refresh -
+  the configuration whose ~1000 recomputed rows make the residual linear layers split their k
+  range into ordered partial sums;
 * config 3 (the benchmarked one): all 32 layers, all 32 units (8593 context + 128 query tokens),
   15 % refresh, check layer 2;
 * config 5 with the 4-bit cache: all 32 layers, the first 16 of its 48 units (4096 context
@@ -49,6 +52,7 @@ CHECK_LAYER = 2
 
 # name -> (workload, layers, units, cache format)
 FULL = {
+    "c2": ("c2", None, None, 0),
     "c3": ("c3", None, None, 0),
     "c5q4": ("c5q4", None, 16, 4),
     "c4": ("c4", 8, 12, 0),
@@ -101,7 +105,7 @@ def _curve(label, errs):
 
 
 @pytest.mark.parametrize("dtype", ["f16", "bf16"])
-@pytest.mark.parametrize("name", ["c3", "c5q4", "c4"])
+@pytest.mark.parametrize("name", ["c2", "c3", "c5q4", "c4"])
 def test_full_depth_corrected_prefill(name, dtype):
     w, omodel, units, fresh_units, ref = _golden(name)
     fmt = FULL[name][3]
